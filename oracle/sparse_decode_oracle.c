@@ -1,0 +1,277 @@
+/*
+ * CPU oracle for query-aware sparse decode attention over a paged KV cache.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT PRODUCT CODE.  It exists so that the CUDA path can
+ * be checked against the paper's equations.  Only the tests, the smoke check and the
+ * CPU-baseline leg of the benchmark may call it.  It shares no code, header, table or
+ * helper with the CUDA library and is never a fallback for it.
+ *
+ * Everything is computed in fp64 on the bf16-rounded inputs (a bf16 value converts to
+ * double exactly), with plain loops in the order the paper's definitions give them:
+ *
+ *   se_oracle_meta     Quest page summaries            (Appendix A, Quest, summary eq.)
+ *   se_oracle_scores   Quest page score, group max     (Appendix A, Quest, score eq.)
+ *   se_oracle_topk     TopK_b(s; A)                    (Appendix A, notation table)
+ *   se_oracle_attend   attention over selected tokens  (Appendix A, selected-attention eq.)
+ *                      + H2O accumulated score         (Appendix A, H2O score eq.)
+ *
+ * Conventions (0-based everywhere; the paper's positions are 1-based):
+ *   logical page b of request r holds tokens [b*p, min(len_r, (b+1)*p)); its physical
+ *   page is page_table[r][b]; an entry of -1 means the page has no physical KV and is
+ *   never summarised, scored, selected or attended.  Query head a reads kv-head
+ *   g(a) = a / G with G = H_q / H_kv.
+ *
+ * Parity pins (tests, CPU only): brute-force min/max, the bound property of the page
+ * score, equality with a token logit on single-token pages, unit-vector closed forms,
+ * argsort brute force for top-k, equality with dense attention when every page is
+ * selected, log-sum-exp against a library routine, the unit sum of attention mass.
+ * Parity with the authors' own code is unpinned: the paper prints no numbers for
+ * this path, and the reduction of a GQA group to one per-kv-head score (max) is a
+ * convention of this build.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double bf16_to_f64(uint16_t bits) {
+    uint32_t w = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+static int tokens_in_page(int len, int b, int p) {
+    int nv = len - b * p;
+    if (nv > p) nv = p;
+    return nv < 0 ? 0 : nv;
+}
+
+/* strictly "x sorts below y" with -0 below +0, so that ties between the two zeros are
+ * resolved the same way on every platform (min keeps -0, max keeps +0). */
+static int lt_signed_zero(uint16_t xb, uint16_t yb) {
+    double x = bf16_to_f64(xb), y = bf16_to_f64(yb);
+    if (x < y) return 1;
+    if (x > y) return 0;
+    return (xb >> 15) > (yb >> 15);
+}
+
+/*
+ * Quest page summaries: for every request r, every logical page b >= first_tok[r]/p that
+ * has a physical page pid, every kv-head h and channel c,
+ *     m[pid,h,c] = min_t K[pid,h,t,c],  M[pid,h,c] = max_t K[pid,h,t,c]
+ * over the tokens t of the page that lie below len_r.  first_tok == NULL recomputes only
+ * the page that holds each request's newest token.  A min or max of bf16 values is one
+ * of them, so the summary is stored as bf16 bits and is exact.
+ *   k_cache [P, H_kv, p, D] bf16 bits      meta [P, H_kv, 2, D] bf16 bits (row 0 min, row 1 max)
+ */
+void se_oracle_meta(int B, int H_kv, int D, int p, int max_pages,
+                    const uint16_t *k_cache, const int32_t *page_table,
+                    const int32_t *seq_lens, const int32_t *first_tok,
+                    uint16_t *meta) {
+    for (int r = 0; r < B; ++r) {
+        int len = seq_lens[r];
+        if (len <= 0) continue;
+        int n_r = (len + p - 1) / p;
+        int b0 = first_tok ? first_tok[r] / p : n_r - 1;
+        if (b0 < 0) b0 = 0;
+        for (int b = b0; b < n_r; ++b) {
+            int pid = page_table[(size_t)r * max_pages + b];
+            if (pid < 0) continue;
+            int nv = tokens_in_page(len, b, p);
+            for (int h = 0; h < H_kv; ++h) {
+                const uint16_t *kp = k_cache + (((size_t)pid * H_kv + h) * p) * D;
+                uint16_t *mn = meta + (((size_t)pid * H_kv + h) * 2 + 0) * D;
+                uint16_t *mx = meta + (((size_t)pid * H_kv + h) * 2 + 1) * D;
+                for (int c = 0; c < D; ++c) {
+                    uint16_t lo = kp[c], hi = kp[c];
+                    for (int t = 1; t < nv; ++t) {
+                        uint16_t v = kp[(size_t)t * D + c];
+                        if (lt_signed_zero(v, lo)) lo = v;
+                        if (lt_signed_zero(hi, v)) hi = v;
+                    }
+                    mn[c] = lo;
+                    mx[c] = hi;
+                }
+            }
+        }
+    }
+}
+
+/*
+ * Quest page score.  For query head a of request r and logical page b with physical page
+ * pid >= 0:
+ *     S[r,a,b] = sm_scale * sum_c max( q[r,a,c]*m[pid,g(a),c], q[r,a,c]*M[pid,g(a),c] )
+ * (channels summed left to right), and the per-kv-head score that is ranked
+ *     P[r,h,b] = max over the query heads a of group h of S[r,a,b]
+ * (group_sum != 0 replaces that max by a sum; the CUDA path implements the max only).
+ * Pages that are absent or lie past the request's length get present = 0 and score 0.
+ *   q [B,H_q,D] bf16 bits   S [B,H_q,max_pages]   P [B,H_kv,max_pages]   present [B,max_pages]
+ */
+void se_oracle_scores(int B, int H_q, int H_kv, int D, int p, int max_pages,
+                      double sm_scale, int group_sum,
+                      const uint16_t *q, const uint16_t *meta,
+                      const int32_t *page_table, const int32_t *seq_lens,
+                      double *S, double *P, uint8_t *present) {
+    int G = H_q / H_kv;
+#pragma omp parallel for schedule(dynamic)
+    for (int rh = 0; rh < B * H_kv; ++rh) {
+        int r = rh / H_kv, h = rh % H_kv;
+        int len = seq_lens[r];
+        int n_r = len > 0 ? (len + p - 1) / p : 0;
+        for (int b = 0; b < max_pages; ++b) {
+            int pid = b < n_r ? page_table[(size_t)r * max_pages + b] : -1;
+            if (h == 0) present[(size_t)r * max_pages + b] = (uint8_t)(pid >= 0);
+            double best = 0.0, total = 0.0;
+            for (int g = 0; g < G; ++g) {
+                int a = h * G + g;
+                double s = 0.0;
+                if (pid >= 0) {
+                    const uint16_t *mn = meta + (((size_t)pid * H_kv + h) * 2 + 0) * D;
+                    const uint16_t *mx = meta + (((size_t)pid * H_kv + h) * 2 + 1) * D;
+                    const uint16_t *qa = q + ((size_t)r * H_q + a) * D;
+                    for (int c = 0; c < D; ++c) {
+                        double qc = bf16_to_f64(qa[c]);
+                        double lo = qc * bf16_to_f64(mn[c]);
+                        double hi = qc * bf16_to_f64(mx[c]);
+                        s += lo > hi ? lo : hi;
+                    }
+                    s *= sm_scale;
+                }
+                S[((size_t)r * H_q + a) * max_pages + b] = s;
+                if (g == 0 || s > best) best = s;
+                total += s;
+            }
+            P[((size_t)r * H_kv + h) * max_pages + b] = group_sum ? total : best;
+        }
+    }
+}
+
+typedef struct { double s; int b; } cand_t;
+
+static int cand_cmp(const void *x, const void *y) {
+    const cand_t *a = (const cand_t *)x, *c = (const cand_t *)y;
+    if (a->s > c->s) return -1;
+    if (a->s < c->s) return 1;
+    return a->b - c->b;                       /* equal scores: lower page first */
+}
+
+static int int_cmp(const void *x, const void *y) {
+    return *(const int *)x - *(const int *)y;
+}
+
+/*
+ * TopK: among the present pages of request r, the k_eff = min(floor(budget/p), #present)
+ * pages with the largest P[r,h,.]; equal scores are ordered by lower logical page.  The
+ * chosen logical page numbers are written in ascending order, the rest of the row is -1.
+ * theta[r,h,0] is the k_eff-th largest score, theta[r,h,1] the (k_eff+1)-th (NaN if none):
+ * the caller uses them to see how close a decision was.
+ *   sel_idx [B,H_kv,k_max]   sel_cnt [B,H_kv]   theta [B,H_kv,2]
+ */
+void se_oracle_topk(int B, int H_kv, int p, int max_pages, int k_max, int budget,
+                    const double *P, const uint8_t *present,
+                    int32_t *sel_idx, int32_t *sel_cnt, double *theta) {
+    int k = budget / p;
+#pragma omp parallel for schedule(dynamic)
+    for (int rh = 0; rh < B * H_kv; ++rh) {
+        int r = rh / H_kv;
+        cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(max_pages > 0 ? max_pages : 1));
+        int n = 0;
+        for (int b = 0; b < max_pages; ++b)
+            if (present[(size_t)r * max_pages + b]) {
+                cand[n].s = P[(size_t)rh * max_pages + b];
+                cand[n].b = b;
+                ++n;
+            }
+        qsort(cand, (size_t)n, sizeof(cand_t), cand_cmp);
+        int k_eff = k < n ? k : n;
+        if (k_eff > k_max) k_eff = k_max;
+        int *chosen = (int *)malloc(sizeof(int) * (size_t)(k_eff > 0 ? k_eff : 1));
+        for (int i = 0; i < k_eff; ++i) chosen[i] = cand[i].b;
+        qsort(chosen, (size_t)k_eff, sizeof(int), int_cmp);
+        for (int i = 0; i < k_max; ++i)
+            sel_idx[(size_t)rh * k_max + i] = i < k_eff ? chosen[i] : -1;
+        sel_cnt[rh] = k_eff;
+        theta[(size_t)rh * 2 + 0] = k_eff > 0 ? cand[k_eff - 1].s : NAN;
+        theta[(size_t)rh * 2 + 1] = k_eff < n ? cand[k_eff].s : NAN;
+        free(chosen);
+        free(cand);
+    }
+}
+
+/*
+ * Attention over the tokens of the selected pages.  For query head a of request r the
+ * attended set T holds every token (b,t) with b in sel_idx[r,g(a),0..sel_cnt) and
+ * t below the number of valid tokens of page b.  Then
+ *     z_j = sm_scale * sum_c q_c k_{j,c},   alpha_j = exp(z_j) / sum_{u in T} exp(z_u),
+ *     out_c = sum_j alpha_j v_{j,c},        lse = ln sum_{u in T} exp(z_u)
+ * (evaluated with the maximum logit subtracted).  An empty T gives out = 0, lse = -inf.
+ * If u_accum is not NULL, the H2O statistic of every attended token slot grows by the
+ * attention mass it received, summed over the query heads of its kv-head:
+ *     u[pid,h,t] += sum_{a in group h} alpha_{a,(b,t)} .
+ *   out [B,H_q,D]   lse [B,H_q]   u_accum [P,H_kv,p] (in/out)
+ */
+void se_oracle_attend(int B, int H_q, int H_kv, int D, int p, int max_pages, int k_max,
+                      double sm_scale,
+                      const uint16_t *q, const uint16_t *k_cache, const uint16_t *v_cache,
+                      const int32_t *page_table, const int32_t *seq_lens,
+                      const int32_t *sel_idx, const int32_t *sel_cnt,
+                      double *out, double *lse, double *u_accum) {
+    int G = H_q / H_kv;
+#pragma omp parallel for schedule(dynamic)
+    for (int rh = 0; rh < B * H_kv; ++rh) {
+        int r = rh / H_kv, h = rh % H_kv;
+        int len = seq_lens[r];
+        int cnt = sel_cnt[rh];
+        double *z = (double *)malloc(sizeof(double) * (size_t)(cnt > 0 ? cnt : 1) * p);
+        for (int g = 0; g < G; ++g) {
+            int a = h * G + g;
+            const uint16_t *qa = q + ((size_t)r * H_q + a) * D;
+            double *o = out + ((size_t)r * H_q + a) * D;
+            for (int c = 0; c < D; ++c) o[c] = 0.0;
+            /* logits */
+            double zmax = -INFINITY;
+            int any = 0;
+            for (int i = 0; i < cnt; ++i) {
+                int b = sel_idx[(size_t)rh * k_max + i];
+                int pid = b >= 0 ? page_table[(size_t)r * max_pages + b] : -1;
+                int nv = (b >= 0 && pid >= 0) ? tokens_in_page(len, b, p) : 0;
+                for (int t = 0; t < p; ++t) {
+                    double zz = -INFINITY;
+                    if (t < nv) {
+                        const uint16_t *kt = k_cache + ((((size_t)pid * H_kv + h) * p) + t) * D;
+                        double s = 0.0;
+                        for (int c = 0; c < D; ++c) s += bf16_to_f64(qa[c]) * bf16_to_f64(kt[c]);
+                        zz = s * sm_scale;
+                        any = 1;
+                        if (zz > zmax) zmax = zz;
+                    }
+                    z[(size_t)i * p + t] = zz;
+                }
+            }
+            if (!any) {
+                lse[(size_t)r * H_q + a] = -INFINITY;
+                continue;
+            }
+            /* normaliser */
+            double denom = 0.0;
+            for (int i = 0; i < cnt * p; ++i)
+                if (z[i] > -INFINITY) denom += exp(z[i] - zmax);
+            lse[(size_t)r * H_q + a] = zmax + log(denom);
+            /* weighted values and the H2O statistic */
+            for (int i = 0; i < cnt; ++i) {
+                int b = sel_idx[(size_t)rh * k_max + i];
+                int pid = b >= 0 ? page_table[(size_t)r * max_pages + b] : -1;
+                for (int t = 0; t < p; ++t) {
+                    double zz = z[(size_t)i * p + t];
+                    if (!(zz > -INFINITY)) continue;
+                    double alpha = exp(zz - zmax) / denom;
+                    const uint16_t *vt = v_cache + ((((size_t)pid * H_kv + h) * p) + t) * D;
+                    for (int c = 0; c < D; ++c) o[c] += alpha * bf16_to_f64(vt[c]);
+                    if (u_accum) u_accum[((size_t)pid * H_kv + h) * p + t] += alpha;
+                }
+            }
+        }
+        free(z);
+    }
+}
