@@ -1,0 +1,172 @@
+/*
+ * sparse_engine.h — C ABI of the B200 (sm_100a) sparse decode-attention library.
+ *
+ * The library implements the data-parallel hot path of one decode step of a sparse-first
+ * inference engine: Quest-style page summaries, query-dependent page scoring, per
+ * (request, kv-head) top-k page selection under a token budget, and split-K paged
+ * attention over the selected pages with a log-sum-exp merge and an optional H2O
+ * accumulated-attention epilogue.  (Paper: Appendix A "Detailed Background and
+ * Notations"; Appendix B "Lifecycle Implementation Details" for the attention-view
+ * payload and the CUDA-graph buffer rules the interface follows.)
+ *
+ * General rules, valid for every entry point
+ * ------------------------------------------
+ *  - All data pointers are DEVICE pointers to contiguous buffers owned by the caller;
+ *    `const se_params*` and `int32_t* host_out` are HOST pointers.  The library never
+ *    allocates, frees or keeps a pointer after the call returns.
+ *  - `stream` is a `cudaStream_t` passed as `void*` (NULL = the default stream).  Calls
+ *    enqueue work on it and return; only `se_last_device_status` synchronises.
+ *  - Return value: SE_OK (0) or a negative SE_ERR_* code.  Arguments are validated on
+ *    the host before anything is launched; on error nothing has been enqueued.
+ *  - Shapes: B requests, H_q query heads, H_kv kv-heads, G = H_q / H_kv in 1..8,
+ *    D in {64, 128}, page size 16 tokens.  Query head a reads kv-head a / G
+ *    (Appendix A, "MHA, MQA, and GQA").
+ *  - Layouts (row-major, innermost last):
+ *      q           [B, H_q, D]               bf16
+ *      k_cache     [P_phys, H_kv, 16, D]     bf16   (one page of one kv-head is contiguous)
+ *      v_cache     [P_phys, H_kv, 16, D]     bf16
+ *      meta        [P_phys, H_kv, 2, D]      bf16   row 0 = channel-wise min, row 1 = max;
+ *                                                   indexed by PHYSICAL page, so aliased
+ *                                                   prefix pages share their summaries
+ *      page_table  [B, max_pages]            int32  physical page of logical page b, or -1
+ *                                                   if that page has no physical KV
+ *                                                   (Appendix A, "Logical Positions and
+ *                                                   Physical Blocks"; 0-based here)
+ *      seq_lens    [B]                       int32  logical tokens of the request, the
+ *                                                   current one included; 0 = padding slot
+ *      sel_idx     [B, H_kv, k_max]          int32  selected LOGICAL pages, ascending,
+ *                                                   padded with -1
+ *      sel_cnt     [B, H_kv]                 int32  number of valid entries per row
+ *      out         [B, H_q, D]               fp32
+ *      lse         [B, H_q]                  fp32   natural-log log-sum-exp of the logits
+ *      score_accum [P_phys, H_kv, 16]        fp32   H2O statistic per token slot
+ *  - All pointers must be 16-byte aligned.
+ *  - Inputs must be finite; behaviour with NaN/Inf in q, K, V is unspecified.
+ *  - Physical page ids outside [0, num_phys_pages) and selected pages outside the
+ *    request are never dereferenced: the access is skipped and a bit is set in the
+ *    device status word (see se_last_device_status).
+ */
+#ifndef SPARSE_ENGINE_H_
+#define SPARSE_ENGINE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SE_OK                       0
+#define SE_ERR_INVALID_ARG         -1   /* a size or value is out of range                 */
+#define SE_ERR_UNSUPPORTED_SHAPE   -2   /* D, G or page_size not supported                 */
+#define SE_ERR_NULL_POINTER        -3   /* a required pointer is NULL                      */
+#define SE_ERR_MISALIGNED          -4   /* a pointer is not 16-byte aligned                */
+#define SE_ERR_CUDA                -5   /* a CUDA runtime call failed (launch, attribute)  */
+
+/* bits of the device status word */
+#define SE_DEV_BAD_PAGE_ID          1u  /* page_table entry >= num_phys_pages              */
+#define SE_DEV_BAD_SELECTION        2u  /* sel_idx entry outside the request / sel_cnt > k_max */
+#define SE_DEV_WAIT_TIMEOUT         4u  /* a bounded wait on an asynchronous copy gave up   */
+
+typedef struct se_params {
+    int32_t B;               /* requests in the batch (>= 1)                                */
+    int32_t H_q;             /* query heads                                                 */
+    int32_t H_kv;            /* kv heads; H_q % H_kv == 0, H_q / H_kv in 1..8               */
+    int32_t D;               /* head dimension, 64 or 128                                   */
+    int32_t page_size;       /* must be 16                                                  */
+    int32_t max_pages;       /* row stride of page_table, >= ceil(max seq_len / 16)         */
+    int32_t num_phys_pages;  /* P_phys, pages in k_cache / v_cache / meta / score_accum     */
+    int32_t k_max;           /* row stride of sel_idx, >= floor(budget / 16), 1..4096       */
+    float   sm_scale;        /* logit scale; 0 selects 1/sqrt(D)                            */
+    uint32_t flags;          /* reserved, must be 0                                         */
+} se_params;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int se_version(void);
+
+/* Text for an SE_ERR_* code (static storage, never NULL). */
+const char *se_strerror(int code);
+
+/*
+ * Bytes of device scratch the calls below need for `p` (host, pure; 0 if `p` is invalid).
+ * The caller allocates that many bytes (256-byte aligned), runs se_workspace_init once,
+ * and may then reuse the buffer for any number of calls with the same `p`.  Calls that
+ * share a workspace must be ordered on the device (same stream or explicit dependencies).
+ */
+size_t se_workspace_bytes(const se_params *p);
+
+/*
+ * Zeroes the control block (completion counters, status word) at the head of the
+ * workspace.  Required once after allocation; the kernels leave the counters at zero
+ * when they finish, so it need not be repeated.
+ */
+int se_workspace_init(const se_params *p, void *workspace, void *stream);
+
+/*
+ * Quest page summaries (Appendix A, "Quest: Query-Dependent Page Selection", summary
+ * equation): for every kv-head h and channel c of a page,
+ *     meta[pid,h,0,c] = min_t K[pid,h,t,c],   meta[pid,h,1,c] = max_t K[pid,h,t,c]
+ * over the tokens t of the page that lie below the request's length.
+ *   first_tok == NULL : recompute only the page holding each request's newest token
+ *                       ("new keys update the extrema of their pages"); run after the
+ *                       token's K has been written to k_cache.
+ *   first_tok != NULL : [B] int32; recompute every page of request r from the page
+ *                       holding token first_tok[r] on (0 = rebuild all, e.g. after prefill).
+ * Pages with page_table == -1 and pages no request refers to are left untouched.  The
+ * result is exact (a min/max of bf16 values); -0 orders below +0.  Requests that alias
+ * the same physical page write identical values.  A request's partially filled last
+ * page must not be aliased by another request of a different length.
+ */
+int se_meta_update(const se_params *p, const void *k_cache, const int32_t *page_table,
+                   const int32_t *seq_lens, const int32_t *first_tok, void *meta,
+                   void *stream);
+
+/*
+ * Page scoring and top-k selection (Appendix A, Quest score equation and the TopK entry
+ * of the notation table).  For request r, kv-head h and every logical page b < ceil(len_r/16)
+ * that has a physical page:
+ *     S[a,b] = sm_scale * sum_c max(q[r,a,c]*min[b,c], q[r,a,c]*max[b,c])   (fp32)
+ *     P[h,b] = max over the query heads a of group h of S[a,b]
+ * and sel_idx[r,h,:] receives the k_eff = min(floor(budget_tokens/16), #present pages)
+ * pages with the largest P (equal scores: lower page first), in ascending page order,
+ * padded with -1; sel_cnt[r,h] = k_eff.  A request with seq_len 0 or no present page
+ * gets sel_cnt 0.  Requires 16 <= budget_tokens <= 16*k_max.  Never writes q, meta or
+ * the page table.  Uses the workspace for the fp32 scores.
+ */
+int se_page_select(const se_params *p, const void *q, const void *meta,
+                   const int32_t *page_table, const int32_t *seq_lens,
+                   int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
+                   void *workspace, void *stream);
+
+/*
+ * Attention over the tokens of the selected pages (Appendix A, "Attention over Selected
+ * Positions"): for every query head a of request r, with T the tokens (below len_r) of
+ * the pages sel_idx[r, a/G, 0..sel_cnt),
+ *     z_j = sm_scale * q.k_j,  alpha_j = exp(z_j)/sum_{u in T} exp(z_u),
+ *     out = sum_j alpha_j v_j,  lse = ln sum_{u in T} exp(z_u).
+ * The selected pages are split over several workers (split-K) whose partial results are
+ * merged through their running maxima; out/lse do not depend on the split beyond fp32
+ * rounding.  An empty T gives out = 0 and lse = -inf.
+ * score_accum != NULL additionally applies the H2O update (Appendix A, H2O accumulated
+ * score equation) to every attended token slot:
+ *     score_accum[pid,h,t] += sum over the query heads a of group h of alpha_{a,(pid,t)} .
+ * With score_accum the physical pages selected by different requests must be distinct
+ * (no aliased prefix), otherwise the read-modify-write races.  Never writes q, K, V,
+ * the page table or the selection.
+ */
+int se_sparse_decode(const se_params *p, const void *q, const void *k_cache,
+                     const void *v_cache, const int32_t *page_table,
+                     const int32_t *seq_lens, const int32_t *sel_idx,
+                     const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                     void *workspace, void *stream);
+
+/*
+ * Copies the device status word (an OR of SE_DEV_* bits, 0 = clean) to *host_out and
+ * clears it.  Synchronises `stream`; the only entry point that does.
+ */
+int se_last_device_status(void *workspace, void *stream, int32_t *host_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSE_ENGINE_H_ */

@@ -1,0 +1,202 @@
+"""Thin ctypes binding of ``libsparse_engine.so`` (see ``include/sparse_engine.h``).
+
+Argument marshalling only: every function takes torch CUDA tensors, checks dtype,
+contiguity and shape, and passes raw device pointers plus the current CUDA stream to
+the C entry point of the same name.  There is no CPU or PyTorch fallback: if the shared
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import _build
+
+SE_OK = 0
+SE_DEV_BAD_PAGE_ID = 1
+SE_DEV_BAD_SELECTION = 2
+SE_DEV_WAIT_TIMEOUT = 4
+
+EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_workspace_init", "se_meta_update",
+           "se_page_select", "se_sparse_decode", "se_last_device_status")
+
+
+class SeParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H_q", ctypes.c_int32), ("H_kv", ctypes.c_int32),
+                ("D", ctypes.c_int32), ("page_size", ctypes.c_int32), ("max_pages", ctypes.c_int32),
+                ("num_phys_pages", ctypes.c_int32), ("k_max", ctypes.c_int32),
+                ("sm_scale", ctypes.c_float), ("flags", ctypes.c_uint32)]
+
+
+class SparseEngineError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True):
+    """Loads the shared library (building it with nvcc first if it is absent or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing and _build.needs_build():
+        _build.build()
+    if not os.path.exists(_build.LIB):
+        raise SparseEngineError("libsparse_engine.so is missing; run `python -m paper_2609_39068_b200._build`")
+    lib = ctypes.CDLL(_build.LIB)
+    vp, i32p, fp = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+    pp = ctypes.POINTER(SeParams)
+    lib.se_version.restype = ctypes.c_int
+    lib.se_strerror.restype = ctypes.c_char_p
+    lib.se_strerror.argtypes = [ctypes.c_int]
+    lib.se_workspace_bytes.restype = ctypes.c_size_t
+    lib.se_workspace_bytes.argtypes = [pp]
+    lib.se_workspace_init.argtypes = [pp, vp, vp]
+    lib.se_meta_update.argtypes = [pp, vp, i32p, i32p, i32p, vp, vp]
+    lib.se_page_select.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
+    lib.se_sparse_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, fp, fp, fp, vp, vp]
+    lib.se_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+    for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_sparse_decode",
+                 "se_last_device_status"):
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(rc: int, what: str):
+    if rc != SE_OK:
+        raise SparseEngineError("%s failed: %s (%d)" % (what, load().se_strerror(rc).decode(), rc))
+
+
+def _ptr(t: Optional[torch.Tensor], dtype, name: str):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise SparseEngineError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype:
+        raise SparseEngineError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise SparseEngineError("%s must be contiguous" % name)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_params(B, H_q, H_kv, D, max_pages, num_phys_pages, k_max, sm_scale=0.0, page_size=16) -> SeParams:
+    return SeParams(B, H_q, H_kv, D, page_size, max_pages, num_phys_pages, k_max, float(sm_scale), 0)
+
+
+def se_version() -> int:
+    return load().se_version()
+
+
+def se_strerror(code: int) -> str:
+    return load().se_strerror(code).decode()
+
+
+def se_workspace_bytes(p: SeParams) -> int:
+    return int(load().se_workspace_bytes(ctypes.byref(p)))
+
+
+def se_workspace_init(p: SeParams, workspace: torch.Tensor) -> None:
+    _check(load().se_workspace_init(ctypes.byref(p), _ptr(workspace, torch.uint8, "workspace"), _stream()),
+           "se_workspace_init")
+
+
+def alloc_workspace(p: SeParams, device="cuda") -> torch.Tensor:
+    """Allocates (through torch) and initialises a workspace for ``p``."""
+    n = se_workspace_bytes(p)
+    if n == 0:
+        raise SparseEngineError("invalid se_params")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    se_workspace_init(p, ws)
+    return ws
+
+
+def se_meta_update(p, k_cache, page_table, seq_lens, meta, first_tok=None) -> None:
+    _check(load().se_meta_update(ctypes.byref(p), _ptr(k_cache, torch.bfloat16, "k_cache"),
+                                 _ptr(page_table, torch.int32, "page_table"),
+                                 _ptr(seq_lens, torch.int32, "seq_lens"),
+                                 _ptr(first_tok, torch.int32, "first_tok"),
+                                 _ptr(meta, torch.bfloat16, "meta"), _stream()), "se_meta_update")
+
+
+def se_page_select(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, workspace) -> None:
+    _check(load().se_page_select(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                 _ptr(meta, torch.bfloat16, "meta"),
+                                 _ptr(page_table, torch.int32, "page_table"),
+                                 _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens),
+                                 _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                 _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_page_select")
+
+
+def se_sparse_decode(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
+                     workspace, score_accum=None) -> None:
+    _check(load().se_sparse_decode(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                   _ptr(k_cache, torch.bfloat16, "k_cache"),
+                                   _ptr(v_cache, torch.bfloat16, "v_cache"),
+                                   _ptr(page_table, torch.int32, "page_table"),
+                                   _ptr(seq_lens, torch.int32, "seq_lens"),
+                                   _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                   _ptr(out, torch.float32, "out"), _ptr(lse, torch.float32, "lse"),
+                                   _ptr(score_accum, torch.float32, "score_accum"),
+                                   _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_sparse_decode")
+
+
+def se_last_device_status(workspace) -> int:
+    word = ctypes.c_int32(0)
+    _check(load().se_last_device_status(_ptr(workspace, torch.uint8, "workspace"), _stream(),
+                                        ctypes.byref(word)), "se_last_device_status")
+    return int(word.value)
+
+
+class DecodeState:
+    """Buffers of one layer's decode step for a fixed shape: params, workspace, summaries,
+    selection and outputs.  Convenience for tests, the smoke check and the benchmark."""
+
+    def __init__(self, w, k_max: Optional[int] = None, sm_scale: float = 0.0):
+        dev = w.q.device
+        self.w = w
+        self.k_max = int(k_max if k_max is not None else max(w.budget // 16, 1))
+        self.p = make_params(w.B, w.H_q, w.H_kv, w.D, w.max_pages, w.num_phys_pages, self.k_max, sm_scale)
+        self.workspace = alloc_workspace(self.p, dev)
+        self.meta = torch.zeros((w.num_phys_pages, w.H_kv, 2, w.D), dtype=torch.bfloat16, device=dev)
+        self.sel_idx = torch.full((w.B, w.H_kv, self.k_max), -7, dtype=torch.int32, device=dev)
+        self.sel_cnt = torch.full((w.B, w.H_kv), -7, dtype=torch.int32, device=dev)
+        self.out = torch.full((w.B, w.H_q, w.D), float("nan"), dtype=torch.float32, device=dev)
+        self.lse = torch.full((w.B, w.H_q), float("nan"), dtype=torch.float32, device=dev)
+
+    def rebuild_meta(self):
+        ft = torch.zeros(self.w.B, dtype=torch.int32, device=self.w.q.device)
+        se_meta_update(self.p, self.w.k_cache, self.w.page_table, self.w.seq_lens, self.meta, first_tok=ft)
+
+    def update_meta(self):
+        se_meta_update(self.p, self.w.k_cache, self.w.page_table, self.w.seq_lens, self.meta)
+
+    def select(self, budget: Optional[int] = None):
+        se_page_select(self.p, self.w.q, self.meta, self.w.page_table, self.w.seq_lens,
+                       self.w.budget if budget is None else budget, self.sel_idx, self.sel_cnt, self.workspace)
+
+    def decode(self, score_accum=None):
+        se_sparse_decode(self.p, self.w.q, self.w.k_cache, self.w.v_cache, self.w.page_table,
+                         self.w.seq_lens, self.sel_idx, self.sel_cnt, self.out, self.lse,
+                         self.workspace, score_accum=score_accum)
+
+    def step(self, score_accum=None):
+        """One decode step of the layer: newest-page summary, selection, attention."""
+        self.update_meta()
+        self.select()
+        self.decode(score_accum)
+
+    def status(self) -> int:
+        return se_last_device_status(self.workspace)

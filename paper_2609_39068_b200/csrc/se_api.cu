@@ -1,0 +1,179 @@
+// C ABI entry points: argument validation, workspace layout, launch geometry.
+#include <math.h>
+
+#include "se_internal.h"
+
+namespace se {
+
+namespace {
+
+constexpr int kAssumedSMs = 148;      // B200; launch geometry and workspace size are derived from
+                                      // this constant so that se_workspace_bytes is a pure function
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+int validate(const se_params *p) {
+    if (!p) return SE_ERR_NULL_POINTER;
+    if (p->page_size != kPage) return SE_ERR_UNSUPPORTED_SHAPE;
+    if (p->D != 64 && p->D != 128) return SE_ERR_UNSUPPORTED_SHAPE;
+    if (p->B < 1 || p->H_q < 1 || p->H_kv < 1) return SE_ERR_INVALID_ARG;
+    if (p->H_q % p->H_kv != 0) return SE_ERR_INVALID_ARG;
+    const int G = p->H_q / p->H_kv;
+    if (G < 1 || G > 8) return SE_ERR_UNSUPPORTED_SHAPE;
+    if (p->max_pages < 1 || p->num_phys_pages < 1) return SE_ERR_INVALID_ARG;
+    if (p->k_max < 1 || p->k_max > 4096) return SE_ERR_INVALID_ARG;
+    if (p->flags != 0) return SE_ERR_INVALID_ARG;
+    if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return SE_ERR_INVALID_ARG;
+    // index arithmetic inside the kernels uses 32-bit page counts and 64-bit byte offsets
+    if ((long long)p->B * p->H_kv > (1ll << 24)) return SE_ERR_INVALID_ARG;
+    if ((long long)p->B * p->max_pages > (1ll << 31) - 1) return SE_ERR_INVALID_ARG;
+    return SE_OK;
+}
+
+bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+}  // namespace
+
+int device_sm_count() { return kAssumedSMs; }
+
+float effective_scale(const se_params &p) {
+    return p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.D);
+}
+
+int decode_warps_per_cta();
+
+DecodePlan make_decode_plan(const se_params &p) {
+    DecodePlan plan;
+    const int warps_per_cta = decode_warps_per_cta();
+    const long long X = (long long)p.B * p.H_kv * p.k_max;
+    const int ctas_per_sm = (p.D == 128) ? 1 : 1;
+    long long warps = (long long)kAssumedSMs * ctas_per_sm * warps_per_cta;
+    long long ppw = (X + warps - 1) / warps;
+    if (ppw < 1) ppw = 1;
+    long long used_warps = (X + ppw - 1) / ppw;
+    long long grid = (used_warps + warps_per_cta - 1) / warps_per_cta;
+    plan.grid = (int)grid;
+    plan.warps_total = (int)(grid * warps_per_cta);
+    plan.pages_per_warp = (int)ppw;
+    plan.max_splits = (int)((p.k_max + ppw - 1) / ppw) + 1;
+    return plan;
+}
+
+WorkspaceLayout make_layout(const se_params &p) {
+    WorkspaceLayout L;
+    const DecodePlan plan = make_decode_plan(p);
+    const size_t pairs = (size_t)p.B * p.H_kv;
+    const int G = p.H_q / p.H_kv;
+    const int GP = next_pow2(G);
+    size_t off = 0;
+    L.status = off;      off += 256;
+    L.sel_tickets = off; off += align256(pairs * 4);
+    L.dec_tickets = off; off += align256(pairs * 4);
+    L.scores = off;      off += align256(pairs * (size_t)p.max_pages * 4);
+    L.partials = off;    off += align256((size_t)p.B * p.H_q * plan.max_splits * (p.D + 4) * 4);
+    L.zbuf = off;        off += align256(pairs * (size_t)p.k_max * kPage * GP * 4);
+    L.total = off;
+    L.max_splits = plan.max_splits;
+    return L;
+}
+
+}  // namespace se
+
+using namespace se;
+
+extern "C" {
+
+int se_version(void) { return 100; }
+
+const char *se_strerror(int code) {
+    switch (code) {
+        case SE_OK: return "ok";
+        case SE_ERR_INVALID_ARG: return "invalid argument";
+        case SE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need page_size 16, D in {64,128}, 1 <= H_q/H_kv <= 8)";
+        case SE_ERR_NULL_POINTER: return "required pointer is NULL";
+        case SE_ERR_MISALIGNED: return "pointer is not 16-byte aligned";
+        case SE_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown error code";
+}
+
+size_t se_workspace_bytes(const se_params *p) {
+    if (validate(p) != SE_OK) return 0;
+    return make_layout(*p).total;
+}
+
+int se_workspace_init(const se_params *p, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!workspace) return SE_ERR_NULL_POINTER;
+    if (!aligned16(workspace)) return SE_ERR_MISALIGNED;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, L.scores, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_meta_update(const se_params *p, const void *k_cache, const int32_t *page_table,
+                   const int32_t *seq_lens, const int32_t *first_tok, void *meta, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!k_cache || !page_table || !seq_lens || !meta) return SE_ERR_NULL_POINTER;
+    if (!aligned16(k_cache) || !aligned16(meta) || !aligned16(page_table) || !aligned16(seq_lens) ||
+        !aligned16(first_tok))
+        return SE_ERR_MISALIGNED;
+    cudaError_t e = launch_meta_update(*p, k_cache, page_table, seq_lens, first_tok, meta,
+                                       static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_page_select(const se_params *p, const void *q, const void *meta, const int32_t *page_table,
+                   const int32_t *seq_lens, int32_t budget_tokens, int32_t *sel_idx,
+                   int32_t *sel_cnt, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!q || !meta || !page_table || !seq_lens || !sel_idx || !sel_cnt || !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(meta) || !aligned16(page_table) || !aligned16(seq_lens) ||
+        !aligned16(sel_idx) || !aligned16(sel_cnt) || !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    if (budget_tokens < kPage) return SE_ERR_INVALID_ARG;
+    const int k_pages = budget_tokens / kPage;
+    if (k_pages > p->k_max) return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_page_select(*p, q, meta, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
+                                       workspace, L, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                     const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+                     const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                     void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!q || !k_cache || !v_cache || !page_table || !seq_lens || !sel_idx || !sel_cnt || !out ||
+        !lse || !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(page_table) ||
+        !aligned16(seq_lens) || !aligned16(sel_idx) || !aligned16(sel_cnt) || !aligned16(out) ||
+        !aligned16(lse) || !aligned16(score_accum) || !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens, sel_idx,
+                                         sel_cnt, out, lse, score_accum, workspace, L,
+                                         static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_last_device_status(void *workspace, void *stream, int32_t *host_out) {
+    if (!workspace || !host_out) return SE_ERR_NULL_POINTER;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(workspace, 0, sizeof word, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return SE_ERR_CUDA;
+    *host_out = (int32_t)word;
+    return SE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,42 @@
+// Host-side declarations shared by the translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "se_device.cuh"
+
+namespace se {
+
+// Decode-kernel geometry that both the workspace sizing and the launcher derive from
+// the problem shape alone (never from device data).
+struct DecodePlan {
+    int warps_total;        // persistent warps over the whole grid
+    int grid;               // CTAs
+    int pages_per_warp;     // contiguous slice of the flattened (pair, selected page) space
+    int max_splits;         // most warps that can touch one (request, head) pair
+};
+
+int  device_sm_count();
+DecodePlan make_decode_plan(const se_params &p);
+WorkspaceLayout make_layout(const se_params &p);
+float effective_scale(const se_params &p);
+
+// kernels' launchers; each returns a cudaError_t from the launch
+cudaError_t launch_meta_update(const se_params &p, const void *k_cache, const int32_t *page_table,
+                               const int32_t *seq_lens, const int32_t *first_tok, void *meta,
+                               cudaStream_t stream);
+
+cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta,
+                               const int32_t *page_table, const int32_t *seq_lens, int k_pages,
+                               int32_t *sel_idx, int32_t *sel_cnt, void *workspace,
+                               const WorkspaceLayout &L, cudaStream_t stream);
+
+cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *k_cache,
+                                 const void *v_cache, const int32_t *page_table,
+                                 const int32_t *seq_lens, const int32_t *sel_idx,
+                                 const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                                 void *workspace, const WorkspaceLayout &L, cudaStream_t stream);
+
+}  // namespace se

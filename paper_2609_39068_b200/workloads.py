@@ -251,6 +251,27 @@ def config5(device="cpu", layer: int = 0, B: int = 128, lo: int = 8192, hi: int 
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
 
 
+def sub_workload(w: Workload, rows, device="cpu") -> Workload:
+    """The requests ``rows`` of ``w`` with their pages gathered into a compact pool of their
+    own (physical ids renumbered, aliasing preserved).  Pure data movement: it lets a few
+    requests of a multi-gigabyte workload be handed to the CPU without copying the pool."""
+    rows = [int(r) for r in rows]
+    pt = w.page_table[rows].cpu().to(torch.int64)
+    used = torch.unique(pt[pt >= 0])
+    remap = torch.full((w.num_phys_pages,), -1, dtype=torch.int64)
+    remap[used] = torch.arange(used.numel())
+    new_pt = torch.where(pt >= 0, remap[pt.clamp(min=0)], torch.full_like(pt, -1))
+    idx = used.to(w.k_cache.device)
+    accum = None if w.score_accum is None else w.score_accum[idx].to(device)
+    ridx = torch.tensor(rows, device=w.q.device)
+    return Workload(
+        name=w.name + "_sub%d" % len(rows), B=len(rows), H_q=w.H_q, H_kv=w.H_kv, D=w.D,
+        budget=w.budget, max_pages=w.max_pages, num_phys_pages=int(used.numel()),
+        q=w.q[ridx].to(device), k_cache=w.k_cache[idx].to(device), v_cache=w.v_cache[idx].to(device),
+        page_table=new_pt.to(torch.int32).to(device), seq_lens=w.seq_lens[ridx].to(device),
+        score_accum=accum)
+
+
 def bf16_bits(t: torch.Tensor):
     """The raw bf16 bit patterns of ``t`` as a numpy uint16 array on the host."""
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view("uint16")

@@ -1,0 +1,78 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+symbol the header declares, sizes its workspace, and rejects bad arguments before
+launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_39068_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        if fn.endswith(".h"):
+            src = open(os.path.join(inc, fn)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names |= set(re.findall(r"\b(se_[a-z_0-9]+)\s*\(", src))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    lib = binding.load()
+    names = declared_symbols()
+    assert {"se_meta_update", "se_page_select", "se_sparse_decode"} <= names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(binding.EXPORTS) <= names
+    assert lib.se_version() >= 100
+
+
+def test_strerror_texts():
+    assert binding.se_strerror(0) == "ok"
+    for code in (-1, -2, -3, -4, -5, -99):
+        assert binding.se_strerror(code)
+
+
+def test_workspace_bytes_is_pure_and_monotone():
+    p = binding.make_params(8, 32, 8, 128, 2048, 16384, 128)
+    n1 = binding.se_workspace_bytes(p)
+    assert n1 > 0 and n1 % 256 == 0 and n1 == binding.se_workspace_bytes(p)
+    p2 = binding.make_params(16, 32, 8, 128, 2048, 16384, 128)
+    assert binding.se_workspace_bytes(p2) > n1
+
+
+@pytest.mark.parametrize("kw", [
+    dict(D=96), dict(page_size=32), dict(H_q=36), dict(H_q=72), dict(B=0), dict(k_max=0),
+    dict(k_max=5000), dict(max_pages=0), dict(num_phys_pages=0), dict(sm_scale=-1.0),
+])
+def test_invalid_params_are_rejected(kw):
+    base = dict(B=2, H_q=32, H_kv=8, D=128, max_pages=64, num_phys_pages=128, k_max=16, sm_scale=0.0,
+                page_size=16)
+    base.update(kw)
+    p = binding.make_params(**base)
+    assert binding.se_workspace_bytes(p) == 0
+    lib = binding.load()
+    fake = ctypes.c_void_p(4096)
+    rc = lib.se_meta_update(ctypes.byref(p), fake, fake, fake, None, fake, None)
+    assert rc in (-1, -2)
+
+
+def test_null_and_misaligned_pointers_are_rejected_before_launch():
+    lib = binding.load()
+    p = binding.make_params(2, 32, 8, 128, 64, 128, 16)
+    ok = ctypes.c_void_p(4096)
+    odd = ctypes.c_void_p(4100)
+    assert lib.se_meta_update(ctypes.byref(p), None, ok, ok, None, ok, None) == -3
+    assert lib.se_meta_update(ctypes.byref(p), odd, ok, ok, None, ok, None) == -4
+    assert lib.se_page_select(ctypes.byref(p), ok, ok, ok, ok, 256, ok, ok, None, None) == -3
+    assert lib.se_page_select(ctypes.byref(p), ok, ok, ok, ok, 8, ok, ok, ok, None) == -1      # budget < one page
+    assert lib.se_page_select(ctypes.byref(p), ok, ok, ok, ok, 16 * 17, ok, ok, ok, None) == -1  # budget > k_max pages
+    assert lib.se_sparse_decode(ctypes.byref(p), ok, ok, ok, ok, ok, ok, ok, ok, None, None, ok, None) == -3
+    assert lib.se_sparse_decode(ctypes.byref(p), ok, ok, ok, ok, ok, ok, ok, ok, ok, odd, ok, None) == -4
+    assert lib.se_workspace_init(None, ok, None) == -3

@@ -1,0 +1,308 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the
+same seeded bf16 inputs.
+
+Bars: page summaries bit-exact; selected-page sets exact except inside the 1e-5 relative
+band around the oracle's k-th score; out within 1e-2 max-abs and 1e-3 mean-abs, lse within
+1e-3 (attention is compared on the GPU's own selection, so a legal swap inside the band
+cannot fail it); H2O increments within 1e-4 + 1e-3*value and summing to the group size.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39068_b200 import binding
+from paper_2609_39068_b200 import workloads as wl
+from helpers import check_selection, host_arrays
+
+pytestmark = pytest.mark.gpu
+
+OUT_MAX_ABS = 1e-2
+OUT_MEAN_ABS = 1e-3
+LSE_ABS = 1e-3
+
+
+def run_gpu(w_cpu, accum=False, incremental_after=None):
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    st.select()
+    u = w.score_accum.clone() if accum else None
+    st.decode(score_accum=u)
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    return w, st, u
+
+
+def compare(w_cpu, st, rows=None, u_before=None, u_after=None, check_meta=True):
+    a = host_arrays(w_cpu)
+    rows = list(range(w_cpu.B)) if rows is None else list(rows)
+    pt, sl, q = a["page_table"][rows], a["seq_lens"][rows], a["q"][rows]
+    # --- summaries
+    meta_gpu = wl.bf16_bits(st.meta)
+    if check_meta:
+        meta_ref = oracle.quest_meta(a["k"], pt, sl, first_tok=np.zeros(len(rows), np.int32), meta=meta_gpu)
+        assert np.array_equal(meta_ref, meta_gpu), "page summaries differ"
+    # --- selection
+    S, P, present = oracle.quest_scores(q, meta_gpu, pt, sl)
+    sel = st.sel_idx.cpu().numpy()[rows]
+    cnt = st.sel_cnt.cpu().numpy()[rows]
+    differing = check_selection(sel, cnt, P, present, w_cpu.budget)
+    assert differing <= max(1, (len(rows) * w_cpu.H_kv) // 4), "too many rows differ inside the tie band"
+    for r in range(len(rows)):
+        for h in range(w_cpu.H_kv):
+            row = sel[r, h, :cnt[r, h]]
+            assert np.all(np.diff(row) > 0), "selection must be ascending"
+    # --- attention on the GPU's selection
+    u_ref = None
+    if u_before is not None:
+        u_ref = u_before.astype(np.float64).copy()
+    out_ref, lse_ref = oracle.attend(q, a["k"], a["v"], pt, sl, sel, cnt, u_accum=u_ref)
+    out = st.out.cpu().numpy()[rows].astype(np.float64)
+    lse = st.lse.cpu().numpy()[rows].astype(np.float64)
+    empty = np.isneginf(lse_ref)
+    assert np.array_equal(np.isneginf(lse), empty)
+    assert np.all(np.isfinite(out))
+    err = np.abs(out - out_ref)
+    assert err.max() <= OUT_MAX_ABS, err.max()
+    assert err.mean() <= OUT_MEAN_ABS, err.mean()
+    assert np.abs(lse[~empty] - lse_ref[~empty]).max(initial=0.0) <= LSE_ABS
+    if u_before is not None:
+        du_gpu = u_after.astype(np.float64) - u_before.astype(np.float64)
+        du_ref = u_ref - u_before.astype(np.float64)
+        assert np.all(np.abs(du_gpu - du_ref) <= 1e-4 + 1e-3 * du_ref + 2e-7 * np.abs(u_before))
+        G = w_cpu.H_q // w_cpu.H_kv
+        touched = du_ref != 0
+        assert np.all(du_gpu[~touched] == 0)
+    return dict(out_err=err.max(), differing=differing)
+
+
+EDGE_CASES = {
+    "len1":            dict(seq=[1], H_q=4, H_kv=1, D=128, budget=64),
+    "len17_partial":   dict(seq=[17, 33, 16, 15], H_q=8, H_kv=2, D=128, budget=16, poison_tail=True),
+    "k_ge_pages":      dict(seq=[100, 260, 40], H_q=8, H_kv=2, D=64, budget=16 * 32, poison_tail=True),
+    "padding_slot":    dict(seq=[0, 300, 0, 77], H_q=8, H_kv=2, D=128, budget=64),
+    "permuted":        dict(seq=[700, 1300, 257, 2049], H_q=8, H_kv=2, D=128, budget=256,
+                            permute_pool=True, poison_tail=True, spare_pages=3),
+    "aliased_prefix":  dict(seq=[900, 1100, 650], H_q=8, H_kv=2, D=128, budget=128,
+                            permute_pool=True, shared_prefix_pages=20),
+    "pruned":          dict(seq=[1500, 900, 333], H_q=8, H_kv=2, D=128, budget=128,
+                            permute_pool=True, prune_fraction=0.3, poison_tail=True),
+    "mostly_pruned":   dict(seq=[640, 320], H_q=4, H_kv=2, D=64, budget=128, prune_fraction=0.97),
+    "outliers":        dict(seq=[3000, 1000], H_q=8, H_kv=2, D=128, budget=512, outliers=True),
+    "many_requests":   dict(seq=list(range(5, 5 + 70 * 37, 37)), H_q=4, H_kv=2, D=64, budget=96,
+                            permute_pool=True, poison_tail=True),
+}
+
+
+@pytest.mark.parametrize("name", sorted(EDGE_CASES))
+def test_edge_cases(name):
+    kw = dict(EDGE_CASES[name])
+    seq = kw.pop("seq")
+    w_cpu = wl.build(name, 800, 0, seq, kw.pop("H_q"), kw.pop("H_kv"), kw.pop("D"), kw.pop("budget"), "cpu", **kw)
+    w, st, _ = run_gpu(w_cpu)
+    compare(w_cpu, st)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_every_group_size(D, G):
+    w_cpu = wl.build("g", 810 + G, 0, [1234, 77, 600], 2 * G, 2, D, 160, "cpu", permute_pool=True,
+                     poison_tail=True)
+    w, st, _ = run_gpu(w_cpu)
+    compare(w_cpu, st)
+
+
+def test_all_pages_pruned_gives_empty_result():
+    w_cpu = wl.build("gone", 820, 0, [200, 90], 8, 2, 128, 64, "cpu")
+    w_cpu.page_table[0, :] = -1
+    w, st, _ = run_gpu(w_cpu)
+    assert st.sel_cnt.cpu()[0].tolist() == [0, 0]
+    assert torch.all(st.out[0] == 0) and torch.all(torch.isneginf(st.lse[0]))
+    compare(w_cpu, st)
+
+
+def test_budget_covering_everything_is_dense_attention():
+    """Selected attention with every page selected must equal dense attention (torch SDPA, fp64)."""
+    w_cpu = wl.build("dense", 830, 0, [777, 1500], 8, 2, 128, 16 * 128, "cpu", permute_pool=True)
+    w, st, _ = run_gpu(w_cpu)
+    a = host_arrays(w_cpu)
+    from helpers import bits_to_f64, tokens_of_request
+    K, V, Q = bits_to_f64(a["k"]), bits_to_f64(a["v"]), bits_to_f64(a["q"])
+    for r in range(w_cpu.B):
+        toks = tokens_of_request(a["page_table"][r], a["seq_lens"][r], 16)
+        for h in range(w_cpu.H_kv):
+            Kd = torch.from_numpy(np.stack([K[pid, h, t] for (_, t, pid) in toks]))[None, None]
+            Vd = torch.from_numpy(np.stack([V[pid, h, t] for (_, t, pid) in toks]))[None, None]
+            for g in range(4):
+                head = h * 4 + g
+                qq = torch.from_numpy(Q[r, head])[None, None, None]
+                o = torch.nn.functional.scaled_dot_product_attention(qq, Kd, Vd)[0, 0, 0].numpy()
+                assert np.abs(st.out[r, head].cpu().numpy() - o).max() <= OUT_MAX_ABS
+
+
+def test_incremental_summary_update_matches_rebuild():
+    """Append one token per request: updating only the newest page equals a rebuild."""
+    w_cpu = wl.build("inc", 840, 0, [161, 320, 49, 16], 8, 2, 128, 64, "cpu", permute_pool=True)
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w)
+    short = (w.seq_lens - 1).contiguous()
+    ft = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    binding.se_meta_update(st.p, w.k_cache, w.page_table, short, st.meta, first_tok=ft)
+    before = st.meta.clone()
+    st.update_meta()                                   # only the page of the newest token
+    inc = st.meta.clone()
+    st.meta.zero_()
+    st.rebuild_meta()
+    torch.cuda.synchronize()
+    assert torch.equal(inc.view(torch.int16), st.meta.view(torch.int16))
+    assert not torch.equal(before.view(torch.int16), inc.view(torch.int16))
+    # a rebuild from a given token on touches only pages from there
+    st.meta.zero_()
+    ft2 = torch.full((w.B,), 32, dtype=torch.int32, device="cuda")
+    binding.se_meta_update(st.p, w.k_cache, w.page_table, w.seq_lens, st.meta, first_tok=ft2)
+    torch.cuda.synchronize()
+    pt = w.page_table.cpu()
+    for r in range(w.B):
+        n_r = (int(w.seq_lens[r]) + 15) // 16
+        for b in range(n_r):
+            touched = bool(st.meta[pt[r, b]].view(torch.int16).ne(0).any())
+            assert touched == (b >= 2), (r, b)
+
+
+def test_summary_signed_zero_and_masking():
+    w_cpu = wl.build("zero", 850, 0, [20], 2, 1, 64, 32, "cpu", poison_tail=True)
+    w_cpu.k_cache[0, 0, 0, 0] = 0.0
+    w_cpu.k_cache[0, 0, 1:, 0] = -0.0
+    w_cpu.k_cache[0, 0, 0, 1] = -0.0
+    w_cpu.k_cache[0, 0, 1:, 1] = 0.0
+    w, st, _ = run_gpu(w_cpu)
+    compare(w_cpu, st)
+    bits = wl.bf16_bits(st.meta)
+    assert bits[0, 0, 0, 0] == 0x8000 and bits[0, 0, 1, 0] == 0x0000
+    assert bits[0, 0, 0, 1] == 0x8000 and bits[0, 0, 1, 1] == 0x0000
+
+
+def test_ties_go_to_the_lower_page_and_inputs_are_not_written():
+    """Identical pages score identically: the lower logical pages must win, and select/decode
+    must leave q, K, V, summaries and the page table untouched."""
+    w_cpu = wl.build("ties", 860, 0, [16 * 40], 4, 1, 128, 16 * 8, "cpu")
+    w_cpu.k_cache[1:] = w_cpu.k_cache[0]
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    torch.cuda.synchronize()
+    snap = [t.clone() for t in (w.q, w.k_cache, w.v_cache, st.meta, w.page_table, w.seq_lens)]
+    st.select()
+    st.decode()
+    torch.cuda.synchronize()
+    assert st.sel_idx.cpu()[0, 0].tolist() == list(range(8))
+    for s, t in zip(snap, (w.q, w.k_cache, w.v_cache, st.meta, w.page_table, w.seq_lens)):
+        assert torch.equal(s.view(torch.uint8), t.view(torch.uint8))
+    compare(w_cpu, st)
+
+
+def test_two_runs_are_bit_identical_and_split_invariant():
+    w_cpu = wl.build("det", 870, 0, [5000, 3000, 9000], 8, 2, 128, 1024, "cpu", permute_pool=True)
+    w, st, _ = run_gpu(w_cpu)
+    o1, l1, s1 = st.out.clone(), st.lse.clone(), st.sel_idx.clone()
+    st.out.fill_(float("nan"))
+    st.select()
+    st.decode()
+    torch.cuda.synchronize()
+    assert torch.equal(o1, st.out) and torch.equal(l1, st.lse) and torch.equal(s1, st.sel_idx)
+    # a larger k_max changes how the selected pages are split over warps, not the result
+    st2 = binding.DecodeState(w, k_max=200)
+    st2.rebuild_meta()
+    st2.select()
+    st2.decode()
+    torch.cuda.synchronize()
+    assert torch.equal(st2.sel_idx[:, :, :64], s1)
+    assert (st2.out - o1).abs().max().item() <= 1e-5
+    assert (st2.lse - l1).abs().max().item() <= 1e-5
+
+
+def test_h2o_accumulation_small():
+    w_cpu = wl.build("h2o", 880, 0, [700, 1300, 90], 8, 2, 128, 256, "cpu", permute_pool=True,
+                     with_score_accum=True, poison_tail=True)
+    w, st, u = run_gpu(w_cpu, accum=True)
+    res = compare(w_cpu, st, u_before=w_cpu.score_accum.numpy(), u_after=u.cpu().numpy())
+    # mass conservation: every (request, kv-head) adds exactly G
+    du = (u - w.score_accum).double()
+    assert abs(du.sum().item() - w_cpu.B * w_cpu.H_q) <= 1e-3 * w_cpu.B * w_cpu.H_q
+    # a second step adds the same amount again
+    st.decode(score_accum=u)
+    torch.cuda.synchronize()
+    du2 = (u - w.score_accum).double()
+    assert torch.allclose(du2, 2 * du, rtol=1e-4, atol=1e-5)
+
+
+def test_bad_selection_sets_status_and_is_skipped():
+    w_cpu = wl.build("bad", 890, 0, [400, 400], 8, 2, 128, 64, "cpu")
+    w, st, _ = run_gpu(w_cpu)
+    good = st.out.clone()
+    st.sel_idx[0, 0, 1] = 10_000                      # outside the request
+    st.decode()
+    torch.cuda.synchronize()
+    assert st.status() & binding.SE_DEV_BAD_SELECTION
+    assert torch.all(torch.isfinite(st.out))
+    assert torch.equal(good[1], st.out[1])
+    assert st.status() == 0                            # reading the status clears it
+
+
+# ---------------------------------------------------------------- the named configurations
+
+def test_config1_tiny():
+    w_cpu = wl.config1("cpu")
+    w, st, _ = run_gpu(w_cpu)
+    compare(w_cpu, st)
+
+
+def test_config2_llama8b_layer():
+    w_cpu = wl.config2("cpu")
+    w, st, _ = run_gpu(w_cpu)
+    compare(w_cpu, st)
+
+
+def _gpu_built(cfg_fn, **kw):
+    """Full-size workload generated on the GPU; the host copy for the oracle shares its bits."""
+    w = cfg_fn("cuda", **kw)
+    return w, w.to("cpu")
+
+
+def test_config3_full_size_sampled_requests():
+    w, w_cpu = _gpu_built(wl.config3)
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    st.step()
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    lens = w_cpu.seq_lens.numpy()
+    rows = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 0, 17, 42, 63})
+    compare(w_cpu, st, rows=rows)
+
+
+def test_config4_long_context_with_h2o():
+    w, w_cpu = _gpu_built(wl.config4)
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    u = w.score_accum.clone()
+    st.step(score_accum=u)
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    compare(w_cpu, st, u_before=w_cpu.score_accum.numpy(), u_after=u.cpu().numpy())
+    du = (u - w.score_accum).double()
+    assert abs(du.sum().item() - w.B * w.H_q) <= 1e-3 * w.B * w.H_q
+
+
+@pytest.mark.parametrize("layer", [0, 27])
+def test_config5_one_layer_sampled_requests(layer):
+    w, w_cpu = _gpu_built(wl.config5, layer=layer)
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    st.step()
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    lens = w_cpu.seq_lens.numpy()
+    rows = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 1, 64, 127})
+    compare(w_cpu, st, rows=rows)
