@@ -1,0 +1,464 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse decode-attention hot path.
+
+A *step* is one pass of the whole path over one batch of synthetic requests, per layer:
+``se_meta_update`` (summary of the page holding each request's newest token) ->
+``se_page_select`` (page scores + top-k) -> ``se_sparse_decode`` (split-K attention over the
+selected pages, LSE merge, optional H2O statistic).  The default workload is the
+continuous-batching mix (config 3: 64 requests, 4096..65536 tokens, 32/8 heads, D=128,
+budget 2048, page tables permuted over one pool); ``--config`` picks another one.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+N > 1 is launched with torch.distributed.run, one rank per GPU; every rank runs the same
+shape on its own data (the path shards by request / kv-head without any collective), so
+scaling is weak.  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2609_39068_b200 import workloads as wl
+
+METRIC = "sparse_decode_us_per_step"
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
+# capture summarised in profiles/ (null until a capture of that workload exists)
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while running."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_sm = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                sm = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), sm, reasons))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_sm, "reasons": ["unavailable"]}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = None
+        if not inside:                       # timed region shorter than one sampling period
+            inside = sorted(self.samples, key=lambda s: abs(s[0] - 0.5 * (t0 + t1)))[:3]
+            note = "nearest_samples"
+        names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        bits = 0
+        for s in inside:
+            bits |= int(s[2])
+        reasons = [n for b, n in names.items() if bits & b]
+        out = {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.max_sm,
+               "reasons": reasons, "samples": len(inside)}
+        if note:
+            out["note"] = note
+        return out
+
+
+# ------------------------------------------------------------------ workload accounting
+def algorithmic_bytes(w, sel_cnt, h2o: bool):
+    """Bytes the method must move per step (per layer): summaries of every present page,
+    K and V of the selected pages, q, out, lse (+ the H2O read-modify-write)."""
+    pt = w.page_table.cpu().numpy()
+    sl = w.seq_lens.cpu().numpy()
+    n_r = (sl + 15) // 16
+    present = sum(int((pt[r, :n_r[r]] >= 0).sum()) for r in range(w.B))
+    meta = present * w.H_kv * 2 * w.D * 2
+    k_eff = int(sel_cnt.sum().item())
+    kv = k_eff * 16 * w.D * 2 * 2
+    q = w.B * w.H_q * w.D * 2
+    outlse = w.B * w.H_q * (4 * w.D + 4)
+    accum = 0
+    if h2o:
+        accum = 2 * 4 * 16 * k_eff          # upper bound: every slot of every selected page
+    return dict(meta=meta, kv=kv, q=q, outlse=outlse, accum=accum,
+                select_call=meta + q, decode_kernel=kv + q + outlse,
+                total=meta + kv + q + outlse + accum, present_pages=present, selected_pages=k_eff)
+
+
+def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0):
+    fn = wl.CONFIGS[config]
+    if batch:
+        base = fn
+        fn = lambda device, layer=0: base(device, layer=layer, B=batch)
+    layers = []
+    first = None
+    for l in range(n_layers):
+        w = fn(device, layer=l + 100 * rank) if config != 5 else fn(device, layer=l)
+        if first is None:
+            first = w
+        else:                                 # the block table is per request, shared by all layers
+            w.page_table, w.seq_lens = first.page_table, first.seq_lens
+        layers.append(w)
+    return layers
+
+
+# ------------------------------------------------------------------ CPU oracle timing
+def oracle_time(w, target_s=(10.0, 30.0)):
+    """Times the oracle, as it stands, on a bounded sample of the workload's requests and
+    scales to the full batch by the number of (present + selected) pages."""
+    import oracle
+    order = list(range(0, w.B, max(1, w.B // 16)))[:16]
+    sub = wl.sub_workload(w, order, "cpu")
+    q, k, v = wl.bf16_bits(sub.q), wl.bf16_bits(sub.k_cache), wl.bf16_bits(sub.v_cache)
+    pt, sl = sub.page_table.numpy(), sub.seq_lens.numpy()
+    meta = oracle.quest_meta(k, pt, sl, first_tok=np.zeros(sub.B, np.int32))
+    u = None if sub.score_accum is None else sub.score_accum.numpy().astype(np.float64)
+    times = []
+    t_begin = time.perf_counter()
+    while len(times) < 3 or (time.perf_counter() - t_begin < target_s[0] and len(times) < 50):
+        t0 = time.perf_counter()
+        oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
+        times.append(time.perf_counter() - t0)
+        if time.perf_counter() - t_begin > target_s[1]:
+            break
+    n_all = (w.seq_lens.cpu().numpy() + 15) // 16
+    n_sub = (sl + 15) // 16
+    scale = float(n_all.sum()) / float(n_sub.sum())
+    best = min(times)
+    return dict(value=best * scale * 1e6, unit="us", cores=oracle.num_threads(), kind="oracle",
+                sample="%d of %d requests (every %d-th), fp64 C oracle with OpenMP over (request, kv-head), "
+                       "best of %d runs = %.1f ms, scaled x%.2f by page count to the full batch"
+                       % (sub.B, w.B, max(1, w.B // 16), len(times), best * 1e3, scale),
+                sample_seconds=best)
+
+
+# ------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3, choices=sorted(wl.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="layers per step (default 1; 28 for config 5)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the number of requests (configs 3-5; for small profiling captures)")
+    ap.add_argument("--no-graph", action="store_true", help="launch the calls directly instead of a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    n_layers = args.layers or (28 if args.config == 5 else 1)
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, n_layers)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2609_39068_b200 import binding
+    binding.load()
+
+    layers = make_layers(args.config, dev, n_layers, rank, args.batch)
+    h2o = layers[0].score_accum is not None
+    states = [binding.DecodeState(w) for w in layers]
+    accums = [w.score_accum.clone() if h2o else None for w in layers]
+    for st in states:
+        st.rebuild_meta()
+    torch.cuda.synchronize()
+
+    def step():
+        for st, u in zip(states, accums):
+            st.step(score_accum=u)
+
+    step()
+    torch.cuda.synchronize()
+    for st in states:
+        if st.status() != 0:
+            raise SystemExit("device status word not clean")
+    bytes_l = [algorithmic_bytes(st.w, st.sel_cnt, h2o) for st in states]
+    total_bytes = sum(b["total"] for b in bytes_l)
+    working_set = total_bytes
+    flush = working_set < 2 * L2_BYTES
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
+
+    graph = None
+    if not args.no_graph:
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            step()
+        torch.cuda.current_stream().wait_stream(s)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+    run_step = graph.replay if graph is not None else step
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        run_step()
+    barrier()
+    K = args.steps
+    t_wall0 = time.perf_counter()
+    if flush:
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        for i in range(K):
+            flush_buf.fill_(i & 0xFF)
+            starts[i].record()
+            run_step()
+            ends[i].record()
+        barrier()
+        total_ms = sum(a.elapsed_time(b) for a, b in zip(starts, ends))
+    else:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            run_step()
+        e1.record()
+        barrier()
+        total_ms = e0.elapsed_time(e1)
+    t_wall1 = time.perf_counter()
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    # ---- per-call timing (same stream, CUDA events, each call in its own loop)
+    def time_call(fn, iters):
+        for _ in range(3):
+            fn()
+        if flush:
+            tot = 0.0
+            for i in range(iters):
+                flush_buf.fill_(i & 0xFF)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                tot += a.elapsed_time(b)
+            return tot / iters * 1e3
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters * 1e3
+
+    iters = max(10, min(K, 200))
+    st0, u0 = states[0], accums[0]
+    call_us = {
+        "se_meta_update": time_call(st0.update_meta, iters),
+        "se_page_select": time_call(st0.select, iters),
+        "se_sparse_decode": time_call(lambda: st0.decode(u0), iters),
+    }
+    b0 = bytes_l[0]
+    peak, peak_kind = measured_peak()
+    dec_gbs = b0["decode_kernel"] / (call_us["se_sparse_decode"] * 1e-6) / 1e9
+    sel_gbs = b0["select_call"] / (call_us["se_page_select"] * 1e-6) / 1e9
+    step_gbs = total_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the public API with host buffers
+    pinned_in = [(w.q.cpu().pin_memory(), w.seq_lens.cpu().pin_memory(), w.page_table.cpu().pin_memory())
+                 for w in layers]
+    pinned_out = [(torch.empty(st.out.shape, dtype=torch.float32).pin_memory(),
+                   torch.empty(st.lse.shape, dtype=torch.float32).pin_memory()) for st in states]
+    h2d = sum(sum(t.numel() * t.element_size() for t in tri) for tri in pinned_in)
+    d2h = sum(sum(t.numel() * t.element_size() for t in pair) for pair in pinned_out)
+
+    def e2e_step():
+        for w, st, u, pin, pout in zip(layers, states, accums, pinned_in, pinned_out):
+            w.q.copy_(pin[0], non_blocking=True)
+            w.seq_lens.copy_(pin[1], non_blocking=True)
+            w.page_table.copy_(pin[2], non_blocking=True)
+            st.step(score_accum=u)
+            pout[0].copy_(st.out, non_blocking=True)
+            pout[1].copy_(st.lse, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    e2e_iters = max(10, min(K, 200))
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(e2e_iters):
+        if flush:
+            flush_buf.fill_(i & 0xFF)
+        e2e_step()
+    b.record()
+    barrier()
+    e2e_ms = a.elapsed_time(b) / e2e_iters
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    sampler.stop()
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_time(layers[0])
+        if n_layers > 1:
+            cpu_baseline["value"] *= n_layers
+            cpu_baseline["sample"] += "; one layer timed, x%d layers" % n_layers
+
+    if rank == 0:
+        launches_per_step = n_layers * (5 if h2o else 4)
+        line = {
+            "metric": METRIC, "value": ms_per_step * 1e3, "unit": "us", "n_gpus": world,
+            "steps": K, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": layers[0].name, "config_id": args.config, "layers": n_layers,
+                "B": layers[0].B, "H_q": layers[0].H_q, "H_kv": layers[0].H_kv, "D": layers[0].D,
+                "page_size": 16, "budget_tokens": layers[0].budget, "storage_dtype": "bf16",
+                "present_pages": b0["present_pages"], "selected_pages": b0["selected_pages"],
+                "h2o_epilogue": h2o, "cuda_graph": graph is not None,
+                "l2": ("flushed with a %d MiB write before every step" % (2 * L2_BYTES >> 20)) if flush
+                      else "inputs larger than L2 (%.0f MB touched per step)" % (working_set / 1e6),
+                "parallelism": "1 GPU" if world == 1 else "%d replicas, no collective" % world,
+            },
+            "algorithmic_bytes_per_step": total_bytes,
+            "achieved_gbs": step_gbs * world,
+            "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+            "frac_of_measured_copy": step_gbs / peak,
+            "calls_us": call_us,
+            "calls_gbs": {"se_page_select": sel_gbs, "se_sparse_decode": dec_gbs},
+            "roofline": {
+                "bound": "hbm", "kernel": "decode_kernel (se_sparse_decode)", "achieved": dec_gbs,
+                "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": dec_gbs / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get(layers[0].name),
+                "algorithmic_bytes": b0["decode_kernel"],
+            },
+            "clocks": clocks,
+            "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches_per_step * K,
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def run_reference(args, n_layers):
+    """Reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    import oracle
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    if dev == "cpu" and args.config in (3, 4, 5):
+        kw = {3: dict(B=4), 4: dict(B=1, length=32768), 5: dict(B=8)}[args.config]
+        w = wl.CONFIGS[args.config](dev, **kw)
+        note = "generated on the CPU at reduced batch (%s)" % kw
+    else:
+        w = wl.CONFIGS[args.config](dev)
+        note = "full workload generated on the GPU, sample copied to the host"
+    order = list(range(0, w.B, max(1, w.B // 16)))[:16]
+    sub = wl.sub_workload(w, order, "cpu")
+    q, k, v = wl.bf16_bits(sub.q), wl.bf16_bits(sub.k_cache), wl.bf16_bits(sub.v_cache)
+    pt, sl = sub.page_table.numpy(), sub.seq_lens.numpy()
+    meta = oracle.quest_meta(k, pt, sl, first_tok=np.zeros(sub.B, np.int32))
+    u = None if sub.score_accum is None else sub.score_accum.numpy().astype(np.float64)
+    n_all = (w.seq_lens.cpu().numpy() + 15) // 16
+    scale = float(n_all.sum()) / float(((sl + 15) // 16).sum()) * n_layers
+    steps = max(1, min(args.steps, 20))
+    warm = max(1, min(args.warmup, 3))
+    for _ in range(warm):
+        oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
+    per = (time.perf_counter() - t0) / steps
+    val = per * scale * 1e6
+    sample = ("%d of %d requests per step (%s), %.1f ms per sample step, scaled x%.2f by page count%s"
+              % (sub.B, w.B, note, per * 1e3, scale, " and layers" if n_layers > 1 else ""))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "us", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": val / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "config_id": args.config, "layers": n_layers},
+        "cpu_baseline": {"value": val, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()
