@@ -27,6 +27,7 @@ int validate(const se_params *p) {
     // index arithmetic inside the kernels uses 32-bit page counts and 64-bit byte offsets
     if ((long long)p->B * p->H_kv > (1ll << 24)) return SE_ERR_INVALID_ARG;
     if ((long long)p->B * p->max_pages > (1ll << 31) - 1) return SE_ERR_INVALID_ARG;
+    if ((long long)p->num_phys_pages * p->H_kv * kPage > (1ll << 31) - 1) return SE_ERR_INVALID_ARG;
     return SE_OK;
 }
 

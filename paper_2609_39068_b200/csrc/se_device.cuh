@@ -102,6 +102,33 @@ __device__ __forceinline__ uint32_t f32_key(float f) {
 
 constexpr uint32_t kKeyAbsent = 0x007fffffu;   // f32_key(-inf): below every finite score
 
+// ---------------------------------------------------------------------------------
+// warp-level matrix helpers (bf16 inputs, fp32 accumulation)
+// ---------------------------------------------------------------------------------
+// Four 8x8 b16 matrices from shared memory; lane l supplies the address of row (l & 7) of
+// matrix (l >> 3) and receives, from matrix i, elements (row l>>2, columns 2*(l&3), +1).
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+// Same, each matrix transposed on the way in.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+// D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 __host__ __device__ constexpr int next_pow2(int x) {
     int p = 1;
     while (p < x) p <<= 1;

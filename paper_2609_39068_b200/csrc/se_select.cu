@@ -2,19 +2,22 @@
 // the notation table).
 //
 // score_kernel   streams the page summaries.  Every warp is an autonomous pipeline: it owns
-//                two shared-memory buffers of PB page summaries, fills them with 1-D bulk
+//                two shared-memory buffers of 16 page summaries, fills them with 1-D bulk
 //                asynchronous copies (one per page and head, completion on an mbarrier) and
 //                computes on one buffer while the other is in flight.  The bound
 //                    sum_c max(q_c*m_c, q_c*M_c)
-//                is evaluated exactly as  sum_c (q_c^- * m_c + q_c^+ * M_c)  with
-//                q^+ = max(q,0), q^- = min(q,0): because M >= m one of the two products is the
-//                maximum and the other factor is zero.  Products of bf16 values are exact in
-//                fp32, accumulation is fp32 with packed two-wide FMAs, the G query heads of a
-//                kv-head share every summary load, and the per-page sums over the lanes that
-//                share a page are formed by a transposing shuffle reduction.
+//                equals  sum_c (q_c^- * m_c + q_c^+ * M_c)  with q^+ = max(q,0), q^- = min(q,0)
+//                (M >= m, so one product is the maximum and the other factor is zero).  That
+//                is a dense [16 pages x 2D] . [2D x G] contraction per batch: the summaries
+//                are the row-major A operand straight out of shared memory (rows padded by
+//                16 bytes so that ldmatrix is bank-conflict free), (q^-|q^+) of the G query
+//                heads is the B operand held in registers, products of bf16 values are exact
+//                and accumulate in fp32.  An earlier plain-FMA version of this kernel was
+//                issue-bound at 64 % of the copy bandwidth (57 warp instructions per page
+//                summary); this one needs 3.
 // topk_kernel    one CTA per (request, kv-head): most-significant-digit radix select over
-//                order-preserving integer keys, then an index-ordered compaction, so equal
-//                scores go to the lower page and the list comes out ascending.
+//                order-preserving integer keys held in registers, then an index-ordered
+//                compaction, so equal scores go to the lower page and the list is ascending.
 #include "se_internal.h"
 
 namespace se {
@@ -22,24 +25,16 @@ namespace se {
 namespace {
 
 constexpr int kScoreWarps = 4;     // warps per CTA of the score kernel
-constexpr int kPB = 16;            // pages per warp batch
+constexpr int kPB = 16;            // pages per warp batch (one m16 tile)
 constexpr int kNBU = 4;            // batches per work unit  -> 64 pages per (pair, unit)
 constexpr int kUnitPages = kPB * kNBU;
 
-template <int D, int G>
+template <int D>
 struct ScoreCfg {
-    static constexpr int GP = next_pow2(G);
-    static constexpr int CPL = (G > 4) ? 4 : 8;         // channels per lane and row
-    static constexpr int LPP = D / CPL;                 // lanes sharing one (page, head)
-    static constexpr int PPP = 32 / LPP;                // pages per warp pass
-    static constexpr int NPS = kPB / PPP;               // passes per batch
-    static constexpr int RB = (NPS < 32 / GP) ? NPS : 32 / GP;   // passes per reduction block
-    static constexpr int NV = RB * GP;                  // partial sums per lane and block
-    static constexpr int NF = (NV / LPP) > 1 ? (NV / LPP) : 1;
-    static constexpr int LPG = LPP / RB;                // lanes that end up holding one page
-    static constexpr int PHB = 2 * D * 2;               // bytes of one page summary
-    static_assert(NPS % RB == 0, "reduction blocks tile the batch");
-    static_assert(LPG >= 1, "");
+    static constexpr int PHB = 2 * D * 2;               // bytes of one page summary (min row, max row)
+    static constexpr int PITCH = PHB + 16;              // shared-memory pitch of a summary
+    static constexpr int KSTEPS = 2 * D / 16;           // k16 steps over (min row | max row)
+    static constexpr int BUF = kPB * PITCH;             // one buffer
 };
 
 struct Batch {
@@ -70,17 +65,17 @@ __device__ __forceinline__ bool decode_unit(int u, int total_units, const int *p
     return true;
 }
 
-template <int D, int G>
+template <int D>
 __global__ void __launch_bounds__(kScoreWarps * 32)
 score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
              const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
-             float *__restrict__ scores, int B, int H_kv, int max_pages, int P_phys, float scale,
+             float *__restrict__ scores, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
              uint32_t *status) {
-    using C = ScoreCfg<D, G>;
+    using C = ScoreCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    // layout: [buffers: warps*2*PB*PHB] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints]
+    // layout: [buffers: warps*2*BUF] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints]
     uint8_t *bufs = smem_raw;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)kScoreWarps * 2 * kPB * C::PHB);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)kScoreWarps * 2 * C::BUF);
     int *prefix = reinterpret_cast<int *>(bars + kScoreWarps * 2);
     int *npages = prefix + (B + 1);
 
@@ -121,36 +116,36 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
     const int gw = blockIdx.x * kScoreWarps + warp;
     const int tw = gridDim.x * kScoreWarps;
 
-    uint8_t *my_buf = bufs + (size_t)warp * 2 * kPB * C::PHB;
+    uint8_t *my_buf = bufs + (size_t)warp * 2 * C::BUF;
+    const uint32_t buf0 = smem_u32(my_buf);
     const uint32_t bar0 = smem_u32(&bars[warp * 2]);
-    const int pp = lane / C::LPP, lg = lane % C::LPP;
+    const int gid = lane >> 2, tid4 = lane & 3;      // fragment coordinates of this lane
 
-    // q registers of the current pair: q^- multiplies the min row, q^+ the max row
-    float2 qn[G][C::CPL / 2], qp[G][C::CPL / 2];
-    uint32_t qraw[G][C::CPL / 2];            // raw bf16 pairs of the pair whose batch was issued last
-    int q_r = -1, q_h = -1;                  // pair the converted registers belong to
+    // B operand: column n = query head n of the group (zero for n >= G); rows k < D carry q^-
+    // (they meet the min row), rows k >= D carry q^+ (they meet the max row).
+    uint32_t bfrag[C::KSTEPS][2];
+    uint32_t qraw[D / 16][2];                // raw q pairs of the pair whose batch was issued last
+    int q_r = -1, q_h = -1;                  // pair the fragments belong to
 
     auto load_qraw = [&](const Batch &d) {
+        const uint16_t *src = q + ((size_t)d.r * H_q + d.h * G + (gid < G ? gid : 0)) * D + 2 * tid4;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const uint16_t *src = q + ((size_t)d.r * H_q + d.h * G + g) * D + lg * C::CPL;
-            if constexpr (C::CPL == 8) {
-                const uint4 w = __ldg(reinterpret_cast<const uint4 *>(src));
-                qraw[g][0] = w.x; qraw[g][1] = w.y; qraw[g][2] = w.z; qraw[g][3] = w.w;
-            } else {
-                const uint2 w = __ldg(reinterpret_cast<const uint2 *>(src));
-                qraw[g][0] = w.x; qraw[g][1] = w.y;
-            }
+        for (int s = 0; s < D / 16; ++s) {
+            const uint32_t w0 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16));
+            const uint32_t w1 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16 + 8));
+            qraw[s][0] = gid < G ? w0 : 0u;
+            qraw[s][1] = gid < G ? w1 : 0u;
         }
     };
     auto convert_q = [&]() {
 #pragma unroll
-        for (int g = 0; g < G; ++g)
+        for (int s = 0; s < D / 16; ++s)
 #pragma unroll
-            for (int j = 0; j < C::CPL / 2; ++j) {
-                const float2 f = bf16x2_to_f2(qraw[g][j]);
-                qp[g][j] = make_float2(fmaxf(f.x, 0.f), fmaxf(f.y, 0.f));
-                qn[g][j] = make_float2(fminf(f.x, 0.f), fminf(f.y, 0.f));
+            for (int j = 0; j < 2; ++j) {
+                const uint32_t w = qraw[s][j];
+                const uint32_t negmask = ((w >> 15) & 0x00010001u) * 0xffffu;   // all-ones per negative half
+                bfrag[s][j] = w & negmask;                   // q^-  (min row part)
+                bfrag[D / 16 + s][j] = w & ~negmask;         // q^+  (max row part)
             }
     };
 
@@ -184,7 +179,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
         __syncwarp();
         if (pid >= 0) {
             const uint8_t *src = meta + ((size_t)pid * H_kv + d.h) * C::PHB;
-            bulk_g2s(smem_u32(my_buf + ((size_t)slot * kPB + lane) * C::PHB), src, C::PHB, bar);
+            bulk_g2s(buf0 + slot * C::BUF + lane * C::PITCH, src, C::PHB, bar);
         }
         return pid;
     };
@@ -199,10 +194,14 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
     int pid_nxt = -1;
     bool failed = false;
 
+    // ldmatrix row address of this lane inside a buffer: matrix (lane>>3) = {pages 0-7 | 8-15} x
+    // {first | second 16-byte piece of the k16 step}
+    const uint32_t lm_off = (uint32_t)(((lane & 7) + 8 * ((lane >> 3) & 1)) * C::PITCH + (lane >> 4) * 16);
+
     while (cur.unit >= 0) {
         nxt = cur;
         next_batch(nxt);
-        // the pair of `cur` may differ from the converted registers: convert before qraw is reused
+        // the pair of `cur` may differ from the converted fragments: convert before qraw is reused
         if (cur.r != q_r || cur.h != q_h) {
             convert_q();
             q_r = cur.r;
@@ -219,64 +218,28 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
         }
         phases ^= (1u << slot);
 
-        const uint8_t *buf = my_buf + (size_t)slot * kPB * C::PHB;
-        float *dst = scores + ((size_t)cur.r * H_kv + cur.h) * max_pages + cur.b0;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t a_base = buf0 + slot * C::BUF + lm_off;
 #pragma unroll
-        for (int rb = 0; rb < C::NPS / C::RB; ++rb) {
-            float v[C::NV];
-#pragma unroll
-            for (int ip = 0; ip < C::RB; ++ip) {
-                const int j = (rb * C::RB + ip) * C::PPP + pp;          // page inside the batch
-                const uint8_t *pg = buf + (size_t)j * C::PHB + lg * (C::CPL * 2);
-                uint32_t mnw[C::CPL / 2], mxw[C::CPL / 2];
-                if constexpr (C::CPL == 8) {
-                    const uint4 a = *reinterpret_cast<const uint4 *>(pg);
-                    const uint4 b = *reinterpret_cast<const uint4 *>(pg + D * 2);
-                    mnw[0] = a.x; mnw[1] = a.y; mnw[2] = a.z; mnw[3] = a.w;
-                    mxw[0] = b.x; mxw[1] = b.y; mxw[2] = b.z; mxw[3] = b.w;
-                } else {
-                    const uint2 a = *reinterpret_cast<const uint2 *>(pg);
-                    const uint2 b = *reinterpret_cast<const uint2 *>(pg + D * 2);
-                    mnw[0] = a.x; mnw[1] = a.y;
-                    mxw[0] = b.x; mxw[1] = b.y;
-                }
-                float2 mnf[C::CPL / 2], mxf[C::CPL / 2];
-#pragma unroll
-                for (int c = 0; c < C::CPL / 2; ++c) {
-                    mnf[c] = bf16x2_to_f2(mnw[c]);
-                    mxf[c] = bf16x2_to_f2(mxw[c]);
-                }
-#pragma unroll
-                for (int g = 0; g < C::GP; ++g) {
-                    if (g < G) {
-                        float2 acc = make_float2(0.f, 0.f);
-#pragma unroll
-                        for (int c = 0; c < C::CPL / 2; ++c) {
-                            acc = ffma2(mnf[c], qn[g < G ? g : 0][c], acc);
-                            acc = ffma2(mxf[c], qp[g < G ? g : 0][c], acc);
-                        }
-                        v[ip * C::GP + g] = acc.x + acc.y;
-                    } else {
-                        v[ip * C::GP + g] = 0.f;
-                    }
-                }
-            }
-            transpose_reduce<C::NV, C::LPP>(v, lane);
-            // lane lg now holds NF sums of page ip = lg / LPG; fold the group's heads by max
-            const int i0 = (C::NV >= C::LPP) ? lg * C::NF : lg / (C::LPP / C::NV);
-            float s = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < C::NF; ++j) {
-                const int g = (i0 + j) % C::GP;
-                if (g < G) s = fmaxf(s, v[j]);
-            }
-#pragma unroll
-            for (int m = 1; m < C::LPG; m <<= 1) s = fmaxf(s, __shfl_xor_sync(kFull, s, m));
-            const int ip = lg / C::LPG;
-            const int j = (rb * C::RB + ip) * C::PPP + pp;
-            const int pid_j = __shfl_sync(kFull, pid_cur, j);
-            if ((lg % C::LPG) == 0 && cur.b0 + j < cur.n_r)
-                dst[j] = (pid_j >= 0) ? s * scale : -INFINITY;
+        for (int s = 0; s < C::KSTEPS; ++s) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(a_base + s * 32, a0, a1, a2, a3);
+            mma_bf16_16816(acc, a0, a1, a2, a3, bfrag[s][0], bfrag[s][1]);
+        }
+        // acc[0],acc[1]: page gid, heads 2*tid4, 2*tid4+1;  acc[2],acc[3]: page gid+8, same heads
+        const float ninf = -INFINITY;
+        float s_lo = fmaxf(2 * tid4 < G ? acc[0] : ninf, 2 * tid4 + 1 < G ? acc[1] : ninf);
+        float s_hi = fmaxf(2 * tid4 < G ? acc[2] : ninf, 2 * tid4 + 1 < G ? acc[3] : ninf);
+        s_lo = fmaxf(s_lo, __shfl_xor_sync(kFull, s_lo, 1));
+        s_hi = fmaxf(s_hi, __shfl_xor_sync(kFull, s_hi, 1));
+        s_lo = fmaxf(s_lo, __shfl_xor_sync(kFull, s_lo, 2));
+        s_hi = fmaxf(s_hi, __shfl_xor_sync(kFull, s_hi, 2));
+        const int pid_lo = __shfl_sync(kFull, pid_cur, gid);
+        const int pid_hi = __shfl_sync(kFull, pid_cur, gid + 8);
+        if (tid4 == 0) {
+            float *dst = scores + ((size_t)cur.r * H_kv + cur.h) * max_pages + cur.b0;
+            if (cur.b0 + gid < cur.n_r) dst[gid] = (pid_lo >= 0) ? s_lo * scale : ninf;
+            if (cur.b0 + gid + 8 < cur.n_r) dst[gid + 8] = (pid_hi >= 0) ? s_hi * scale : ninf;
         }
         __syncwarp();        // every lane is done reading the buffer before it is refilled
         cur = nxt;
@@ -294,14 +257,44 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
 // top-k: one CTA per (request, kv-head)
 // ---------------------------------------------------------------------------------
 constexpr int kTopkThreads = 256;
+constexpr int kTopkWarps = kTopkThreads / 32;
 
+// Exclusive prefix sum over the CTA of one int per thread, in thread order.
+__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot, int &total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    int before = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kTopkWarps; ++w) {
+        const int c = warp_tot[w];
+        if (w < warp) before += c;
+        tot += c;
+    }
+    __syncthreads();
+    total = tot;
+    return before + inc - v;
+}
+
+// KPT = keys per thread held in registers (n <= KPT*256); KPT == 0 streams the keys from
+// global memory on every pass instead (any n).
+template <int KPT>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_lens, int H_kv,
             int max_pages, int k_pages, int k_max, int32_t *__restrict__ sel_idx,
             int32_t *__restrict__ sel_cnt) {
+    constexpr bool kCached = KPT > 0;
+    constexpr int NK = kCached ? KPT : 1;
     __shared__ int hist[256];
     __shared__ int s_present, s_digit, s_above, s_inbin;
-    __shared__ int warp_eq[kTopkThreads / 32], warp_sel[kTopkThreads / 32];
+    __shared__ int warp_tot[kTopkWarps];
+    __shared__ int cnt_tile[kCached ? KPT * kTopkWarps : 1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair = blockIdx.x;
     const int r = pair / H_kv;
@@ -310,6 +303,22 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     if (n > max_pages) n = max_pages;
     const float *row = scores + (size_t)pair * max_pages;
     int32_t *out = sel_idx + (size_t)pair * k_max;
+
+    // element j of thread t is page j*256 + t (tile-major, so index order = (j, t) order)
+    uint32_t keys[NK];
+    if constexpr (kCached) {
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const int i = j * kTopkThreads + tid;
+            keys[j] = (i < n) ? f32_key(__ldg(row + i)) : 0u;
+        }
+    }
+    const int tiles = (n + kTopkThreads - 1) / kTopkThreads;
+    auto key_at = [&](int j) -> uint32_t {
+        if constexpr (kCached) return keys[j];
+        const int i = j * kTopkThreads + tid;
+        return (i < n) ? f32_key(row[i]) : 0u;
+    };
 
     uint32_t prefix = 0;          // digits fixed so far (higher bits), lower bits zero
     int remaining = 0;            // how many still to take among keys matching the prefix
@@ -321,14 +330,22 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
         hist[tid] = 0;
         __syncthreads();
         int present = 0;
-        for (int i = tid; i < n; i += kTopkThreads) {
-            const uint32_t key = f32_key(row[i]);
+        auto visit = [&](int j) {
+            const int i = j * kTopkThreads + tid;
+            if (i >= n) return;
+            const uint32_t key = key_at(j);
             if (shift == 24) {
                 present += (key != kKeyAbsent);
                 atomicAdd(&hist[key >> 24], 1);
             } else if ((key >> (shift + 8)) == (prefix >> (shift + 8))) {
                 atomicAdd(&hist[(key >> shift) & 255u], 1);
             }
+        };
+        if constexpr (kCached) {
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) visit(j);
+        } else {
+            for (int j = 0; j < tiles; ++j) visit(j);
         }
         if (shift == 24 && present) atomicAdd(&s_present, present);
         __syncthreads();
@@ -382,55 +399,107 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     const uint32_t T = prefix;
     const int need = ge_mode ? 0x7fffffff : remaining;
 
-    int run_eq = 0, run_sel = 0;
-    for (int base = 0; base < n; base += kTopkThreads) {
-        const int i = base + tid;
-        uint32_t key = 0;
-        bool gt = false, eq = false;
-        if (i < n) {
-            key = f32_key(row[i]);
-            gt = ge_mode ? (key >= T) : (key > T);
-            eq = !ge_mode && (key == T);
-        }
-        const unsigned beq = __ballot_sync(kFull, eq);
-        if (lane == 0) warp_eq[warp] = __popc(beq);
-        __syncthreads();
-        int eq_before = run_eq, eq_total = 0;
+    if constexpr (kCached) {
+        // ---- registers: rank the ties, then the selected, with two CTA-wide scans over (tile, warp)
+        uint32_t eqmask = 0, takemask = 0;
 #pragma unroll
-        for (int w = 0; w < kTopkThreads / 32; ++w) {
-            const int c = warp_eq[w];
-            if (w < warp) eq_before += c;
-            eq_total += c;
+        for (int j = 0; j < KPT; ++j) {
+            const int i = j * kTopkThreads + tid;
+            const bool valid = i < n;
+            const bool gt = valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T));
+            const bool eq = valid && !ge_mode && (keys[j] == T);
+            eqmask |= (uint32_t)eq << j;
+            takemask |= (uint32_t)gt << j;
         }
-        eq_before += __popc(beq & ((1u << lane) - 1u));
-        const bool take = gt || (eq && eq_before < need);
-        const unsigned bsel = __ballot_sync(kFull, take);
-        if (lane == 0) warp_sel[warp] = __popc(bsel);
-        __syncthreads();
-        int pos = run_sel, sel_total = 0;
+        int total;
+        if (!ge_mode) {
 #pragma unroll
-        for (int w = 0; w < kTopkThreads / 32; ++w) {
-            const int c = warp_sel[w];
-            if (w < warp) pos += c;
-            sel_total += c;
+            for (int j = 0; j < KPT; ++j) {
+                const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
+                if (lane == 0) cnt_tile[j * kTopkWarps + warp] = __popc(b);
+            }
+            __syncthreads();
+            const int mine = tid < KPT * kTopkWarps ? cnt_tile[tid] : 0;
+            const int off = block_exclusive_scan(mine, warp_tot, total);
+            if (tid < KPT * kTopkWarps) cnt_tile[tid] = off;
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) {
+                const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
+                const int rank = cnt_tile[j * kTopkWarps + warp] + __popc(b & ((1u << lane) - 1u));
+                if (((eqmask >> j) & 1u) && rank < need) takemask |= 1u << j;
+            }
+            __syncthreads();
         }
-        pos += __popc(bsel & ((1u << lane) - 1u));
-        if (take && pos < k_max) out[pos] = i;
-        run_eq += eq_total;
-        run_sel += sel_total;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
+            if (lane == 0) cnt_tile[j * kTopkWarps + warp] = __popc(b);
+        }
         __syncthreads();
+        const int mine = tid < KPT * kTopkWarps ? cnt_tile[tid] : 0;
+        const int off = block_exclusive_scan(mine, warp_tot, total);
+        if (tid < KPT * kTopkWarps) cnt_tile[tid] = off;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
+            const int pos = cnt_tile[j * kTopkWarps + warp] + __popc(b & ((1u << lane) - 1u));
+            if (((takemask >> j) & 1u) && pos < k_max) out[pos] = j * kTopkThreads + tid;
+        }
+    } else {
+        // ---- streaming: tile by tile, carrying the running counts
+        int run_eq = 0, run_sel = 0;
+        __shared__ int warp_eq[kTopkWarps], warp_sel[kTopkWarps];
+        for (int base = 0; base < n; base += kTopkThreads) {
+            const int i = base + tid;
+            uint32_t key = 0;
+            bool gt = false, eq = false;
+            if (i < n) {
+                key = f32_key(row[i]);
+                gt = ge_mode ? (key >= T) : (key > T);
+                eq = !ge_mode && (key == T);
+            }
+            const unsigned beq = __ballot_sync(kFull, eq);
+            if (lane == 0) warp_eq[warp] = __popc(beq);
+            __syncthreads();
+            int eq_before = run_eq, eq_total = 0;
+#pragma unroll
+            for (int w = 0; w < kTopkWarps; ++w) {
+                const int c = warp_eq[w];
+                if (w < warp) eq_before += c;
+                eq_total += c;
+            }
+            eq_before += __popc(beq & ((1u << lane) - 1u));
+            const bool take = gt || (eq && eq_before < need);
+            const unsigned bsel = __ballot_sync(kFull, take);
+            if (lane == 0) warp_sel[warp] = __popc(bsel);
+            __syncthreads();
+            int pos = run_sel, sel_total = 0;
+#pragma unroll
+            for (int w = 0; w < kTopkWarps; ++w) {
+                const int c = warp_sel[w];
+                if (w < warp) pos += c;
+                sel_total += c;
+            }
+            pos += __popc(bsel & ((1u << lane) - 1u));
+            if (take && pos < k_max) out[pos] = i;
+            run_eq += eq_total;
+            run_sel += sel_total;
+            __syncthreads();
+        }
     }
     for (int i = k_eff + tid; i < k_max; i += kTopkThreads) out[i] = -1;
     if (tid == 0) sel_cnt[pair] = k_eff;
 }
 
-template <int D, int G>
+template <int D>
 cudaError_t launch_score(const se_params &p, const void *q, const void *meta, const int32_t *page_table,
                          const int32_t *seq_lens, float *scores, uint32_t *status, cudaStream_t stream) {
-    using C = ScoreCfg<D, G>;
-    const size_t smem = (size_t)kScoreWarps * 2 * kPB * C::PHB + kScoreWarps * 2 * 8 +
+    using C = ScoreCfg<D>;
+    const size_t smem = (size_t)kScoreWarps * 2 * C::BUF + kScoreWarps * 2 * 8 +
                         (size_t)(2 * p.B + 1) * sizeof(int);
-    auto kern = score_kernel<D, G>;
+    auto kern = score_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const long long units_ub = (long long)p.B * p.H_kv * ((p.max_pages + kUnitPages - 1) / kUnitPages);
@@ -443,24 +512,8 @@ cudaError_t launch_score(const se_params &p, const void *q, const void *meta, co
     if (grid < 1) grid = 1;
     kern<<<(unsigned)grid, kScoreWarps * 32, smem, stream>>>(
         (const uint16_t *)q, (const uint8_t *)meta, page_table, seq_lens, scores, p.B, p.H_kv,
-        p.max_pages, p.num_phys_pages, effective_scale(p), status);
+        p.H_q / p.H_kv, p.max_pages, p.num_phys_pages, effective_scale(p), status);
     return cudaGetLastError();
-}
-
-template <int D>
-cudaError_t dispatch_score(const se_params &p, const void *q, const void *meta, const int32_t *page_table,
-                           const int32_t *seq_lens, float *scores, uint32_t *status, cudaStream_t stream) {
-    switch (p.H_q / p.H_kv) {
-        case 1: return launch_score<D, 1>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 2: return launch_score<D, 2>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 3: return launch_score<D, 3>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 4: return launch_score<D, 4>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 5: return launch_score<D, 5>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 6: return launch_score<D, 6>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 7: return launch_score<D, 7>(p, q, meta, page_table, seq_lens, scores, status, stream);
-        case 8: return launch_score<D, 8>(p, q, meta, page_table, seq_lens, scores, status, stream);
-    }
-    return cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -473,11 +526,18 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     float *scores = reinterpret_cast<float *>(ws + L.scores);
     uint32_t *status = reinterpret_cast<uint32_t *>(ws + L.status);
     cudaError_t e = (p.D == 128)
-                        ? dispatch_score<128>(p, q, meta, page_table, seq_lens, scores, status, stream)
-                        : dispatch_score<64>(p, q, meta, page_table, seq_lens, scores, status, stream);
+                        ? launch_score<128>(p, q, meta, page_table, seq_lens, scores, status, stream)
+                        : launch_score<64>(p, q, meta, page_table, seq_lens, scores, status, stream);
     if (e != cudaSuccess) return e;
-    topk_kernel<<<p.B * p.H_kv, kTopkThreads, 0, stream>>>(scores, seq_lens, p.H_kv, p.max_pages,
-                                                         k_pages, p.k_max, sel_idx, sel_cnt);
+    const int pairs = p.B * p.H_kv;
+#define SE_TOPK(KPT)                                                                                   \
+    topk_kernel<KPT><<<pairs, kTopkThreads, 0, stream>>>(scores, seq_lens, p.H_kv, p.max_pages, k_pages, \
+                                                         p.k_max, sel_idx, sel_cnt)
+    if (p.max_pages <= 4 * kTopkThreads) SE_TOPK(4);
+    else if (p.max_pages <= 16 * kTopkThreads) SE_TOPK(16);
+    else if (p.max_pages <= 32 * kTopkThreads) SE_TOPK(32);
+    else SE_TOPK(0);
+#undef SE_TOPK
     return cudaGetLastError();
 }
 
