@@ -74,7 +74,8 @@ typedef struct se_params {
     int32_t H_kv;            /* kv heads; H_q % H_kv == 0, H_q / H_kv in 1..8               */
     int32_t D;               /* head dimension, 64 or 128                                   */
     int32_t page_size;       /* must be 16                                                  */
-    int32_t max_pages;       /* row stride of page_table, >= ceil(max seq_len / 16)         */
+    int32_t max_pages;       /* row stride of page_table, >= ceil(max seq_len / 16), <= 8192
+                                (contexts up to 131072 tokens)                              */
     int32_t num_phys_pages;  /* P_phys, pages in k_cache / v_cache / meta / score_accum     */
     int32_t k_max;           /* row stride of sel_idx, >= floor(budget / 16), 1..4096       */
     float   sm_scale;        /* logit scale; 0 selects 1/sqrt(D)                            */

@@ -20,7 +20,7 @@ int validate(const se_params *p) {
     if (p->H_q % p->H_kv != 0) return SE_ERR_INVALID_ARG;
     const int G = p->H_q / p->H_kv;
     if (G < 1 || G > 8) return SE_ERR_UNSUPPORTED_SHAPE;
-    if (p->max_pages < 1 || p->num_phys_pages < 1) return SE_ERR_INVALID_ARG;
+    if (p->max_pages < 1 || p->max_pages > 8192 || p->num_phys_pages < 1) return SE_ERR_INVALID_ARG;
     if (p->k_max < 1 || p->k_max > 4096) return SE_ERR_INVALID_ARG;
     if (p->flags != 0) return SE_ERR_INVALID_ARG;
     if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return SE_ERR_INVALID_ARG;
@@ -28,6 +28,8 @@ int validate(const se_params *p) {
     if ((long long)p->B * p->H_kv > (1ll << 24)) return SE_ERR_INVALID_ARG;
     if ((long long)p->B * p->max_pages > (1ll << 31) - 1) return SE_ERR_INVALID_ARG;
     if ((long long)p->num_phys_pages * p->H_kv * kPage > (1ll << 31) - 1) return SE_ERR_INVALID_ARG;
+    if ((long long)p->B * p->H_kv * p->k_max > (1ll << 30)) return SE_ERR_INVALID_ARG;
+    if (p->H_kv > 127) return SE_ERR_INVALID_ARG;
     return SE_OK;
 }
 
@@ -43,20 +45,23 @@ float effective_scale(const se_params &p) {
 
 int decode_warps_per_cta();
 
+// Split-K geometry: every (request, kv-head) pair is cut into the same number of splits, as many
+// as the persistent warps of the grid can take in one round (one unit per warp), so that no warp
+// carries two pairs and every warp has the same number of pages.
 DecodePlan make_decode_plan(const se_params &p) {
     DecodePlan plan;
     const int warps_per_cta = decode_warps_per_cta();
-    const long long X = (long long)p.B * p.H_kv * p.k_max;
-    const int ctas_per_sm = (p.D == 128) ? 1 : 1;
-    long long warps = (long long)kAssumedSMs * ctas_per_sm * warps_per_cta;
-    long long ppw = (X + warps - 1) / warps;
-    if (ppw < 1) ppw = 1;
-    long long used_warps = (X + ppw - 1) / ppw;
-    long long grid = (used_warps + warps_per_cta - 1) / warps_per_cta;
+    const long long pairs = (long long)p.B * p.H_kv;
+    const long long warps = (long long)kAssumedSMs * warps_per_cta;
+    long long splits = warps / pairs;
+    if (splits < 1) splits = 1;
+    if (splits > p.k_max) splits = p.k_max;
+    const int pps = (int)((p.k_max + splits - 1) / splits);
+    plan.pages_per_split = pps;
+    plan.max_splits = (p.k_max + pps - 1) / pps;
+    const long long units = pairs * plan.max_splits;
+    long long grid = units < kAssumedSMs ? units : kAssumedSMs;
     plan.grid = (int)grid;
-    plan.warps_total = (int)(grid * warps_per_cta);
-    plan.pages_per_warp = (int)ppw;
-    plan.max_splits = (int)((p.k_max + ppw - 1) / ppw) + 1;
     return plan;
 }
 

@@ -24,12 +24,27 @@
 
 #include "se_internal.h"
 
+// Optional per-warp phase timing for development builds (-DSE_DECODE_PROFILE); compiled out of
+// the library otherwise.
+#ifdef SE_DECODE_PROFILE
+__device__ long long g_dec_prof[8 * 4096];
+#define SE_PROF_DECL long long prof_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long prof_t_ = clock64(); const long long prof_t0_ = prof_t_;
+#define SE_PROF_LAP(i) { const long long t_ = clock64(); prof_[i] += t_ - prof_t_; prof_t_ = t_; }
+#define SE_PROF_ADD(i, v) { prof_[i] += (v); }
+#define SE_PROF_STORE(w) { if ((threadIdx.x & 31) == 0 && (w) < 4096) { prof_[7] = clock64() - prof_t0_; for (int i_ = 0; i_ < 8; ++i_) g_dec_prof[(w) * 8 + i_] = prof_[i_]; } }
+#else
+#define SE_PROF_DECL
+#define SE_PROF_LAP(i)
+#define SE_PROF_ADD(i, v)
+#define SE_PROF_STORE(w)
+#endif
+
 namespace se {
 
 namespace {
 
 constexpr int kDecWarps = 8;
-constexpr int kWin = 32;                 // selected pages looked up at once
+constexpr int kChunk = 128;              // selected-page slots looked up at once
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileBytes = kPage * 128;  // one TMA box: 16 rows x 64 bf16
@@ -67,7 +82,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
               const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ sel_idx,
               const int32_t *__restrict__ sel_cnt, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ partials, uint32_t *__restrict__ tickets, float *__restrict__ zbuf,
-              int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_warp,
+              int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
               int max_splits, float scale_log2, uint32_t *status) {
     using C = DecCfg<D>;
     extern __shared__ uint8_t smem_dyn[];
@@ -88,10 +103,13 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     const int H_q = H_kv * G;
     const int gid = lane >> 2, tid4 = lane & 3;          // fragment coordinates: head row / column pair
     const bool head_ok = gid < G;
-    const long long X = (long long)B * H_kv * k_max;     // flat slots
-    const long long gw = (long long)blockIdx.x * kDecWarps + warp;
-    long long x = gw * pages_per_warp;
-    const long long x_end = min(X, x + (long long)pages_per_warp);
+    // Work unit = (pair, split): slots [pair*k_max + split*pages_per_split, +pages_per_split) of the
+    // flat slot space slot = pair*k_max + i (the host guarantees it fits 31 bits).  Units are dealt
+    // to warps so that warp w of every CTA is busy before warp w+1 of any CTA.
+    const int n_units = B * H_kv * max_splits;
+    const int gw = warp * gridDim.x + blockIdx.x;
+    const int warps_total = kDecWarps * gridDim.x;
+    int x_end = 0;                                   // end of the current unit's slot range
 
     // ldmatrix lane offsets inside a 16x128-byte swizzled tile.
     // K (B operand, not transposed): matrices {tok 0-7 | 8-15} x {chunk c | c+1}
@@ -101,16 +119,102 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     const int v_row = (lane & 7) + 8 * ((lane >> 3) & 1);
     const int v_chunk_add = lane >> 4;
 
+    SE_PROF_DECL
     uint32_t phases = 0;          // parity bit per stage
     int stage_c = 0, stage_i = 0; // next stage to consume / to fill
     bool failed = false;
 
-    while (x < x_end && !failed) {
-        // ---- the part of one pair that lies in this warp's slice
-        const int pair = (int)(x / k_max);
-        const int i_lo = (int)(x - (long long)pair * k_max);
-        const int i_hi_slot = (int)min((long long)k_max, x_end - (long long)pair * k_max);
-        x = (long long)pair * k_max + i_hi_slot;                      // next pair starts here
+    // ---- page list.  The valid selected pages of a chunk of up to kChunk slots are looked up
+    // at once (selection -> page table, two dependent loads for the whole chunk) and kept in
+    // shared memory; the copy pipeline then runs over that list without any further global
+    // look-ups, across pair boundaries.
+    //   ent_y    row of the page's first token in the [pages*heads*16, D] view of the cache
+    //   ent_info valid tokens (bits 0-4) | selection index i (bits 5-16) | slot - chunk_base (bits 17-23)
+    int *ent_y = reinterpret_cast<int *>(smem_al + (size_t)kDecWarps * C::WARP_SMEM + kDecWarps * C::NSTAGE * 8) +
+                 warp * 2 * kChunk;
+    int *ent_info = ent_y + kChunk;
+    int chunk_base = 0, chunk_end = 0;           // slots [chunk_base, chunk_end) are in the list
+    int n_ent = 0, ce = 0, pe = 0;               // entries, next to consume, next to issue
+
+    auto fill_chunk = [&](int base) {
+        chunk_base = base;
+        chunk_end = min(x_end, base + kChunk);
+        const int pair0 = base / k_max;
+        const int i0 = base - pair0 * k_max;
+        int sl_pid[kChunk / 32], sl_meta[kChunk / 32];
+#pragma unroll
+        for (int rep = 0; rep < kChunk / 32; ++rep) {
+            const int off = rep * 32 + lane;
+            int pid = -1, meta = 0;
+            if (base + off < chunk_end) {
+                const int dp = (i0 + off) / k_max;
+                const int pair = pair0 + dp;
+                const int i = i0 + off - dp * k_max;
+                const int r = pair / H_kv;
+                const int hh = pair - r * H_kv;
+                const int b = __ldg(sel_idx + base + off);      // speculative: checked against cnt below
+                const int cnt = min(__ldg(sel_cnt + pair), k_max);
+                const int len = __ldg(seq_lens + r);
+                const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
+                if (i < cnt && n_r > 0) {
+                    if (b < 0 || b >= n_r) {
+                        atomicOr(status, SE_DEV_BAD_SELECTION);
+                    } else {
+                        pid = __ldg(page_table + (size_t)r * max_pages + b);
+                        meta = min(kPage, len - b * kPage) | (i << 5) | (off << 17) | (hh << 24);
+                    }
+                }
+            }
+            sl_pid[rep] = pid;
+            sl_meta[rep] = meta;
+        }
+        int count = 0;
+#pragma unroll
+        for (int rep = 0; rep < kChunk / 32; ++rep) {
+            int pid = sl_pid[rep];
+            const bool looked_up = sl_meta[rep] != 0;
+            if (looked_up && pid >= P_phys) {
+                atomicOr(status, SE_DEV_BAD_PAGE_ID);
+                pid = -1;
+            } else if (looked_up && pid < 0) {
+                atomicOr(status, SE_DEV_BAD_SELECTION);
+            }
+            const unsigned vm = __ballot_sync(kFull, pid >= 0);
+            if (pid >= 0) {
+                const int pos = count + __popc(vm & ((1u << lane) - 1u));
+                ent_y[pos] = (pid * H_kv + (sl_meta[rep] >> 24)) * kPage;
+                ent_info[pos] = sl_meta[rep] & 0x00ffffff;
+            }
+            count += __popc(vm);
+        }
+        __syncwarp();
+        n_ent = count;
+        ce = 0;
+        pe = 0;
+    };
+    // called between pages, when no stage is being read: fill every free stage.  Lane 0 arms the
+    // barrier; one lane per 16x64 tile issues its tensor copy.
+    auto top_up = [&]() {
+        while (pe < n_ent && pe < ce + C::NSTAGE) {
+            const uint32_t bar = bar0 + stage_i * 8;
+            if (lane == 0) mbar_expect_tx(bar, C::STAGEB);
+            __syncwarp();
+            if (lane < 2 * C::HALVES) {
+                const int y = ent_y[pe];
+                const int hf = lane >> 1;
+                const uint32_t dst = ring0 + stage_i * C::STAGEB + (lane & 1) * C::PAGEB + hf * kTileBytes;
+                tma_load_2d(dst, (lane & 1) ? &v_map : &k_map, hf * 64, y, bar);
+            }
+            stage_i = (stage_i + 1 == C::NSTAGE) ? 0 : stage_i + 1;
+            ++pe;
+        }
+    };
+
+    for (int unit = gw; unit < n_units && !failed; unit += warps_total) {
+        const int pair = unit / max_splits;
+        const int my_split = unit - pair * max_splits;
+        const int i_lo = my_split * pages_per_split;
+        if (i_lo >= k_max) continue;
         const int r = pair / H_kv, h = pair % H_kv;
         int cnt = sel_cnt[pair];
         if (cnt > k_max) {
@@ -120,7 +224,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         const int len = seq_lens[r];
         const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
         if (cnt <= 0 || n_r == 0) {
-            if (i_lo == 0) {          // the warp holding the pair's first slot reports "nothing attended"
+            if (my_split == 0) {      // the first split of the pair reports "nothing attended"
                 for (int g = 0; g < G; ++g) {
                     float *o = out + ((size_t)r * H_q + h * G + g) * D;
                     for (int c = lane; c < D; c += 32) o[c] = 0.f;
@@ -130,11 +234,16 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             continue;
         }
         if (i_lo >= cnt) continue;
-        const int i_hi = min(i_hi_slot, cnt);
-        const int w_first = (int)(((long long)pair * k_max) / pages_per_warp);
-        const int w_last = (int)(((long long)pair * k_max + cnt - 1) / pages_per_warp);
-        const int n_split = w_last - w_first + 1;
-        const int my_split = (int)(gw - w_first);
+        const int i_hi = min(min(i_lo + pages_per_split, k_max), cnt);
+        const int seg_begin = pair * k_max + i_lo;
+        const int seg_end = pair * k_max + i_hi;                      // first slot past this unit
+        const int n_split = (cnt + pages_per_split - 1) / pages_per_split;   // splits of this pair that hold pages
+        x_end = seg_end;
+
+        // make sure the page list covers the start of the segment, and get copies going before
+        // the (dependent) q loads below are waited for
+        fill_chunk(seg_begin);
+        top_up();
 
         // ---- Q as the A operand: row gid = query head gid of the group (rows >= G and 8..15 are zero)
         uint32_t qa[C::KSTEPS][2];
@@ -154,128 +263,99 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             o_acc[nt][0] = 0.f; o_acc[nt][1] = 0.f; o_acc[nt][2] = 0.f; o_acc[nt][3] = 0.f;
         }
         float m_run = -INFINITY, l_run = 0.f;       // of head gid; l is this lane's share (its 4 token columns)
+        SE_PROF_LAP(0)
 
-        for (int win = i_lo; win < i_hi && !failed; win += kWin) {
-            // ---- look up up to 32 selected pages
-            const int i_me = win + lane;
-            int pid = -1, nv = 0;
-            if (i_me < i_hi) {
-                const int b = sel_idx[(size_t)pair * k_max + i_me];
-                if (b < 0 || b >= n_r) {
-                    atomicOr(status, SE_DEV_BAD_SELECTION);
-                } else {
-                    pid = page_table[(size_t)r * max_pages + b];
-                    if (pid >= P_phys) {
-                        atomicOr(status, SE_DEV_BAD_PAGE_ID);
-                        pid = -1;
-                    } else if (pid < 0) {
-                        atomicOr(status, SE_DEV_BAD_SELECTION);
-                    }
-                    nv = min(kPage, len - b * kPage);
-                }
+        while (!failed) {
+            if (ce == n_ent) {                       // list exhausted: more slots of this segment left?
+                if (chunk_end >= seg_end) break;
+                fill_chunk(chunk_end);
+                top_up();
+                continue;
             }
-            const unsigned vmask = __ballot_sync(kFull, pid >= 0);
-            const int nvalid = __popc(vmask);
-
-            auto issue = [&](int j) {
-                const int src_lane = __fns(vmask, 0, j + 1);
-                const int pj = __shfl_sync(kFull, pid, src_lane);
-                if (lane == 0) {
-                    const uint32_t bar = bar0 + stage_i * 8;
-                    const uint32_t dst = ring0 + stage_i * C::STAGEB;
-                    mbar_expect_tx(bar, C::STAGEB);
-                    const int y = (pj * H_kv + h) * kPage;
-#pragma unroll
-                    for (int hf = 0; hf < C::HALVES; ++hf) {
-                        tma_load_2d(dst + hf * kTileBytes, &k_map, hf * 64, y, bar);
-                        tma_load_2d(dst + C::PAGEB + hf * kTileBytes, &v_map, hf * 64, y, bar);
-                    }
-                }
-                stage_i = (stage_i + 1 == C::NSTAGE) ? 0 : stage_i + 1;
-            };
-
-            const int pre = min(C::NSTAGE - 1, nvalid);
-            for (int j = 0; j < pre; ++j) issue(j);
-
-            for (int j = 0; j < nvalid; ++j) {
-                if (j + C::NSTAGE - 1 < nvalid) issue(j + C::NSTAGE - 1);
-                const int src_lane = __fns(vmask, 0, j + 1);
-                const int nv_j = __shfl_sync(kFull, nv, src_lane);
-                const int i_j = win + src_lane;
-                if (!mbar_wait(bar0 + stage_c * 8, (phases >> stage_c) & 1u)) {
-                    failed = true;
-                    break;
-                }
-                phases ^= (1u << stage_c);
-                const uint32_t Ks = ring0 + stage_c * C::STAGEB;
-                const uint32_t Vs = Ks + C::PAGEB;
-                stage_c = (stage_c + 1 == C::NSTAGE) ? 0 : stage_c + 1;
-
-                // ---- S^T[head, token] = Q . K^T : two n8 tiles (tokens 0-7, 8-15)
-                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int s = 0; s < C::KSTEPS; ++s) {
-                    const int hf = s >> 2;
-                    const int chunk = 2 * (s & 3) + k_chunk_add;
-                    uint32_t b00, b01, b10, b11;     // {tok 0-7: k lo, k hi}, {tok 8-15: k lo, k hi}
-                    ldmatrix_x4(Ks + hf * kTileBytes + k_row * 128 + ((chunk ^ (k_row & 7)) << 4), b00, b01, b10, b11);
-                    mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
-                    mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
-                }
-                // this lane: head gid, tokens 2*tid4, 2*tid4+1 (s0) and 8+2*tid4, 9+2*tid4 (s1)
-                const int t0 = 2 * tid4;
-                float z[4];
-                z[0] = (t0 < nv_j) ? s0[0] * scale_log2 : -INFINITY;
-                z[1] = (t0 + 1 < nv_j) ? s0[1] * scale_log2 : -INFINITY;
-                z[2] = (t0 + 8 < nv_j) ? s1[0] * scale_log2 : -INFINITY;
-                z[3] = (t0 + 9 < nv_j) ? s1[1] * scale_log2 : -INFINITY;
-                if (zbuf != nullptr && head_ok) {
-                    float *zp = zbuf + (((size_t)pair * k_max + i_j) * kPage) * GP + gid;
-                    zp[(t0) * GP] = z[0];
-                    zp[(t0 + 1) * GP] = z[1];
-                    zp[(t0 + 8) * GP] = z[2];
-                    zp[(t0 + 9) * GP] = z[3];
-                }
-                float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
-                pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
-                pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
-                const float m_new = fmaxf(m_run, pmax);           // finite: token 0 of a page is always valid
-                const float corr = exp2f(m_run - m_new);          // 0 on the first page (m_run = -inf)
-                if (__any_sync(kFull, m_new != m_run)) {
-                    l_run *= corr;
-#pragma unroll
-                    for (int nt = 0; nt < C::NTILES; ++nt) {
-                        o_acc[nt][0] *= corr;
-                        o_acc[nt][1] *= corr;
-                    }
-                    m_run = m_new;
-                }
-                float p[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) p[e] = exp2f(z[e] - m_run);    // exp2(-inf) = 0 for masked tokens
-                l_run += (p[0] + p[1]) + (p[2] + p[3]);
-                // P as the A operand, split into two bf16 terms so that p_hi + p_lo carries 16 bits
-                const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
-                const float2 f0 = bf16x2_to_f2(ph0), f1 = bf16x2_to_f2(ph1);
-                const uint32_t pl0 = pack_bf16(p[0] - f0.x, p[1] - f0.y), pl1 = pack_bf16(p[2] - f1.x, p[3] - f1.y);
-
-                // ---- O[head, :] += P . V : n8 tiles over the channels, k16 = the 16 tokens
-#pragma unroll
-                for (int c2 = 0; c2 < C::NTILES / 2; ++c2) {
-                    const int hf = c2 >> 2;
-                    const int chunk = 2 * (c2 & 3) + v_chunk_add;
-                    uint32_t v00, v01, v10, v11;     // {chunk c: tok 0-7, tok 8-15}, {chunk c+1: ...}
-                    ldmatrix_x4_trans(Vs + hf * kTileBytes + v_row * 128 + ((chunk ^ (v_row & 7)) << 4), v00, v01, v10, v11);
-                    mma_bf16_16816(o_acc[2 * c2], ph0, 0u, ph1, 0u, v00, v01);
-                    mma_bf16_16816(o_acc[2 * c2], pl0, 0u, pl1, 0u, v00, v01);
-                    mma_bf16_16816(o_acc[2 * c2 + 1], ph0, 0u, ph1, 0u, v10, v11);
-                    mma_bf16_16816(o_acc[2 * c2 + 1], pl0, 0u, pl1, 0u, v10, v11);
-                }
-                __syncwarp();     // all lanes are done with this stage before it is refilled
+            const int info = ent_info[ce];
+            if (chunk_base + (info >> 17) >= seg_end) break;    // next entry belongs to the next pair
+            const int nv_j = info & 31;
+            const int i_j = (info >> 5) & 4095;
+            if (!mbar_wait(bar0 + stage_c * 8, (phases >> stage_c) & 1u)) {
+                failed = true;
+                break;
             }
+            phases ^= (1u << stage_c);
+            SE_PROF_LAP(1)
+            SE_PROF_ADD(5, 1)
+            const uint32_t Ks = ring0 + stage_c * C::STAGEB;
+            const uint32_t Vs = Ks + C::PAGEB;
+            stage_c = (stage_c + 1 == C::NSTAGE) ? 0 : stage_c + 1;
+
+            // ---- S^T[head, token] = Q . K^T : two n8 tiles (tokens 0-7, 8-15)
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int s = 0; s < C::KSTEPS; ++s) {
+                const int hf = s >> 2;
+                const int chunk = 2 * (s & 3) + k_chunk_add;
+                uint32_t b00, b01, b10, b11;     // {tok 0-7: k lo, k hi}, {tok 8-15: k lo, k hi}
+                ldmatrix_x4(Ks + hf * kTileBytes + k_row * 128 + ((chunk ^ (k_row & 7)) << 4), b00, b01, b10, b11);
+                mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+            }
+            // this lane: head gid, tokens 2*tid4, 2*tid4+1 (s0) and 8+2*tid4, 9+2*tid4 (s1)
+            const int t0 = 2 * tid4;
+            float z[4];
+            z[0] = (t0 < nv_j) ? s0[0] * scale_log2 : -INFINITY;
+            z[1] = (t0 + 1 < nv_j) ? s0[1] * scale_log2 : -INFINITY;
+            z[2] = (t0 + 8 < nv_j) ? s1[0] * scale_log2 : -INFINITY;
+            z[3] = (t0 + 9 < nv_j) ? s1[1] * scale_log2 : -INFINITY;
+            if (zbuf != nullptr && head_ok) {
+                float *zp = zbuf + (((size_t)pair * k_max + i_j) * kPage) * GP + gid;
+                zp[(t0) * GP] = z[0];
+                zp[(t0 + 1) * GP] = z[1];
+                zp[(t0 + 8) * GP] = z[2];
+                zp[(t0 + 9) * GP] = z[3];
+            }
+            float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+            pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
+            pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
+            const float m_new = fmaxf(m_run, pmax);           // finite: token 0 of a page is always valid
+            const float corr = exp2f(m_run - m_new);          // 0 on the first page (m_run = -inf)
+            if (__any_sync(kFull, m_new != m_run)) {
+                l_run *= corr;
+#pragma unroll
+                for (int nt = 0; nt < C::NTILES; ++nt) {
+                    o_acc[nt][0] *= corr;
+                    o_acc[nt][1] *= corr;
+                }
+                m_run = m_new;
+            }
+            float p[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) p[e] = exp2f(z[e] - m_run);    // exp2(-inf) = 0 for masked tokens
+            l_run += (p[0] + p[1]) + (p[2] + p[3]);
+            // P as the A operand, split into two bf16 terms so that p_hi + p_lo carries 16 bits
+            const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
+            const float2 f0 = bf16x2_to_f2(ph0), f1 = bf16x2_to_f2(ph1);
+            const uint32_t pl0 = pack_bf16(p[0] - f0.x, p[1] - f0.y), pl1 = pack_bf16(p[2] - f1.x, p[3] - f1.y);
+
+            // ---- O[head, :] += P . V : n8 tiles over the channels, k16 = the 16 tokens
+#pragma unroll
+            for (int c2 = 0; c2 < C::NTILES / 2; ++c2) {
+                const int hf = c2 >> 2;
+                const int chunk = 2 * (c2 & 3) + v_chunk_add;
+                uint32_t v00, v01, v10, v11;     // {chunk c: tok 0-7, tok 8-15}, {chunk c+1: ...}
+                ldmatrix_x4_trans(Vs + hf * kTileBytes + v_row * 128 + ((chunk ^ (v_row & 7)) << 4), v00, v01, v10, v11);
+                mma_bf16_16816(o_acc[2 * c2], ph0, 0u, ph1, 0u, v00, v01);
+                mma_bf16_16816(o_acc[2 * c2], pl0, 0u, pl1, 0u, v00, v01);
+                mma_bf16_16816(o_acc[2 * c2 + 1], ph0, 0u, ph1, 0u, v10, v11);
+                mma_bf16_16816(o_acc[2 * c2 + 1], pl0, 0u, pl1, 0u, v10, v11);
+            }
+            __syncwarp();     // all lanes are done with this stage before it is refilled
+            ++ce;
+            SE_PROF_LAP(2)
+            top_up();
+            SE_PROF_LAP(4)
         }
         if (failed) break;
 
+        SE_PROF_LAP(6)
         // ---- the four lanes of a head hold disjoint token columns: fold their l
         l_run += __shfl_xor_sync(kFull, l_run, 1);
         l_run += __shfl_xor_sync(kFull, l_run, 2);
@@ -312,31 +392,70 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         if ((int)old != n_split - 1) continue;
         __threadfence();
         if (lane == 0) tickets[pair] = 0u;                 // ready for the next launch
-        for (int g = 0; g < G; ++g) {
-            const float *pr = partials + (((size_t)r * H_q + h * G + g) * max_splits) * C::PSTRIDE;
-            float m_all = -INFINITY;
-            for (int s = 0; s < n_split; ++s) m_all = fmaxf(m_all, __ldcg(pr + (size_t)s * C::PSTRIDE + D));
-            float L = 0.f;
-            float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int s = 0; s < n_split; ++s) {
-                const float ms = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
-                const float ls = __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
-                const float w = (ms == -INFINITY) ? 0.f : exp2f(ms - m_all);
-                L += w * ls;
-                if (lane * 4 < D) {
-                    const float4 a = __ldcg(reinterpret_cast<const float4 *>(pr + (size_t)s * C::PSTRIDE) + lane);
-                    o4.x += w * a.x; o4.y += w * a.y; o4.z += w * a.z; o4.w += w * a.w;
+        // Merge: lane s first fetches (m_s, l_s) of split s for every head (all loads in flight
+        // together), the weights follow from warp reductions, then the accumulators are summed
+        // with each lane owning four channels.  More than 32 splits are folded block by block.
+        const float *pr0 = partials + (((size_t)r * H_q + h * G) * max_splits) * C::PSTRIDE;
+        float mg[8], lg[8], og[8][4];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            mg[g] = -INFINITY;
+            lg[g] = 0.f;
+            og[g][0] = og[g][1] = og[g][2] = og[g][3] = 0.f;
+        }
+        for (int s0 = 0; s0 < n_split; s0 += 32) {
+            const int ns = min(32, n_split - s0);
+            float ms[8], ls[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                ms[g] = -INFINITY;
+                ls[g] = 0.f;
+                if (g < G && lane < ns) {
+                    const float *pp = pr0 + ((size_t)g * max_splits + s0 + lane) * C::PSTRIDE + D;
+                    ms[g] = __ldcg(pp);
+                    ls[g] = __ldcg(pp + 1);
                 }
             }
-            const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                if (g >= G) continue;
+                float mb = ms[g];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(kFull, mb, o));
+                const float m_new = fmaxf(mg[g], mb);
+                const float wl = (ms[g] == -INFINITY) ? 0.f : exp2f(ms[g] - m_new);    // weight of split s0+lane
+                float lb = wl * ls[g];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) lb += __shfl_xor_sync(kFull, lb, o);
+                const float keep = (mg[g] == -INFINITY) ? 0.f : exp2f(mg[g] - m_new);
+                lg[g] = lg[g] * keep + lb;
+                og[g][0] *= keep; og[g][1] *= keep; og[g][2] *= keep; og[g][3] *= keep;
+                mg[g] = m_new;
+                const float *pa = pr0 + ((size_t)g * max_splits + s0) * C::PSTRIDE;
+#pragma unroll 4
+                for (int s = 0; s < ns; ++s) {
+                    const float ws = __shfl_sync(kFull, wl, s);
+                    if (lane * 4 < D) {
+                        const float4 a = __ldcg(reinterpret_cast<const float4 *>(pa + (size_t)s * C::PSTRIDE) + lane);
+                        og[g][0] += ws * a.x; og[g][1] += ws * a.y; og[g][2] += ws * a.z; og[g][3] += ws * a.w;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            if (g >= G) continue;
+            const float inv = lg[g] > 0.f ? 1.f / lg[g] : 0.f;
             if (lane * 4 < D) {
                 float4 *dst = reinterpret_cast<float4 *>(out + ((size_t)r * H_q + h * G + g) * D) + lane;
-                *dst = make_float4(o4.x * inv, o4.y * inv, o4.z * inv, o4.w * inv);
+                *dst = make_float4(og[g][0] * inv, og[g][1] * inv, og[g][2] * inv, og[g][3] * inv);
             }
             if (lane == 0)
-                lse[(size_t)r * H_q + h * G + g] = L > 0.f ? (m_all + log2f(L)) * kLn2 : -INFINITY;
+                lse[(size_t)r * H_q + h * G + g] = lg[g] > 0.f ? (mg[g] + log2f(lg[g])) * kLn2 : -INFINITY;
         }
     }
+    SE_PROF_LAP(3)
+    SE_PROF_STORE(gw)
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // bounded wait for whatever this warp still has in flight before the CTA can retire
@@ -418,7 +537,8 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     CUtensorMap k_map, v_map;
     if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
-    const size_t smem = (size_t)kDecWarps * C::WARP_SMEM + (size_t)kDecWarps * C::NSTAGE * 8 + 1024;
+    const size_t smem = (size_t)kDecWarps * C::WARP_SMEM + (size_t)kDecWarps * C::NSTAGE * 8 +
+                        (size_t)kDecWarps * 2 * kChunk * sizeof(int) + 1024;
     auto kern = decode_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -427,7 +547,7 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
         k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
         reinterpret_cast<float *>(ws + L.partials), reinterpret_cast<uint32_t *>(ws + L.dec_tickets), zbuf,
-        p.B, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_warp, plan.max_splits,
+        p.B, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
         effective_scale(p) * kLog2e, reinterpret_cast<uint32_t *>(ws + L.status));
     e = cudaGetLastError();
     if (e != cudaSuccess || !score_accum) return e;
@@ -444,6 +564,12 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
 }  // namespace
 
 int decode_warps_per_cta() { return kDecWarps; }
+
+#ifdef SE_DECODE_PROFILE
+extern "C" int se_debug_decode_profile(long long *host_out, int n_warps) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_dec_prof, sizeof(long long) * 8 * n_warps);
+}
+#endif
 
 cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *k_cache,
                                  const void *v_cache, const int32_t *page_table,

@@ -12,10 +12,9 @@ namespace se {
 // Decode-kernel geometry that both the workspace sizing and the launcher derive from
 // the problem shape alone (never from device data).
 struct DecodePlan {
-    int warps_total;        // persistent warps over the whole grid
     int grid;               // CTAs
-    int pages_per_warp;     // contiguous slice of the flattened (pair, selected page) space
-    int max_splits;         // most warps that can touch one (request, head) pair
+    int pages_per_split;    // selected pages one warp handles for one (request, head) pair
+    int max_splits;         // splits per pair = ceil(k_max / pages_per_split)
 };
 
 int  device_sm_count();

@@ -16,7 +16,7 @@
 //                issue-bound at 64 % of the copy bandwidth (57 warp instructions per page
 //                summary); this one needs 3.
 // topk_kernel    one CTA per (request, kv-head): most-significant-digit radix select over
-//                order-preserving integer keys held in registers, then an index-ordered
+//                order-preserving integer keys held in registers, then a page-ordered
 //                compaction, so equal scores go to the lower page and the list is ascending.
 #include "se_internal.h"
 
@@ -125,7 +125,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
     // (they meet the min row), rows k >= D carry q^+ (they meet the max row).
     uint32_t bfrag[C::KSTEPS][2];
     uint32_t qraw[D / 16][2];                // raw q pairs of the pair whose batch was issued last
-    int q_r = -1, q_h = -1;                  // pair the fragments belong to
 
     auto load_qraw = [&](const Batch &d) {
         const uint16_t *src = q + ((size_t)d.r * H_q + d.h * G + (gid < G ? gid : 0)) * D + 2 * tid4;
@@ -160,18 +159,19 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
         decode_unit(d.unit + tw, total_units, prefix, npages, B, H_kv, d);
     };
 
-    // issue the copies of one batch into buffer `slot`; returns this lane's physical page (or -1)
-    auto issue = [&](const Batch &d, int slot) -> int {
+    // page-table entries of a batch: lane j < 16 loads the entry of page b0 + j.  The value is not
+    // looked at here, so the load stays in flight while the warp carries on.
+    auto load_pids = [&](const Batch &d) -> int {
         int pid = -1;
-        if (lane < kPB) {
-            const int b = d.b0 + lane;
-            if (b < d.n_r) {
-                pid = page_table[(size_t)d.r * max_pages + b];
-                if (pid >= P_phys) {
-                    atomicOr(status, SE_DEV_BAD_PAGE_ID);
-                    pid = -1;
-                }
-            }
+        if (d.unit >= 0 && lane < kPB && d.b0 + lane < d.n_r)
+            pid = __ldg(page_table + (size_t)d.r * max_pages + d.b0 + lane);
+        return pid;
+    };
+    // issue the copies of one batch into buffer `slot`; returns this lane's physical page (or -1)
+    auto issue = [&](const Batch &d, int slot, int pid) -> int {
+        if (pid >= P_phys) {
+            atomicOr(status, SE_DEV_BAD_PAGE_ID);
+            pid = -1;
         }
         const unsigned valid = __ballot_sync(kFull, pid >= 0);
         const uint32_t bar = bar0 + slot * 8;
@@ -184,14 +184,26 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
         return pid;
     };
 
-    Batch cur, nxt;
+    // Three batches are live: `cur` is computed, `nxt` is in flight, `nn` has only its page-table
+    // entries on the way, so that its copies can be issued the moment a buffer frees up.
+    Batch cur, nxt, nn;
     decode_unit(gw, total_units, prefix, npages, B, H_kv, cur);
     if (cur.unit < 0) return;
     uint32_t phases = 0u;            // parity bit per buffer
     int slot = 0;
-    int pid_cur = issue(cur, slot);
+    int pid_cur = issue(cur, 0, load_pids(cur));
     load_qraw(cur);
+    convert_q();
+    nxt = cur;
+    next_batch(nxt);
     int pid_nxt = -1;
+    if (nxt.unit >= 0) {
+        pid_nxt = issue(nxt, 1, load_pids(nxt));
+        if (nxt.r != cur.r || nxt.h != cur.h) load_qraw(nxt);
+    }
+    nn = nxt;
+    next_batch(nn);
+    int pid_nn = load_pids(nn);
     bool failed = false;
 
     // ldmatrix row address of this lane inside a buffer: matrix (lane>>3) = {pages 0-7 | 8-15} x
@@ -199,18 +211,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
     const uint32_t lm_off = (uint32_t)(((lane & 7) + 8 * ((lane >> 3) & 1)) * C::PITCH + (lane >> 4) * 16);
 
     while (cur.unit >= 0) {
-        nxt = cur;
-        next_batch(nxt);
-        // the pair of `cur` may differ from the converted fragments: convert before qraw is reused
-        if (cur.r != q_r || cur.h != q_h) {
-            convert_q();
-            q_r = cur.r;
-            q_h = cur.h;
-        }
-        if (nxt.unit >= 0) {
-            pid_nxt = issue(nxt, slot ^ 1);
-            if (nxt.r != cur.r || nxt.h != cur.h) load_qraw(nxt);
-        }
         // wait for the current buffer
         if (!mbar_wait(bar0 + slot * 8, (phases >> slot) & 1u)) {
             failed = true;
@@ -242,8 +242,19 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
             if (cur.b0 + gid + 8 < cur.n_r) dst[gid + 8] = (pid_hi >= 0) ? s_hi * scale : ninf;
         }
         __syncwarp();        // every lane is done reading the buffer before it is refilled
+
+        // refill the buffer just consumed with `nn` (its page-table entries arrived long ago)
+        if (nn.unit >= 0) pid_nn = issue(nn, slot, pid_nn);
+        // advance: cur <- nxt <- nn <- the batch after
+        const bool pair_changed = nxt.unit >= 0 && (nxt.r != cur.r || nxt.h != cur.h);
         cur = nxt;
         pid_cur = pid_nxt;
+        if (pair_changed) convert_q();                 // qraw holds q of the pair that is now current
+        nxt = nn;
+        pid_nxt = pid_nn;
+        if (nxt.unit >= 0 && (nxt.r != cur.r || nxt.h != cur.h)) load_qraw(nxt);
+        next_batch(nn);
+        pid_nn = load_pids(nn);
         slot ^= 1;
     }
     if (failed) {
@@ -254,243 +265,239 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
 }
 
 // ---------------------------------------------------------------------------------
-// top-k: one CTA per (request, kv-head)
+// top-k: one CTA of 256 threads per (request, kv-head); thread t holds keys t, t+256, ...
+// in registers.  Radix select with 8-bit digits (shared-memory histogram, double buffered, one
+// CTA barrier per digit, every warp locates the crossing digit on its own), then a page-ordered
+// compaction with one more barrier.
 // ---------------------------------------------------------------------------------
+#ifndef SE_TOPK_MARK
+#define SE_TOPK_MARK(i)          // hook for an external timing probe; empty in the library
+#endif
 constexpr int kTopkThreads = 256;
 constexpr int kTopkWarps = kTopkThreads / 32;
 
-// Exclusive prefix sum over the CTA of one int per thread, in thread order.
-__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot, int &total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int inc = v;
+// Exclusive prefix over `entries` (multiple of 32, <= 256) ints in shared memory, computed by the
+// calling warp alone and written back in place.  Every warp of the CTA may run it on the same
+// array at the same time: they all write the same values.
+template <int ENTRIES>
+__device__ __forceinline__ int warp_scan_inplace(int *a, int lane) {
+    constexpr int EPL = ENTRIES / 32;
+    int v[EPL], sum = 0;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+        v[e] = a[lane * EPL + e];
+        sum += v[e];
+    }
+    int inc = sum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int t = __shfl_up_sync(kFull, inc, o);
         if (lane >= o) inc += t;
     }
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    int before = 0, tot = 0;
+    const int total = __shfl_sync(kFull, inc, 31);
+    int run = inc - sum;
+    __syncwarp();
 #pragma unroll
-    for (int w = 0; w < kTopkWarps; ++w) {
-        const int c = warp_tot[w];
-        if (w < warp) before += c;
-        tot += c;
+    for (int e = 0; e < EPL; ++e) {
+        a[lane * EPL + e] = run;
+        run += v[e];
     }
-    __syncthreads();
-    total = tot;
-    return before + inc - v;
+    __syncwarp();
+    return total;
 }
 
-// KPT = keys per thread held in registers (n <= KPT*256); KPT == 0 streams the keys from
-// global memory on every pass instead (any n).
+// KPT = keys per thread held in registers (n <= 256*KPT, KPT in {4,8,16,32}).
 template <int KPT>
-__global__ void __launch_bounds__(kTopkThreads)
+__global__ void __launch_bounds__(kTopkThreads, KPT <= 16 ? 4 : 2)
 topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_lens, int H_kv,
             int max_pages, int k_pages, int k_max, int32_t *__restrict__ sel_idx,
             int32_t *__restrict__ sel_cnt) {
-    constexpr bool kCached = KPT > 0;
-    constexpr int NK = kCached ? KPT : 1;
-    __shared__ int hist[256];
-    __shared__ int s_present, s_digit, s_above, s_inbin;
-    __shared__ int warp_tot[kTopkWarps];
-    __shared__ int cnt_tile[kCached ? KPT * kTopkWarps : 1];
+    constexpr int ENTRIES = KPT * kTopkWarps;          // (tile, warp) cells of the compaction
+    __shared__ int s_red[3][kTopkWarps];
+    __shared__ int s_hist[2][256];
+    __shared__ int s_cnt[2][ENTRIES];
+    SE_TOPK_MARK(9);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair = blockIdx.x;
     const int r = pair / H_kv;
     const int len = seq_lens[r];
     int n = len > 0 ? (len + kPage - 1) / kPage : 0;
     if (n > max_pages) n = max_pages;
+    if (n > KPT * kTopkThreads) n = KPT * kTopkThreads;       // cannot happen: the launcher picks KPT from max_pages
     const float *row = scores + (size_t)pair * max_pages;
     int32_t *out = sel_idx + (size_t)pair * k_max;
-
-    // element j of thread t is page j*256 + t (tile-major, so index order = (j, t) order)
-    uint32_t keys[NK];
-    if constexpr (kCached) {
-#pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            const int i = j * kTopkThreads + tid;
-            keys[j] = (i < n) ? f32_key(__ldg(row + i)) : 0u;
-        }
-    }
+    const unsigned lt_mask = (1u << lane) - 1u;
     const int tiles = (n + kTopkThreads - 1) / kTopkThreads;
-    auto key_at = [&](int j) -> uint32_t {
-        if constexpr (kCached) return keys[j];
+
+    // key j of thread t is page j*256 + t (tile-major, so (tile, thread) order is page order)
+    uint32_t keys[KPT];
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
         const int i = j * kTopkThreads + tid;
-        return (i < n) ? f32_key(row[i]) : 0u;
-    };
-
-    uint32_t prefix = 0;          // digits fixed so far (higher bits), lower bits zero
-    int remaining = 0;            // how many still to take among keys matching the prefix
-    int k_eff = 0;
-    bool ge_mode = false;         // take every key >= prefix (the whole bin is wanted)
-
-    if (tid == 0) s_present = 0;
-    for (int shift = 24; shift >= 0 && !ge_mode; shift -= 8) {
-        hist[tid] = 0;
-        __syncthreads();
-        int present = 0;
-        auto visit = [&](int j) {
-            const int i = j * kTopkThreads + tid;
-            if (i >= n) return;
-            const uint32_t key = key_at(j);
-            if (shift == 24) {
-                present += (key != kKeyAbsent);
-                atomicAdd(&hist[key >> 24], 1);
-            } else if ((key >> (shift + 8)) == (prefix >> (shift + 8))) {
-                atomicAdd(&hist[(key >> shift) & 255u], 1);
-            }
-        };
-        if constexpr (kCached) {
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) visit(j);
-        } else {
-            for (int j = 0; j < tiles; ++j) visit(j);
-        }
-        if (shift == 24 && present) atomicAdd(&s_present, present);
-        __syncthreads();
-        if (shift == 24) {
-            k_eff = min(min(k_pages, k_max), s_present);
-            remaining = k_eff;
-            if (k_eff == 0) break;
-        }
-        // find the digit d with  #(digits > d) < remaining <= #(digits >= d)
-        if (warp == 0) {
-            int loc[8], sum = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                loc[j] = hist[lane * 8 + j];
-                sum += loc[j];
-            }
-            int suf = sum;          // inclusive suffix sum over lanes (higher lanes = higher digits)
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int t = __shfl_down_sync(kFull, suf, o);
-                if (lane + o < 32) suf += t;
-            }
-            const int above_lane = suf - sum;      // digits in higher lanes
-            if (above_lane < remaining && remaining <= suf) {
-                int above = above_lane;
-#pragma unroll
-                for (int j = 7; j >= 0; --j) {
-                    if (above < remaining && remaining <= above + loc[j]) {
-                        s_digit = lane * 8 + j;
-                        s_above = above;
-                        s_inbin = loc[j];
-                    }
-                    above += loc[j];
-                }
-            }
-        }
-        __syncthreads();
-        prefix |= (uint32_t)s_digit << shift;
-        remaining -= s_above;
-        if (s_inbin == remaining) ge_mode = true;      // the whole bin is taken: no ties to break
-        __syncthreads();
+        keys[j] = (i < n) ? f32_key(__ldg(row + i)) : kKeyAbsent;
     }
+    SE_TOPK_MARK(0);
+
+    // ---- present pages, and the range of their keys
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    int present = 0;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const bool ok = keys[j] != kKeyAbsent;
+        present += ok;
+        kmin = ok ? min(kmin, keys[j]) : kmin;
+        kmax = ok ? max(kmax, keys[j]) : kmax;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        present += __shfl_xor_sync(kFull, present, o);
+        kmin = min(kmin, __shfl_xor_sync(kFull, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
+    }
+    if (lane == 0) {
+        s_red[0][warp] = present;
+        s_red[1][warp] = (int)kmin;
+        s_red[2][warp] = (int)kmax;
+    }
+    s_hist[0][tid] = 0;
+    __syncthreads();
+    present = 0;
+#pragma unroll
+    for (int w = 0; w < kTopkWarps; ++w) {
+        present += s_red[0][w];
+        kmin = min(kmin, (uint32_t)s_red[1][w]);
+        kmax = max(kmax, (uint32_t)s_red[2][w]);
+    }
+    const int k_eff = min(min(k_pages, k_max), present);
+    SE_TOPK_MARK(1);
+
+    // ---- radix select of the k_eff-th largest key.  All present keys share the bits above the
+    // highest bit in which kmin and kmax differ, so the digits start there (scores of one
+    // request typically share sign, exponent and a few mantissa bits).
+    uint32_t prefix = 0;          // bits decided so far, lower bits zero
+    int remaining = k_eff;        // how many still to take among keys matching the prefix
+    bool ge_mode = false;         // take every key >= prefix (no ties to break)
+    if (k_eff > 0) {
+        if (k_eff == present) {               // everything present is wanted
+            prefix = kmin;
+            ge_mode = true;
+        } else if (kmin == kmax) {            // all equal: ties only
+            prefix = kmax;
+        } else {
+            int hi = 32 - __clz(kmin ^ kmax);                   // undecided low bits
+            prefix = (hi >= 32) ? 0u : (kmax >> hi) << hi;
+            int par = 0;
+            while (hi > 0 && !ge_mode) {
+                const int w = hi < 8 ? hi : 8;
+                const int shift = hi - w;
+                int *hist = s_hist[par];
+                // the digits are spread after the range narrowing, so plain shared-memory atomics
+                // rarely collide; tiles past the request's length are skipped altogether
+#pragma unroll
+                for (int j = 0; j < KPT; ++j) {
+                    if (j < tiles) {
+                        const uint32_t key = keys[j];
+                        const bool active = key != kKeyAbsent && ((hi >= 32) || ((key >> hi) == (prefix >> hi)));
+                        if (active) atomicAdd(&hist[(key >> shift) & ((1u << w) - 1u)], 1);
+                    }
+                }
+                s_hist[par ^ 1][tid] = 0;            // the other buffer serves the next digit
+                __syncthreads();
+                // every warp finds the digit d with  #(digits > d) < remaining <= #(digits >= d)
+                // on its own: lane l owns digits 8l..8l+7, higher lanes hold higher digits
+                int loc[8], sum = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    loc[j] = hist[lane * 8 + j];
+                    sum += loc[j];
+                }
+                int suf = sum;              // inclusive suffix sum over lanes
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_down_sync(kFull, suf, o);
+                    if (lane + o < 32) suf += t;
+                }
+                const int above_lane = suf - sum;
+                const bool mine = above_lane < remaining && remaining <= suf;
+                int digit = 0, above_d = 0, inbin = 0;
+                if (mine) {
+                    int above = above_lane;
+#pragma unroll
+                    for (int j = 7; j >= 0; --j) {
+                        if (above < remaining && remaining <= above + loc[j]) {
+                            digit = lane * 8 + j;
+                            above_d = above;
+                            inbin = loc[j];
+                        }
+                        above += loc[j];
+                    }
+                }
+                const int owner = __ffs(__ballot_sync(kFull, mine)) - 1;
+                digit = __shfl_sync(kFull, digit, owner);
+                above_d = __shfl_sync(kFull, above_d, owner);
+                inbin = __shfl_sync(kFull, inbin, owner);
+                prefix |= (uint32_t)digit << shift;
+                remaining -= above_d;
+                if (inbin == remaining) ge_mode = true;      // the whole bin is taken
+                hi = shift;
+                par ^= 1;
+                SE_TOPK_MARK(2);
+            }
+        }
+    }
+    SE_TOPK_MARK(3);
 
     if (k_eff == 0) {
         for (int i = tid; i < k_max; i += kTopkThreads) out[i] = -1;
         if (tid == 0) sel_cnt[pair] = 0;
         return;
     }
-    // keys > T are taken; keys == T are taken in index order until `need` of them are in.
-    // In ge_mode every key >= prefix is taken (T = prefix, need = unlimited).
+    // ---- ordered compaction: keys > T are taken; keys == T are taken in page order until `need`
+    // of them are in; in ge_mode every key >= T is taken.
     const uint32_t T = prefix;
-    const int need = ge_mode ? 0x7fffffff : remaining;
-
-    if constexpr (kCached) {
-        // ---- registers: rank the ties, then the selected, with two CTA-wide scans over (tile, warp)
-        uint32_t eqmask = 0, takemask = 0;
+    uint32_t takemask = 0, eqmask = 0;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const bool valid = keys[j] != kKeyAbsent;
+        const bool gt = valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T));
+        const bool eq = valid && !ge_mode && (keys[j] == T);
+        takemask |= (uint32_t)gt << j;
+        eqmask |= (uint32_t)eq << j;
+    }
+    if (!ge_mode) {                            // rank the ties (CTA-uniform branch)
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-            const int i = j * kTopkThreads + tid;
-            const bool valid = i < n;
-            const bool gt = valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T));
-            const bool eq = valid && !ge_mode && (keys[j] == T);
-            eqmask |= (uint32_t)eq << j;
-            takemask |= (uint32_t)gt << j;
-        }
-        int total;
-        if (!ge_mode) {
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
-                if (lane == 0) cnt_tile[j * kTopkWarps + warp] = __popc(b);
-            }
-            __syncthreads();
-            const int mine = tid < KPT * kTopkWarps ? cnt_tile[tid] : 0;
-            const int off = block_exclusive_scan(mine, warp_tot, total);
-            if (tid < KPT * kTopkWarps) cnt_tile[tid] = off;
-            __syncthreads();
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
-                const int rank = cnt_tile[j * kTopkWarps + warp] + __popc(b & ((1u << lane) - 1u));
-                if (((eqmask >> j) & 1u) && rank < need) takemask |= 1u << j;
-            }
-            __syncthreads();
-        }
-#pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
-            if (lane == 0) cnt_tile[j * kTopkWarps + warp] = __popc(b);
+            const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
+            if (lane == 0) s_cnt[1][j * kTopkWarps + warp] = __popc(b);
         }
         __syncthreads();
-        const int mine = tid < KPT * kTopkWarps ? cnt_tile[tid] : 0;
-        const int off = block_exclusive_scan(mine, warp_tot, total);
-        if (tid < KPT * kTopkWarps) cnt_tile[tid] = off;
-        __syncthreads();
+        warp_scan_inplace<ENTRIES>(s_cnt[1], lane);
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-            const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
-            const int pos = cnt_tile[j * kTopkWarps + warp] + __popc(b & ((1u << lane) - 1u));
-            if (((takemask >> j) & 1u) && pos < k_max) out[pos] = j * kTopkThreads + tid;
-        }
-    } else {
-        // ---- streaming: tile by tile, carrying the running counts
-        int run_eq = 0, run_sel = 0;
-        __shared__ int warp_eq[kTopkWarps], warp_sel[kTopkWarps];
-        for (int base = 0; base < n; base += kTopkThreads) {
-            const int i = base + tid;
-            uint32_t key = 0;
-            bool gt = false, eq = false;
-            if (i < n) {
-                key = f32_key(row[i]);
-                gt = ge_mode ? (key >= T) : (key > T);
-                eq = !ge_mode && (key == T);
-            }
-            const unsigned beq = __ballot_sync(kFull, eq);
-            if (lane == 0) warp_eq[warp] = __popc(beq);
-            __syncthreads();
-            int eq_before = run_eq, eq_total = 0;
-#pragma unroll
-            for (int w = 0; w < kTopkWarps; ++w) {
-                const int c = warp_eq[w];
-                if (w < warp) eq_before += c;
-                eq_total += c;
-            }
-            eq_before += __popc(beq & ((1u << lane) - 1u));
-            const bool take = gt || (eq && eq_before < need);
-            const unsigned bsel = __ballot_sync(kFull, take);
-            if (lane == 0) warp_sel[warp] = __popc(bsel);
-            __syncthreads();
-            int pos = run_sel, sel_total = 0;
-#pragma unroll
-            for (int w = 0; w < kTopkWarps; ++w) {
-                const int c = warp_sel[w];
-                if (w < warp) pos += c;
-                sel_total += c;
-            }
-            pos += __popc(bsel & ((1u << lane) - 1u));
-            if (take && pos < k_max) out[pos] = i;
-            run_eq += eq_total;
-            run_sel += sel_total;
-            __syncthreads();
+            const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
+            const int rank = s_cnt[1][j * kTopkWarps + warp] + __popc(b & lt_mask);
+            if (((eqmask >> j) & 1u) && rank < remaining) takemask |= 1u << j;
         }
     }
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
+        if (lane == 0) s_cnt[0][j * kTopkWarps + warp] = __popc(b);
+    }
+    __syncthreads();
+    warp_scan_inplace<ENTRIES>(s_cnt[0], lane);
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        if (j < tiles) {
+            const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
+            const int pos = s_cnt[0][j * kTopkWarps + warp] + __popc(b & lt_mask);
+            if (((takemask >> j) & 1u) && pos < k_max) out[pos] = j * kTopkThreads + tid;
+        }
+    }
+    SE_TOPK_MARK(4);
     for (int i = k_eff + tid; i < k_max; i += kTopkThreads) out[i] = -1;
     if (tid == 0) sel_cnt[pair] = k_eff;
+    SE_TOPK_MARK(5);
 }
 
 template <int D>
@@ -530,13 +537,13 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
                         : launch_score<64>(p, q, meta, page_table, seq_lens, scores, status, stream);
     if (e != cudaSuccess) return e;
     const int pairs = p.B * p.H_kv;
-#define SE_TOPK(KPT)                                                                                   \
+#define SE_TOPK(KPT)                                                                                    \
     topk_kernel<KPT><<<pairs, kTopkThreads, 0, stream>>>(scores, seq_lens, p.H_kv, p.max_pages, k_pages, \
                                                          p.k_max, sel_idx, sel_cnt)
     if (p.max_pages <= 4 * kTopkThreads) SE_TOPK(4);
+    else if (p.max_pages <= 8 * kTopkThreads) SE_TOPK(8);
     else if (p.max_pages <= 16 * kTopkThreads) SE_TOPK(16);
-    else if (p.max_pages <= 32 * kTopkThreads) SE_TOPK(32);
-    else SE_TOPK(0);
+    else SE_TOPK(32);
 #undef SE_TOPK
     return cudaGetLastError();
 }
