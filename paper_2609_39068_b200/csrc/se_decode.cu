@@ -216,12 +216,31 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         const int i_lo = my_split * pages_per_split;
         if (i_lo >= k_max) continue;
         const int r = pair / H_kv, h = pair % H_kv;
-        int cnt = sel_cnt[pair];
+        const int seg_begin = pair * k_max + i_lo;
+
+        // ---- Q as the A operand: row gid = query head gid of the group (rows >= G and 8..15 are
+        // zero).  Issued first: these loads depend on nothing and overlap the look-ups below.
+        uint32_t qa[C::KSTEPS][2];
+        {
+            const uint16_t *src = q + ((size_t)r * H_q + h * G + (head_ok ? gid : 0)) * D + 2 * tid4;
+#pragma unroll
+            for (int s = 0; s < C::KSTEPS; ++s) {
+                const uint32_t w0 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16));
+                const uint32_t w1 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16 + 8));
+                qa[s][0] = head_ok ? w0 : 0u;
+                qa[s][1] = head_ok ? w1 : 0u;
+            }
+        }
+        // ---- page list of the unit's slot range: selection entries, selection count and length
+        // travel together (one round trip), the page-table entries follow (a second one)
+        x_end = pair * k_max + min(i_lo + pages_per_split, k_max);
+        fill_chunk(seg_begin);
+        int cnt = __ldg(sel_cnt + pair);          // same words the look-up just fetched: cache hits
         if (cnt > k_max) {
             if (lane == 0) atomicOr(status, SE_DEV_BAD_SELECTION);
             cnt = k_max;
         }
-        const int len = seq_lens[r];
+        const int len = __ldg(seq_lens + r);
         const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
         if (cnt <= 0 || n_r == 0) {
             if (my_split == 0) {      // the first split of the pair reports "nothing attended"
@@ -235,28 +254,10 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         }
         if (i_lo >= cnt) continue;
         const int i_hi = min(min(i_lo + pages_per_split, k_max), cnt);
-        const int seg_begin = pair * k_max + i_lo;
         const int seg_end = pair * k_max + i_hi;                      // first slot past this unit
         const int n_split = (cnt + pages_per_split - 1) / pages_per_split;   // splits of this pair that hold pages
-        x_end = seg_end;
-
-        // make sure the page list covers the start of the segment, and get copies going before
-        // the (dependent) q loads below are waited for
-        fill_chunk(seg_begin);
         top_up();
 
-        // ---- Q as the A operand: row gid = query head gid of the group (rows >= G and 8..15 are zero)
-        uint32_t qa[C::KSTEPS][2];
-        {
-            const uint16_t *src = q + ((size_t)r * H_q + h * G + (head_ok ? gid : 0)) * D + 2 * tid4;
-#pragma unroll
-            for (int s = 0; s < C::KSTEPS; ++s) {
-                const uint32_t w0 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16));
-                const uint32_t w1 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16 + 8));
-                qa[s][0] = head_ok ? w0 : 0u;
-                qa[s][1] = head_ok ? w1 : 0u;
-            }
-        }
         float o_acc[C::NTILES][4];
 #pragma unroll
         for (int nt = 0; nt < C::NTILES; ++nt) {
