@@ -62,6 +62,7 @@ extern "C" {
 #define SE_ERR_NULL_POINTER        -3   /* a required pointer is NULL                      */
 #define SE_ERR_MISALIGNED          -4   /* a pointer is not 16-byte aligned                */
 #define SE_ERR_CUDA                -5   /* a CUDA runtime call failed (launch, attribute)  */
+#define SE_ERR_SCRATCH_TOO_SMALL   -6   /* problem exceeds the built-in scratch (se_page_select_static) */
 
 /* bits of the device status word */
 #define SE_DEV_BAD_PAGE_ID          1u  /* page_table entry >= num_phys_pages              */
@@ -160,6 +161,38 @@ int se_sparse_decode(const se_params *p, const void *q, const void *k_cache,
                      const int32_t *seq_lens, const int32_t *sel_idx,
                      const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
                      void *workspace, void *stream);
+
+/*
+ * se_page_select without any caller-provided scratch.  (The paper has no counterpart: this entry
+ * point exists for the way some hosts have to call the library.)
+ *
+ * Who needs it: code that may not allocate device memory at the point where it runs the
+ * selection - a serving loop whose memory pool is fully handed out before the first request, a
+ * plug-in that receives tensors but no allocator, a real-time thread in which cudaMalloc's
+ * implicit synchronisation is not acceptable.  Those callers cannot size and allocate the
+ * workspace that se_page_select wants, so here the only scratch the selection needs - the fp32
+ * page scores - lives in a fixed array inside the library: SE_STATIC_SCRATCH_BYTES of device
+ * memory that every GPU which loads the library holds until the process exits.
+ *
+ * Same arguments, same results (bit for bit) as se_page_select, except:
+ *   - no workspace argument; nothing is allocated or freed, by this call or on its behalf;
+ *   - dev_status (nullable, 4-byte aligned DEVICE pointer, caller-owned) receives the status
+ *     word of this call (SE_DEV_* bits) once the stream reaches that point;
+ *   - the shape is limited by the array: 256 + 4*B*H_kv*max_pages bytes must not exceed
+ *     SE_STATIC_SCRATCH_BYTES, otherwise SE_ERR_SCRATCH_TOO_SMALL is returned and nothing is
+ *     enqueued.
+ * The first call on a device looks up the array's device address (a set-up step, done once per
+ * device with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps the contents of the last call: the call
+ * clears the status word itself, and the scores are rewritten before they are read.  Two calls
+ * whose kernels may overlap on the GPU (different streams without an ordering between them)
+ * race on the array; order them.
+ */
+#define SE_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u)
+int se_page_select_static(const se_params *p, const void *q, const void *meta,
+                          const int32_t *page_table, const int32_t *seq_lens,
+                          int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
+                          int32_t *dev_status, void *stream);
 
 /*
  * Copies the device status word (an OR of SE_DEV_* bits, 0 = clean) to *host_out and

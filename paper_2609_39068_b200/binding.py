@@ -21,7 +21,8 @@ SE_DEV_BAD_SELECTION = 2
 SE_DEV_WAIT_TIMEOUT = 4
 
 EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_workspace_init", "se_meta_update",
-           "se_page_select", "se_sparse_decode", "se_last_device_status")
+           "se_page_select", "se_sparse_decode", "se_last_device_status", "se_page_select_static")
+SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
 class SeParams(ctypes.Structure):
@@ -64,8 +65,9 @@ def load(build_if_missing: bool = True):
     lib.se_page_select.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_sparse_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, fp, fp, fp, vp, vp]
     lib.se_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_sparse_decode",
-                 "se_last_device_status"):
+                 "se_last_device_status", "se_page_select_static"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -151,6 +153,21 @@ def se_sparse_decode(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_
                                    _ptr(out, torch.float32, "out"), _ptr(lse, torch.float32, "lse"),
                                    _ptr(score_accum, torch.float32, "score_accum"),
                                    _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_sparse_decode")
+
+
+def se_page_select_static(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,
+                          dev_status=None) -> None:
+    """Page selection that uses the library's built-in scratch array instead of a workspace
+    (for callers that cannot allocate); ``dev_status`` is an optional 1-element int32 CUDA
+    tensor that receives the call's status word."""
+    _check(load().se_page_select_static(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                        _ptr(meta, torch.bfloat16, "meta"),
+                                        _ptr(page_table, torch.int32, "page_table"),
+                                        _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens),
+                                        _ptr(sel_idx, torch.int32, "sel_idx"),
+                                        _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                        _ptr(dev_status, torch.int32, "dev_status"), _stream()),
+           "se_page_select_static")
 
 
 def se_last_device_status(workspace) -> int:

@@ -99,6 +99,7 @@ const char *se_strerror(int code) {
         case SE_ERR_NULL_POINTER: return "required pointer is NULL";
         case SE_ERR_MISALIGNED: return "pointer is not 16-byte aligned";
         case SE_ERR_CUDA: return "CUDA runtime error";
+        case SE_ERR_SCRATCH_TOO_SMALL: return "problem exceeds the built-in scratch array";
     }
     return "unknown error code";
 }

@@ -549,3 +549,68 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
 }
 
 }  // namespace se
+
+// ---------------------------------------------------------------------------------
+// se_page_select_static: page selection for callers that cannot allocate device memory.
+// The fp32 page scores (the only scratch the selection needs) live in the array below, which
+// every GPU that loads this library holds from load to exit.
+// ---------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_select_scratch[SE_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+void *g_scratch_ptr[kMaxDevices];          // device address of g_select_scratch, per device ordinal
+bool g_scratch_ready[kMaxDevices];
+
+// The array's name is only a host-side handle: the address kernels can use has to be asked for,
+// once per device, with that device current.
+int static_scratch(void **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SE_ERR_CUDA;
+    if (!g_scratch_ready[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_select_scratch) != cudaSuccess || ptr == nullptr) return SE_ERR_CUDA;
+        g_scratch_ptr[dev] = ptr;
+        g_scratch_ready[dev] = true;
+    }
+    *out = g_scratch_ptr[dev];
+    return SE_OK;
+}
+
+}  // namespace
+
+extern "C" int se_page_select_static(const se_params *p, const void *q, const void *meta,
+                                     const int32_t *page_table, const int32_t *seq_lens,
+                                     int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
+                                     int32_t *dev_status, void *stream) {
+    if (!p) return SE_ERR_NULL_POINTER;
+    if (se_workspace_bytes(p) == 0) return SE_ERR_INVALID_ARG;          // same shape rules as every call
+    if (!q || !meta || !page_table || !seq_lens || !sel_idx || !sel_cnt) return SE_ERR_NULL_POINTER;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(meta) |
+                           reinterpret_cast<uintptr_t>(page_table) | reinterpret_cast<uintptr_t>(seq_lens) |
+                           reinterpret_cast<uintptr_t>(sel_idx) | reinterpret_cast<uintptr_t>(sel_cnt);
+    if ((bits & 15u) || (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return SE_ERR_MISALIGNED;
+    if (budget_tokens < se::kPage || budget_tokens / se::kPage > p->k_max) return SE_ERR_INVALID_ARG;
+    // scratch layout: [status word, padded to 256 bytes][fp32 scores, B*H_kv*max_pages]
+    const size_t need = 256 + (size_t)p->B * p->H_kv * p->max_pages * sizeof(float);
+    if (need > SE_STATIC_SCRATCH_BYTES) return SE_ERR_SCRATCH_TOO_SMALL;
+    void *scratch = nullptr;
+    const int rc = static_scratch(&scratch);
+    if (rc != SE_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the last call left: the status word has to start at zero, the
+    // scores are rewritten for every page before they are read
+    if (cudaMemsetAsync(scratch, 0, 256, s) != cudaSuccess) return SE_ERR_CUDA;
+    se::WorkspaceLayout L = {};
+    L.status = 0;
+    L.scores = 256;
+    L.total = need;
+    cudaError_t e = se::launch_page_select(*p, q, meta, page_table, seq_lens, budget_tokens / se::kPage,
+                                           sel_idx, sel_cnt, scratch, L, s);
+    if (e != cudaSuccess) return SE_ERR_CUDA;
+    if (dev_status &&
+        cudaMemcpyAsync(dev_status, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return SE_ERR_CUDA;
+    return SE_OK;
+}
