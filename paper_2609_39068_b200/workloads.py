@@ -272,6 +272,23 @@ def sub_workload(w: Workload, rows, device="cpu") -> Workload:
         score_accum=accum)
 
 
+def shard_kv_heads(w: Workload, rank: int, world: int) -> Workload:
+    """Tensor-parallel shard ``rank`` of ``world``: a contiguous block of kv-heads with their
+    query heads.  Page table and lengths are replicated; no step of the path needs data of
+    another shard (pure slicing, no arithmetic)."""
+    assert w.H_kv % world == 0
+    hk = w.H_kv // world
+    G = w.H_q // w.H_kv
+    ks = slice(rank * hk, (rank + 1) * hk)
+    qs = slice(rank * hk * G, (rank + 1) * hk * G)
+    return Workload(
+        name="%s_tp%dof%d" % (w.name, rank, world), B=w.B, H_q=hk * G, H_kv=hk, D=w.D, budget=w.budget,
+        max_pages=w.max_pages, num_phys_pages=w.num_phys_pages, q=w.q[:, qs].contiguous(),
+        k_cache=w.k_cache[:, ks].contiguous(), v_cache=w.v_cache[:, ks].contiguous(),
+        page_table=w.page_table, seq_lens=w.seq_lens,
+        score_accum=None if w.score_accum is None else w.score_accum[:, ks].contiguous())
+
+
 def bf16_bits(t: torch.Tensor):
     """The raw bf16 bit patterns of ``t`` as a numpy uint16 array on the host."""
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view("uint16")
