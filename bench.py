@@ -40,7 +40,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
 # capture summarised in profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/decode_kernel_config3_b24.md: 205.57 MB for 24576 tiles, scaled to 65536 tiles
+    "config3_contbatch_b64_mix": 548.2e6,
+}
 
 
 def measured_peak():
