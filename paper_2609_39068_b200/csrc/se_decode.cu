@@ -93,7 +93,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)kDecWarps * C::WARP_SMEM) + warp * C::NSTAGE;
     if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(smem_u32(&bars[s]), 2 * C::HALVES);
         mbar_fence_init();
     }
     __syncwarp();
@@ -192,17 +192,17 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         ce = 0;
         pe = 0;
     };
-    // called between pages, when no stage is being read: fill every free stage.  Lane 0 arms the
-    // barrier; one lane per 16x64 tile issues its tensor copy.
+    // called between pages, when no stage is being read: fill every free stage.  One lane per
+    // 16x64 tile arms the stage's barrier with its own byte count and issues its tensor copy (the
+    // barrier expects one arrival per tile, so the lanes need no ordering among themselves).
     auto top_up = [&]() {
         while (pe < n_ent && pe < ce + C::NSTAGE) {
-            const uint32_t bar = bar0 + stage_i * 8;
-            if (lane == 0) mbar_expect_tx(bar, C::STAGEB);
-            __syncwarp();
             if (lane < 2 * C::HALVES) {
+                const uint32_t bar = bar0 + stage_i * 8;
                 const int y = ent_y[pe];
                 const int hf = lane >> 1;
                 const uint32_t dst = ring0 + stage_i * C::STAGEB + (lane & 1) * C::PAGEB + hf * kTileBytes;
+                mbar_expect_tx(bar, kTileBytes);
                 tma_load_2d(dst, (lane & 1) ? &v_map : &k_map, hf * 64, y, bar);
             }
             stage_i = (stage_i + 1 == C::NSTAGE) ? 0 : stage_i + 1;
@@ -290,15 +290,22 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
 
             // ---- S^T[head, token] = Q . K^T : two n8 tiles (tokens 0-7, 8-15)
             float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+            float s0b[4] = {0.f, 0.f, 0.f, 0.f}, s1b[4] = {0.f, 0.f, 0.f, 0.f};   // odd k-steps: shorter chains
 #pragma unroll
             for (int s = 0; s < C::KSTEPS; ++s) {
                 const int hf = s >> 2;
                 const int chunk = 2 * (s & 3) + k_chunk_add;
                 uint32_t b00, b01, b10, b11;     // {tok 0-7: k lo, k hi}, {tok 8-15: k lo, k hi}
                 ldmatrix_x4(Ks + hf * kTileBytes + k_row * 128 + ((chunk ^ (k_row & 7)) << 4), b00, b01, b10, b11);
-                mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
-                mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+                if (s & 1) {
+                    mma_bf16_16816(s0b, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                    mma_bf16_16816(s1b, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+                } else {
+                    mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                    mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+                }
             }
+            s0[0] += s0b[0]; s0[1] += s0b[1]; s1[0] += s1b[0]; s1[1] += s1b[1];
             // this lane: head gid, tokens 2*tid4, 2*tid4+1 (s0) and 8+2*tid4, 9+2*tid4 (s1)
             const int t0 = 2 * tid4;
             float z[4];
