@@ -148,6 +148,15 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
             }
     };
 
+    // Work units are handed out dynamically: a warp's first unit is its own index, every further
+    // one comes from a global counter.  The counter is bumped when a unit is entered and the
+    // answer is only needed when that unit ends (four batches later), so the round trip is hidden.
+    // SMs that get less memory bandwidth simply fetch fewer units.
+    uint32_t *queue = status + 16, *done = status + 17;
+    int pending_unit = 0;                        // valid in lane 0
+    auto request_unit = [&]() {
+        if (lane == 0) pending_unit = tw + (int)atomicAdd(queue, 1u);
+    };
     // advance a descriptor to the next batch of this warp's stream
     auto next_batch = [&](Batch &d) {
         if (d.unit < 0) return;
@@ -156,7 +165,18 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
             d.b0 += kPB;
             return;
         }
-        decode_unit(d.unit + tw, total_units, prefix, npages, B, H_kv, d);
+        const int u = __shfl_sync(kFull, pending_unit, 0);
+        if (decode_unit(u, total_units, prefix, npages, B, H_kv, d)) request_unit();
+    };
+    // every warp checks out once; the last one leaves the counters at zero for the next launch
+    auto check_out = [&]() {
+        if (lane == 0) {
+            const uint32_t old = atomicAdd(done, 1u);
+            if (old == (uint32_t)tw - 1u) {
+                *queue = 0u;
+                *done = 0u;
+            }
+        }
     };
 
     // page-table entries of a batch: lane j < 16 loads the entry of page b0 + j.  The value is not
@@ -188,7 +208,11 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
     // entries on the way, so that its copies can be issued the moment a buffer frees up.
     Batch cur, nxt, nn;
     decode_unit(gw, total_units, prefix, npages, B, H_kv, cur);
-    if (cur.unit < 0) return;
+    if (cur.unit < 0) {
+        check_out();
+        return;
+    }
+    request_unit();
     uint32_t phases = 0u;            // parity bit per buffer
     int slot = 0;
     int pid_cur = issue(cur, 0, load_pids(cur));
@@ -262,6 +286,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
         // give the copy that may still be in flight a bounded chance to land before leaving
         mbar_wait(bar0 + (slot ^ 1) * 8, (phases >> (slot ^ 1)) & 1u);
     }
+    check_out();
 }
 
 // ---------------------------------------------------------------------------------
