@@ -81,6 +81,9 @@ typedef struct se_params {
     int32_t k_max;           /* row stride of sel_idx, >= floor(budget / 16), 1..4096       */
     float   sm_scale;        /* logit scale; 0 selects 1/sqrt(D)                            */
     uint32_t flags;          /* reserved, must be 0                                         */
+    int32_t sink_pages;      /* se_page_select: the first this many logical pages of every  */
+    int32_t recent_pages;    /* request and the last this many are always selected, outside
+                                the budget (0 = pure top-k); see se_page_select             */
 } se_params;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -132,8 +135,14 @@ int se_meta_update(const se_params *p, const void *k_cache, const int32_t *page_
  * and sel_idx[r,h,:] receives the k_eff = min(floor(budget_tokens/16), #present pages)
  * pages with the largest P (equal scores: lower page first), in ascending page order,
  * padded with -1; sel_cnt[r,h] = k_eff.  A request with seq_len 0 or no present page
- * gets sel_cnt 0.  Requires 16 <= budget_tokens <= 16*k_max.  Never writes q, meta or
- * the page table.  Uses the workspace for the fp32 scores.
+ * gets sel_cnt 0.  Never writes q, meta or the page table.  Uses the workspace for the fp32
+ * scores.
+ * Forced pages (the paper's Quest settings read "sink" and "recent" tokens in addition to the
+ * selected budget, Appendix C "Experimental Settings"): with p->sink_pages = s and
+ * p->recent_pages = t, the logical pages 0..s-1 and ceil(len_r/16)-t..ceil(len_r/16)-1 of every
+ * request are always part of the result when they are present; they are not candidates of the
+ * top-k and do not count against the budget, so sel_cnt can reach floor(budget/16) + s + t.
+ * Requires 16 <= budget_tokens and floor(budget_tokens/16) + s + t <= k_max.
  */
 int se_page_select(const se_params *p, const void *q, const void *meta,
                    const int32_t *page_table, const int32_t *seq_lens,

@@ -120,18 +120,26 @@ def quest_scores(q, meta, page_table, seq_lens, page_size=16, sm_scale=None, gro
     return S, P, present.astype(bool)
 
 
-def topk_pages(P, present, budget, page_size=16, k_max=None):
+def topk_pages(P, present, budget, page_size=16, k_max=None, sink_pages=0, recent_pages=0, seq_lens=None):
     """Returns (sel_idx [B,H_kv,k_max] int32 ascending / -1 padded, sel_cnt [B,H_kv],
-    theta [B,H_kv,2] = the k_eff-th and (k_eff+1)-th largest score, NaN where undefined)."""
+    theta [B,H_kv,2] = the k_eff-th and (k_eff+1)-th largest candidate score, NaN where
+    undefined).  ``sink_pages`` / ``recent_pages`` force the first / last pages of every request
+    into the result outside the budget (``seq_lens`` then tells where a request ends)."""
     P = np.ascontiguousarray(P, dtype=np.float64)
     B, H_kv, max_pages = P.shape
     pres = np.ascontiguousarray(present, dtype=np.uint8)
     if k_max is None:
-        k_max = max(budget // page_size, 1)
+        k_max = max(budget // page_size + sink_pages + recent_pages, 1)
+    n_pages = None
+    if seq_lens is not None:
+        n_pages = np.ascontiguousarray((np.asarray(seq_lens, dtype=np.int64) + page_size - 1) // page_size, dtype=np.int32)
+    elif recent_pages:
+        raise ValueError("recent_pages needs seq_lens")
     sel_idx = np.full((B, H_kv, k_max), -1, dtype=np.int32)
     sel_cnt = np.zeros((B, H_kv), dtype=np.int32)
     theta = np.zeros((B, H_kv, 2), dtype=np.float64)
     _load().se_oracle_topk(B, H_kv, page_size, max_pages, k_max, int(budget),
+                           int(sink_pages), int(recent_pages), _p(n_pages, ctypes.c_int32),
                            _p(P, ctypes.c_double), _p(pres, ctypes.c_uint8),
                            _p(sel_idx, ctypes.c_int32), _p(sel_cnt, ctypes.c_int32),
                            _p(theta, ctypes.c_double))
@@ -170,11 +178,11 @@ def attend(q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
 
 
 def decode_step(q, k_cache, v_cache, page_table, seq_lens, budget, meta=None,
-                page_size=16, sm_scale=None, u_accum=None, k_max=None):
+                page_size=16, sm_scale=None, u_accum=None, k_max=None, sink_pages=0, recent_pages=0):
     """One decode step: summary of the newest page, scores, top-k, attention."""
     meta = quest_meta(k_cache, page_table, seq_lens, page_size, first_tok=None, meta=meta)
     S, P, present = quest_scores(q, meta, page_table, seq_lens, page_size, sm_scale)
-    sel_idx, sel_cnt, theta = topk_pages(P, present, budget, page_size, k_max)
+    sel_idx, sel_cnt, theta = topk_pages(P, present, budget, page_size, k_max, sink_pages, recent_pages, seq_lens)
     out, lse = attend(q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
                       page_size, sm_scale, u_accum)
     return dict(meta=meta, S=S, P=P, present=present, sel_idx=sel_idx, sel_cnt=sel_cnt,

@@ -161,37 +161,49 @@ static int int_cmp(const void *x, const void *y) {
 }
 
 /*
- * TopK: among the present pages of request r, the k_eff = min(floor(budget/p), #present)
+ * TopK: among the present pages of request r, the k_eff = min(floor(budget/p), #candidates)
  * pages with the largest P[r,h,.]; equal scores are ordered by lower logical page.  The
  * chosen logical page numbers are written in ascending order, the rest of the row is -1.
- * theta[r,h,0] is the k_eff-th largest score, theta[r,h,1] the (k_eff+1)-th (NaN if none):
- * the caller uses them to see how close a decision was.
+ * Forced pages (the paper's Quest settings keep "sink" and "recent" tokens outside the selected
+ * budget): the first sink_pages logical pages and the last recent_pages logical pages of the
+ * request (n_pages[r] = pages the request's length spans) are always in the result when present;
+ * they are not candidates and do not count against the budget.
+ * theta[r,h,0] is the k_eff-th largest candidate score, theta[r,h,1] the (k_eff+1)-th (NaN if
+ * none): the caller uses them to see how close a decision was.
  *   sel_idx [B,H_kv,k_max]   sel_cnt [B,H_kv]   theta [B,H_kv,2]
  */
 void se_oracle_topk(int B, int H_kv, int p, int max_pages, int k_max, int budget,
+                    int sink_pages, int recent_pages, const int32_t *n_pages,
                     const double *P, const uint8_t *present,
                     int32_t *sel_idx, int32_t *sel_cnt, double *theta) {
     int k = budget / p;
 #pragma omp parallel for schedule(dynamic)
     for (int rh = 0; rh < B * H_kv; ++rh) {
         int r = rh / H_kv;
+        int n_r = n_pages ? n_pages[r] : max_pages;
         cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(max_pages > 0 ? max_pages : 1));
-        int n = 0;
-        for (int b = 0; b < max_pages; ++b)
-            if (present[(size_t)r * max_pages + b]) {
+        int *chosen = (int *)malloc(sizeof(int) * (size_t)(max_pages > 0 ? max_pages : 1));
+        int n = 0, n_chosen = 0;
+        for (int b = 0; b < max_pages; ++b) {
+            if (!present[(size_t)r * max_pages + b]) continue;
+            int forced = (b < sink_pages) || (b >= n_r - recent_pages && b < n_r);
+            if (forced) {
+                chosen[n_chosen++] = b;
+            } else {
                 cand[n].s = P[(size_t)rh * max_pages + b];
                 cand[n].b = b;
                 ++n;
             }
+        }
         qsort(cand, (size_t)n, sizeof(cand_t), cand_cmp);
         int k_eff = k < n ? k : n;
-        if (k_eff > k_max) k_eff = k_max;
-        int *chosen = (int *)malloc(sizeof(int) * (size_t)(k_eff > 0 ? k_eff : 1));
-        for (int i = 0; i < k_eff; ++i) chosen[i] = cand[i].b;
-        qsort(chosen, (size_t)k_eff, sizeof(int), int_cmp);
+        if (k_eff > k_max - n_chosen) k_eff = k_max - n_chosen > 0 ? k_max - n_chosen : 0;
+        if (n_chosen > k_max) n_chosen = k_max;
+        for (int i = 0; i < k_eff; ++i) chosen[n_chosen++] = cand[i].b;
+        qsort(chosen, (size_t)n_chosen, sizeof(int), int_cmp);
         for (int i = 0; i < k_max; ++i)
-            sel_idx[(size_t)rh * k_max + i] = i < k_eff ? chosen[i] : -1;
-        sel_cnt[rh] = k_eff;
+            sel_idx[(size_t)rh * k_max + i] = i < n_chosen ? chosen[i] : -1;
+        sel_cnt[rh] = n_chosen;
         theta[(size_t)rh * 2 + 0] = k_eff > 0 ? cand[k_eff - 1].s : NAN;
         theta[(size_t)rh * 2 + 1] = k_eff < n ? cand[k_eff].s : NAN;
         free(chosen);

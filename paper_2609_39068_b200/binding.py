@@ -29,7 +29,8 @@ class SeParams(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H_q", ctypes.c_int32), ("H_kv", ctypes.c_int32),
                 ("D", ctypes.c_int32), ("page_size", ctypes.c_int32), ("max_pages", ctypes.c_int32),
                 ("num_phys_pages", ctypes.c_int32), ("k_max", ctypes.c_int32),
-                ("sm_scale", ctypes.c_float), ("flags", ctypes.c_uint32)]
+                ("sm_scale", ctypes.c_float), ("flags", ctypes.c_uint32),
+                ("sink_pages", ctypes.c_int32), ("recent_pages", ctypes.c_int32)]
 
 
 class SparseEngineError(RuntimeError):
@@ -94,8 +95,10 @@ def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_params(B, H_q, H_kv, D, max_pages, num_phys_pages, k_max, sm_scale=0.0, page_size=16) -> SeParams:
-    return SeParams(B, H_q, H_kv, D, page_size, max_pages, num_phys_pages, k_max, float(sm_scale), 0)
+def make_params(B, H_q, H_kv, D, max_pages, num_phys_pages, k_max, sm_scale=0.0, page_size=16,
+                sink_pages=0, recent_pages=0) -> SeParams:
+    return SeParams(B, H_q, H_kv, D, page_size, max_pages, num_phys_pages, k_max, float(sm_scale), 0,
+                    int(sink_pages), int(recent_pages))
 
 
 def se_version() -> int:
@@ -181,11 +184,13 @@ class DecodeState:
     """Buffers of one layer's decode step for a fixed shape: params, workspace, summaries,
     selection and outputs.  Convenience for tests, the smoke check and the benchmark."""
 
-    def __init__(self, w, k_max: Optional[int] = None, sm_scale: float = 0.0):
+    def __init__(self, w, k_max: Optional[int] = None, sm_scale: float = 0.0, sink_pages: int = 0,
+                 recent_pages: int = 0):
         dev = w.q.device
         self.w = w
-        self.k_max = int(k_max if k_max is not None else max(w.budget // 16, 1))
-        self.p = make_params(w.B, w.H_q, w.H_kv, w.D, w.max_pages, w.num_phys_pages, self.k_max, sm_scale)
+        self.k_max = int(k_max if k_max is not None else max(w.budget // 16 + sink_pages + recent_pages, 1))
+        self.p = make_params(w.B, w.H_q, w.H_kv, w.D, w.max_pages, w.num_phys_pages, self.k_max, sm_scale,
+                             sink_pages=sink_pages, recent_pages=recent_pages)
         self.workspace = alloc_workspace(self.p, dev)
         self.meta = torch.zeros((w.num_phys_pages, w.H_kv, 2, w.D), dtype=torch.bfloat16, device=dev)
         self.sel_idx = torch.full((w.B, w.H_kv, self.k_max), -7, dtype=torch.int32, device=dev)

@@ -23,6 +23,8 @@ int validate(const se_params *p) {
     if (p->max_pages < 1 || p->max_pages > 8192 || p->num_phys_pages < 1) return SE_ERR_INVALID_ARG;
     if (p->k_max < 1 || p->k_max > 4096) return SE_ERR_INVALID_ARG;
     if (p->flags != 0) return SE_ERR_INVALID_ARG;
+    if (p->sink_pages < 0 || p->recent_pages < 0 || p->sink_pages > 4096 || p->recent_pages > 4096)
+        return SE_ERR_INVALID_ARG;
     if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return SE_ERR_INVALID_ARG;
     // index arithmetic inside the kernels uses 32-bit page counts and 64-bit byte offsets
     if ((long long)p->B * p->H_kv > (1ll << 24)) return SE_ERR_INVALID_ARG;
@@ -144,7 +146,7 @@ int se_page_select(const se_params *p, const void *q, const void *meta, const in
         return SE_ERR_MISALIGNED;
     if (budget_tokens < kPage) return SE_ERR_INVALID_ARG;
     const int k_pages = budget_tokens / kPage;
-    if (k_pages > p->k_max) return SE_ERR_INVALID_ARG;
+    if (k_pages + p->sink_pages + p->recent_pages > p->k_max) return SE_ERR_INVALID_ARG;
     const WorkspaceLayout L = make_layout(*p);
     cudaError_t e = launch_page_select(*p, q, meta, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
                                        workspace, L, static_cast<cudaStream_t>(stream));

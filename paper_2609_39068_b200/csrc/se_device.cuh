@@ -101,6 +101,7 @@ __device__ __forceinline__ uint32_t f32_key(float f) {
 }
 
 constexpr uint32_t kKeyAbsent = 0x007fffffu;   // f32_key(-inf): below every finite score
+constexpr uint32_t kKeyForced = 0xffffffffu;   // marks a page that is selected regardless of its score
 
 // ---------------------------------------------------------------------------------
 // warp-level matrix helpers (bf16 inputs, fp32 accumulation)

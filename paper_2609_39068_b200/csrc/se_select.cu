@@ -335,10 +335,10 @@ __device__ __forceinline__ int warp_scan_inplace(int *a, int lane) {
 template <int KPT>
 __global__ void __launch_bounds__(kTopkThreads, KPT <= 16 ? 4 : 2)
 topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_lens, int H_kv,
-            int max_pages, int k_pages, int k_max, int32_t *__restrict__ sel_idx,
-            int32_t *__restrict__ sel_cnt) {
+            int max_pages, int k_pages, int k_max, int sink_pages, int recent_pages,
+            int32_t *__restrict__ sel_idx, int32_t *__restrict__ sel_cnt) {
     constexpr int ENTRIES = KPT * kTopkWarps;          // (tile, warp) cells of the compaction
-    __shared__ int s_red[3][kTopkWarps];
+    __shared__ int s_red[4][kTopkWarps];
     __shared__ int s_hist[2][256];
     __shared__ int s_cnt[2][ENTRIES];
     SE_TOPK_MARK(9);
@@ -348,6 +348,7 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     const int len = seq_lens[r];
     int n = len > 0 ? (len + kPage - 1) / kPage : 0;
     if (n > max_pages) n = max_pages;
+    const int n_full = n;                                     // pages the request's length spans
     if (n > KPT * kTopkThreads) n = KPT * kTopkThreads;       // cannot happen: the launcher picks KPT from max_pages
     const float *row = scores + (size_t)pair * max_pages;
     int32_t *out = sel_idx + (size_t)pair * k_max;
@@ -359,23 +360,28 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
         const int i = j * kTopkThreads + tid;
-        keys[j] = (i < n) ? f32_key(__ldg(row + i)) : kKeyAbsent;
+        uint32_t key = (i < n) ? f32_key(__ldg(row + i)) : kKeyAbsent;
+        // forced pages (sink / recent) leave the competition and are taken unconditionally
+        if (key != kKeyAbsent && (i < sink_pages || i >= n_full - recent_pages)) key = kKeyForced;
+        keys[j] = key;
     }
     SE_TOPK_MARK(0);
 
     // ---- present pages, and the range of their keys
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-    int present = 0;
+    int present = 0, forced = 0;          // candidates / forced pages
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const bool ok = keys[j] != kKeyAbsent;
+        const bool ok = keys[j] != kKeyAbsent && keys[j] != kKeyForced;
         present += ok;
+        forced += keys[j] == kKeyForced;
         kmin = ok ? min(kmin, keys[j]) : kmin;
         kmax = ok ? max(kmax, keys[j]) : kmax;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         present += __shfl_xor_sync(kFull, present, o);
+        forced += __shfl_xor_sync(kFull, forced, o);
         kmin = min(kmin, __shfl_xor_sync(kFull, kmin, o));
         kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
     }
@@ -383,17 +389,21 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
         s_red[0][warp] = present;
         s_red[1][warp] = (int)kmin;
         s_red[2][warp] = (int)kmax;
+        s_red[3][warp] = forced;
     }
     s_hist[0][tid] = 0;
     __syncthreads();
     present = 0;
+    forced = 0;
 #pragma unroll
     for (int w = 0; w < kTopkWarps; ++w) {
         present += s_red[0][w];
+        forced += s_red[3][w];
         kmin = min(kmin, (uint32_t)s_red[1][w]);
         kmax = max(kmax, (uint32_t)s_red[2][w]);
     }
-    const int k_eff = min(min(k_pages, k_max), present);
+    forced = min(forced, k_max);
+    const int k_eff = min(min(k_pages, k_max - forced), present);      // candidates to take
     SE_TOPK_MARK(1);
 
     // ---- radix select of the k_eff-th largest key.  All present keys share the bits above the
@@ -422,7 +432,8 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
                 for (int j = 0; j < KPT; ++j) {
                     if (j < tiles) {
                         const uint32_t key = keys[j];
-                        const bool active = key != kKeyAbsent && ((hi >= 32) || ((key >> hi) == (prefix >> hi)));
+                        const bool active = key != kKeyAbsent && key != kKeyForced &&
+                                            ((hi >= 32) || ((key >> hi) == (prefix >> hi)));
                         if (active) atomicAdd(&hist[(key >> shift) & ((1u << w) - 1u)], 1);
                     }
                 }
@@ -472,10 +483,14 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     }
     SE_TOPK_MARK(3);
 
-    if (k_eff == 0) {
+    if (k_eff + forced == 0) {
         for (int i = tid; i < k_max; i += kTopkThreads) out[i] = -1;
         if (tid == 0) sel_cnt[pair] = 0;
         return;
+    }
+    if (k_eff == 0) {             // only forced pages: nothing competes
+        ge_mode = true;
+        prefix = kKeyForced;
     }
     // ---- ordered compaction: keys > T are taken; keys == T are taken in page order until `need`
     // of them are in; in ge_mode every key >= T is taken.
@@ -483,8 +498,8 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     uint32_t takemask = 0, eqmask = 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const bool valid = keys[j] != kKeyAbsent;
-        const bool gt = valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T));
+        const bool valid = keys[j] != kKeyAbsent && keys[j] != kKeyForced;
+        const bool gt = (keys[j] == kKeyForced) || (valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T)));
         const bool eq = valid && !ge_mode && (keys[j] == T);
         takemask |= (uint32_t)gt << j;
         eqmask |= (uint32_t)eq << j;
@@ -520,8 +535,8 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
         }
     }
     SE_TOPK_MARK(4);
-    for (int i = k_eff + tid; i < k_max; i += kTopkThreads) out[i] = -1;
-    if (tid == 0) sel_cnt[pair] = k_eff;
+    for (int i = k_eff + forced + tid; i < k_max; i += kTopkThreads) out[i] = -1;
+    if (tid == 0) sel_cnt[pair] = k_eff + forced;
     SE_TOPK_MARK(5);
 }
 
@@ -564,7 +579,7 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     const int pairs = p.B * p.H_kv;
 #define SE_TOPK(KPT)                                                                                    \
     topk_kernel<KPT><<<pairs, kTopkThreads, 0, stream>>>(scores, seq_lens, p.H_kv, p.max_pages, k_pages, \
-                                                         p.k_max, sel_idx, sel_cnt)
+                                                         p.k_max, p.sink_pages, p.recent_pages, sel_idx, sel_cnt)
     if (p.max_pages <= 4 * kTopkThreads) SE_TOPK(4);
     else if (p.max_pages <= 8 * kTopkThreads) SE_TOPK(8);
     else if (p.max_pages <= 16 * kTopkThreads) SE_TOPK(16);
@@ -616,7 +631,8 @@ extern "C" int se_page_select_static(const se_params *p, const void *q, const vo
                            reinterpret_cast<uintptr_t>(page_table) | reinterpret_cast<uintptr_t>(seq_lens) |
                            reinterpret_cast<uintptr_t>(sel_idx) | reinterpret_cast<uintptr_t>(sel_cnt);
     if ((bits & 15u) || (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return SE_ERR_MISALIGNED;
-    if (budget_tokens < se::kPage || budget_tokens / se::kPage > p->k_max) return SE_ERR_INVALID_ARG;
+    if (budget_tokens < se::kPage || budget_tokens / se::kPage + p->sink_pages + p->recent_pages > p->k_max)
+        return SE_ERR_INVALID_ARG;
     // scratch layout: [status word, padded to 256 bytes][fp32 scores, B*H_kv*max_pages]
     const size_t need = 256 + (size_t)p->B * p->H_kv * p->max_pages * sizeof(float);
     if (need > SE_STATIC_SCRATCH_BYTES) return SE_ERR_SCRATCH_TOO_SMALL;

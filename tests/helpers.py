@@ -51,26 +51,39 @@ def dense_attention_np(qv, K, V, scale):
     return (e[:, None] * V).sum(0) / e.sum(), m + np.log(e.sum())
 
 
-def check_selection(sel_gpu, cnt_gpu, P_oracle, present, budget, p=16, rel_band=1e-5):
-    """Selected-page rule: with theta the oracle's k_eff-th largest score and
-    eps = rel_band*|theta|, the set must hold exactly k_eff distinct present pages,
-    every page scoring above theta+eps and none scoring below theta-eps.
+def check_selection(sel_gpu, cnt_gpu, P_oracle, present, budget, p=16, rel_band=1e-5,
+                    sink_pages=0, recent_pages=0, seq_lens=None):
+    """Selected-page rule.  Forced pages (first ``sink_pages`` / last ``recent_pages`` logical pages
+    of a request, when present) must all be in the set.  Among the other present pages, with theta
+    the oracle's k_eff-th largest score and eps = rel_band*|theta|, the set must hold exactly k_eff
+    of them, every page scoring above theta+eps and none scoring below theta-eps.
     Returns the number of (request, head) rows whose set differs from the strict top-k."""
     B, H, n = P_oracle.shape
     k = budget // p
     differing = 0
     for r in range(B):
-        cand = np.nonzero(present[r])[0]
+        pres = np.nonzero(present[r])[0]
+        n_r = n if seq_lens is None else (int(seq_lens[r]) + p - 1) // p
+        is_forced = (pres < sink_pages) | ((pres >= n_r - recent_pages) & (pres < n_r))
+        forced = set(pres[is_forced].tolist())
+        cand = pres[~is_forced]
         for h in range(H):
             k_eff = min(k, len(cand))
-            assert int(cnt_gpu[r, h]) == k_eff, (r, h, int(cnt_gpu[r, h]), k_eff)
+            total = k_eff + len(forced)
+            assert int(cnt_gpu[r, h]) == total, (r, h, int(cnt_gpu[r, h]), total)
             row = np.asarray(sel_gpu[r, h])
-            got = row[:k_eff]
-            assert np.all(row[k_eff:] == -1), "padding must be -1"
-            if k_eff == 0:
+            got = row[:total]
+            assert np.all(row[total:] == -1), "padding must be -1"
+            if total == 0:
                 continue
-            assert len(set(got.tolist())) == k_eff, "duplicate pages selected"
+            assert len(set(got.tolist())) == total, "duplicate pages selected"
             assert np.all(present[r][got]), "absent page selected"
+            gs = set(got.tolist())
+            assert forced <= gs, (r, h, "forced pages missing", sorted(forced - gs)[:5])
+            gs -= forced
+            if k_eff == 0:
+                assert not gs
+                continue
             s = P_oracle[r, h]
             order = cand[np.lexsort((cand, -s[cand]))]
             strict = set(order[:k_eff].tolist())
@@ -78,7 +91,6 @@ def check_selection(sel_gpu, cnt_gpu, P_oracle, present, budget, p=16, rel_band=
             eps = rel_band * abs(theta)
             must = set(cand[s[cand] > theta + eps].tolist())
             never = set(cand[s[cand] < theta - eps].tolist())
-            gs = set(got.tolist())
             assert must <= gs, (r, h, "missing pages above the band", sorted(must - gs)[:5])
             assert not (gs & never), (r, h, "pages below the band", sorted(gs & never)[:5])
             if gs != strict:

@@ -22,9 +22,9 @@ OUT_MEAN_ABS = 1e-3
 LSE_ABS = 1e-3
 
 
-def run_gpu(w_cpu, accum=False, incremental_after=None):
+def run_gpu(w_cpu, accum=False, sink_pages=0, recent_pages=0):
     w = w_cpu.to("cuda")
-    st = binding.DecodeState(w)
+    st = binding.DecodeState(w, sink_pages=sink_pages, recent_pages=recent_pages)
     st.rebuild_meta()
     st.select()
     u = w.score_accum.clone() if accum else None
@@ -34,7 +34,7 @@ def run_gpu(w_cpu, accum=False, incremental_after=None):
     return w, st, u
 
 
-def compare(w_cpu, st, rows=None, u_before=None, u_after=None, check_meta=True):
+def compare(w_cpu, st, rows=None, u_before=None, u_after=None, check_meta=True, sink_pages=0, recent_pages=0):
     a = host_arrays(w_cpu)
     rows = list(range(w_cpu.B)) if rows is None else list(rows)
     pt, sl, q = a["page_table"][rows], a["seq_lens"][rows], a["q"][rows]
@@ -47,7 +47,8 @@ def compare(w_cpu, st, rows=None, u_before=None, u_after=None, check_meta=True):
     S, P, present = oracle.quest_scores(q, meta_gpu, pt, sl)
     sel = st.sel_idx.cpu().numpy()[rows]
     cnt = st.sel_cnt.cpu().numpy()[rows]
-    differing = check_selection(sel, cnt, P, present, w_cpu.budget)
+    differing = check_selection(sel, cnt, P, present, w_cpu.budget, sink_pages=sink_pages,
+                                recent_pages=recent_pages, seq_lens=sl)
     assert differing <= max(1, (len(rows) * w_cpu.H_kv) // 4), "too many rows differ inside the tie band"
     for r in range(len(rows)):
         for h in range(w_cpu.H_kv):
@@ -111,6 +112,20 @@ def test_every_group_size(D, G):
                      poison_tail=True)
     w, st, _ = run_gpu(w_cpu)
     compare(w_cpu, st)
+
+
+@pytest.mark.parametrize("sink,recent,budget", [(4, 16, 256), (0, 3, 64), (2, 0, 32), (6, 6, 16 * 200), (3, 5, 16)])
+def test_forced_sink_and_recent_pages(sink, recent, budget):
+    """Sink and recent pages are read in addition to the selected budget."""
+    w_cpu = wl.build("forced", 825, 0, [2000, 50, 333, 16 * 4, 1], 8, 2, 128, budget, "cpu", permute_pool=True,
+                     prune_fraction=0.15, poison_tail=True)
+    w, st, _ = run_gpu(w_cpu, sink_pages=sink, recent_pages=recent)
+    compare(w_cpu, st, sink_pages=sink, recent_pages=recent)
+    # and the result is what the oracle selects, page for page, when no score is inside the band
+    a = host_arrays(w_cpu)
+    ref = oracle.decode_step(a["q"], a["k"], a["v"], a["page_table"], a["seq_lens"], budget,
+                             meta=wl.bf16_bits(st.meta), sink_pages=sink, recent_pages=recent)
+    assert np.array_equal(ref["sel_cnt"], st.sel_cnt.cpu().numpy())
 
 
 def test_all_pages_pruned_gives_empty_result():

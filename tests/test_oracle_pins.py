@@ -263,6 +263,33 @@ def test_topk_budget_rounds_down_to_pages():
     assert cnt[0, 0] == 3 and sel[0, 0, :3].tolist() == [7, 8, 9]
 
 
+def test_topk_forced_sink_and_recent_pages():
+    """The first `sink` and last `recent` pages are always in, outside the budget; the budget is
+    spent on the rest (brute force)."""
+    rng = np.random.default_rng(200)
+    B, H, n = 4, 2, 40
+    P = rng.standard_normal((B, H, n))
+    seq = np.array([16 * 40, 16 * 23 + 5, 16 * 3, 16 * 9 + 1])
+    n_pages = (seq + 15) // 16
+    present = np.zeros((B, n), bool)
+    for r in range(B):
+        present[r, :n_pages[r]] = rng.random(n_pages[r]) > 0.15
+    present[0, 0] = False                      # a pruned sink page is simply not there
+    for sink, recent, k in [(2, 3, 5), (0, 4, 2), (3, 0, 50), (4, 4, 1)]:
+        sel, cnt, theta = oracle.topk_pages(P, present, 16 * k, sink_pages=sink, recent_pages=recent,
+                                            seq_lens=seq, k_max=k + sink + recent)
+        for r in range(B):
+            pres = np.nonzero(present[r])[0]
+            forced = [b for b in pres if b < sink or b >= n_pages[r] - recent]
+            cand = [b for b in pres if b not in forced]
+            for h in range(H):
+                best = sorted(cand, key=lambda b: (-P[r, h, b], b))[:k]
+                want = sorted(forced + best)
+                assert cnt[r, h] == len(want)
+                assert sel[r, h, :len(want)].tolist() == want
+                assert np.all(sel[r, h, len(want):] == -1)
+
+
 # ---------------------------------------------------------------- O4 attention
 
 def sdpa_reference(w, a, r):
