@@ -298,8 +298,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
 #ifndef SE_TOPK_MARK
 #define SE_TOPK_MARK(i)          // hook for an external timing probe; empty in the library
 #endif
-constexpr int kTopkThreads = 256;
-constexpr int kTopkWarps = kTopkThreads / 32;
 
 // Exclusive prefix over `entries` (multiple of 32, <= 256) ints in shared memory, computed by the
 // calling warp alone and written back in place.  Every warp of the CTA may run it on the same
@@ -331,13 +329,15 @@ __device__ __forceinline__ int warp_scan_inplace(int *a, int lane) {
     return total;
 }
 
-// KPT = keys per thread held in registers (n <= 256*KPT, KPT in {4,8,16,32}).
-template <int KPT>
-__global__ void __launch_bounds__(kTopkThreads, KPT <= 16 ? 4 : 2)
+// kTopkThreads threads per CTA, KPT keys per thread held in registers (n <= kTopkThreads*KPT).
+template <int kTopkThreads, int KPT, bool kForced>
+__global__ void __launch_bounds__(kTopkThreads, (kTopkThreads * KPT <= 4096 && kTopkThreads <= 512) ? 1024 / kTopkThreads : 1)
 topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_lens, int H_kv,
             int max_pages, int k_pages, int k_max, int sink_pages, int recent_pages,
             int32_t *__restrict__ sel_idx, int32_t *__restrict__ sel_cnt) {
+    constexpr int kTopkWarps = kTopkThreads / 32;
     constexpr int ENTRIES = KPT * kTopkWarps;          // (tile, warp) cells of the compaction
+    static_assert(ENTRIES % 32 == 0 && ENTRIES <= 1024, "compaction cells");
     __shared__ int s_red[4][kTopkWarps];
     __shared__ int s_hist[2][256];
     __shared__ int s_cnt[2][ENTRIES];
@@ -362,7 +362,7 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
         const int i = j * kTopkThreads + tid;
         uint32_t key = (i < n) ? f32_key(__ldg(row + i)) : kKeyAbsent;
         // forced pages (sink / recent) leave the competition and are taken unconditionally
-        if (key != kKeyAbsent && (i < sink_pages || i >= n_full - recent_pages)) key = kKeyForced;
+        if (kForced && key != kKeyAbsent && (i < sink_pages || i >= n_full - recent_pages)) key = kKeyForced;
         keys[j] = key;
     }
     SE_TOPK_MARK(0);
@@ -372,9 +372,9 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     int present = 0, forced = 0;          // candidates / forced pages
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const bool ok = keys[j] != kKeyAbsent && keys[j] != kKeyForced;
+        const bool ok = keys[j] != kKeyAbsent && (!kForced || keys[j] != kKeyForced);
         present += ok;
-        forced += keys[j] == kKeyForced;
+        if (kForced) forced += keys[j] == kKeyForced;
         kmin = ok ? min(kmin, keys[j]) : kmin;
         kmax = ok ? max(kmax, keys[j]) : kmax;
     }
@@ -391,7 +391,7 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
         s_red[2][warp] = (int)kmax;
         s_red[3][warp] = forced;
     }
-    s_hist[0][tid] = 0;
+    if (tid < 256) s_hist[0][tid] = 0;
     __syncthreads();
     present = 0;
     forced = 0;
@@ -432,12 +432,12 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
                 for (int j = 0; j < KPT; ++j) {
                     if (j < tiles) {
                         const uint32_t key = keys[j];
-                        const bool active = key != kKeyAbsent && key != kKeyForced &&
+                        const bool active = key != kKeyAbsent && (!kForced || key != kKeyForced) &&
                                             ((hi >= 32) || ((key >> hi) == (prefix >> hi)));
                         if (active) atomicAdd(&hist[(key >> shift) & ((1u << w) - 1u)], 1);
                     }
                 }
-                s_hist[par ^ 1][tid] = 0;            // the other buffer serves the next digit
+                if (tid < 256) s_hist[par ^ 1][tid] = 0;   // the other buffer serves the next digit
                 __syncthreads();
                 // every warp finds the digit d with  #(digits > d) < remaining <= #(digits >= d)
                 // on its own: lane l owns digits 8l..8l+7, higher lanes hold higher digits
@@ -498,8 +498,8 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     uint32_t takemask = 0, eqmask = 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const bool valid = keys[j] != kKeyAbsent && keys[j] != kKeyForced;
-        const bool gt = (keys[j] == kKeyForced) || (valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T)));
+        const bool valid = keys[j] != kKeyAbsent && (!kForced || keys[j] != kKeyForced);
+        const bool gt = (kForced && keys[j] == kKeyForced) || (valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T)));
         const bool eq = valid && !ge_mode && (keys[j] == T);
         takemask |= (uint32_t)gt << j;
         eqmask |= (uint32_t)eq << j;
@@ -577,13 +577,21 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
                         : launch_score<64>(p, q, meta, page_table, seq_lens, scores, status, stream);
     if (e != cudaSuccess) return e;
     const int pairs = p.B * p.H_kv;
-#define SE_TOPK(KPT)                                                                                    \
-    topk_kernel<KPT><<<pairs, kTopkThreads, 0, stream>>>(scores, seq_lens, p.H_kv, p.max_pages, k_pages, \
-                                                         p.k_max, p.sink_pages, p.recent_pages, sel_idx, sel_cnt)
-    if (p.max_pages <= 4 * kTopkThreads) SE_TOPK(4);
-    else if (p.max_pages <= 8 * kTopkThreads) SE_TOPK(8);
-    else if (p.max_pages <= 16 * kTopkThreads) SE_TOPK(16);
-    else SE_TOPK(32);
+#define SE_TOPK(THREADS, KPT)                                                                         \
+    do {                                                                                              \
+        if (p.sink_pages || p.recent_pages)                                                           \
+            topk_kernel<THREADS, KPT, true><<<pairs, THREADS, 0, stream>>>(                           \
+                scores, seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, p.sink_pages, p.recent_pages, \
+                sel_idx, sel_cnt);                                                                    \
+        else                                                                                          \
+            topk_kernel<THREADS, KPT, false><<<pairs, THREADS, 0, stream>>>(                          \
+                scores, seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, 0, 0, sel_idx, sel_cnt);     \
+    } while (0)
+    // short requests: fewer keys per thread; long ones: more threads, so the per-thread chains stay short
+    if (p.max_pages <= 1024) SE_TOPK(256, 4);
+    else if (p.max_pages <= 2048) SE_TOPK(256, 8);
+    else if (p.max_pages <= 4096) SE_TOPK(256, 16);
+    else SE_TOPK(1024, 8);
 #undef SE_TOPK
     return cudaGetLastError();
 }
