@@ -101,7 +101,7 @@ const char *se_strerror(int code);
 size_t se_workspace_bytes(const se_params *p);
 
 /*
- * Zeroes the control block (completion counters, status word) at the head of the
+ * Zeroes the control block (status word, work-queue counters) at the head of the
  * workspace.  Required once after allocation; the kernels leave the counters at zero
  * when they finish, so it need not be repeated.
  */
@@ -156,8 +156,8 @@ int se_page_select(const se_params *p, const void *q, const void *meta,
  *     z_j = sm_scale * q.k_j,  alpha_j = exp(z_j)/sum_{u in T} exp(z_u),
  *     out = sum_j alpha_j v_j,  lse = ln sum_{u in T} exp(z_u).
  * The selected pages are split over several workers (split-K) whose partial results are
- * merged through their running maxima; out/lse do not depend on the split beyond fp32
- * rounding.  An empty T gives out = 0 and lse = -inf.
+ * merged through their running maxima by a second kernel; out/lse do not depend on the split
+ * beyond fp32 rounding.  An empty T gives out = 0 and lse = -inf.
  * score_accum != NULL additionally applies the H2O update (Appendix A, H2O accumulated
  * score equation) to every attended token slot:
  *     score_accum[pid,h,t] += sum over the query heads a of group h of alpha_{a,(pid,t)} .

@@ -14,12 +14,13 @@
 //                    O[head, :]      += P[head, token] . V[token, :]    (P split into two bf16 terms)
 //                The accumulator layout of S^T is the A-operand layout of P, so the
 //                probabilities never leave registers.  A warp that holds all pages of a pair
-//                writes out/lse itself; otherwise it stores a partial (acc, m, l) and the warp
-//                that finishes last merges them (an atomic ticket, no waiting).
+//                writes out/lse itself; otherwise it stores a partial (acc, m, l).
 //                An earlier plain-FMA version of this kernel needed ~1050 warp instructions per
 //                page (8 KB) and was issue-bound at 65 % of the copy bandwidth.
-// h2o_kernel     adds exp(z - lse), summed over the query heads of the kv-head, to the
-//                accumulated score of every attended token slot.
+// combine_kernel merges the split partials of every pair (one warp per query head, so the
+//                merge of many splits is spread wide instead of falling on one warp) and adds
+//                exp(z - lse), summed over the query heads of the kv-head, to the accumulated
+//                score of every attended token slot (the H2O epilogue).
 #include <cuda.h>
 
 #include "se_internal.h"
@@ -81,7 +82,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
               const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
               const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ sel_idx,
               const int32_t *__restrict__ sel_cnt, float *__restrict__ out, float *__restrict__ lse,
-              float *__restrict__ partials, uint32_t *__restrict__ tickets, float *__restrict__ zbuf,
+              float *__restrict__ partials, float *__restrict__ zbuf,
               int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
               int max_splits, float scale_log2, uint32_t *status) {
     using C = DecCfg<D>;
@@ -381,7 +382,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             continue;
         }
 
-        // ---- store the partial, take a ticket, the last one merges
+        // ---- store the partial; combine_kernel merges the splits of a pair afterwards
         if (head_ok) {
             float *pr = partials + (((size_t)r * H_q + h * G + gid) * max_splits + my_split) * C::PSTRIDE;
 #pragma unroll
@@ -391,75 +392,6 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 pr[D] = m_run;
                 pr[D + 1] = l_run;
             }
-        }
-        __threadfence();
-        __syncwarp();
-        unsigned old = 0;
-        if (lane == 0) old = atomicAdd(&tickets[pair], 1u);
-        old = __shfl_sync(kFull, old, 0);
-        if ((int)old != n_split - 1) continue;
-        __threadfence();
-        if (lane == 0) tickets[pair] = 0u;                 // ready for the next launch
-        // Merge: lane s first fetches (m_s, l_s) of split s for every head (all loads in flight
-        // together), the weights follow from warp reductions, then the accumulators are summed
-        // with each lane owning four channels.  More than 32 splits are folded block by block.
-        const float *pr0 = partials + (((size_t)r * H_q + h * G) * max_splits) * C::PSTRIDE;
-        float mg[8], lg[8], og[8][4];
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            mg[g] = -INFINITY;
-            lg[g] = 0.f;
-            og[g][0] = og[g][1] = og[g][2] = og[g][3] = 0.f;
-        }
-        for (int s0 = 0; s0 < n_split; s0 += 32) {
-            const int ns = min(32, n_split - s0);
-            float ms[8], ls[8];
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                ms[g] = -INFINITY;
-                ls[g] = 0.f;
-                if (g < G && lane < ns) {
-                    const float *pp = pr0 + ((size_t)g * max_splits + s0 + lane) * C::PSTRIDE + D;
-                    ms[g] = __ldcg(pp);
-                    ls[g] = __ldcg(pp + 1);
-                }
-            }
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                if (g >= G) continue;
-                float mb = ms[g];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(kFull, mb, o));
-                const float m_new = fmaxf(mg[g], mb);
-                const float wl = (ms[g] == -INFINITY) ? 0.f : exp2f(ms[g] - m_new);    // weight of split s0+lane
-                float lb = wl * ls[g];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) lb += __shfl_xor_sync(kFull, lb, o);
-                const float keep = (mg[g] == -INFINITY) ? 0.f : exp2f(mg[g] - m_new);
-                lg[g] = lg[g] * keep + lb;
-                og[g][0] *= keep; og[g][1] *= keep; og[g][2] *= keep; og[g][3] *= keep;
-                mg[g] = m_new;
-                const float *pa = pr0 + ((size_t)g * max_splits + s0) * C::PSTRIDE;
-#pragma unroll 4
-                for (int s = 0; s < ns; ++s) {
-                    const float ws = __shfl_sync(kFull, wl, s);
-                    if (lane * 4 < D) {
-                        const float4 a = __ldcg(reinterpret_cast<const float4 *>(pa + (size_t)s * C::PSTRIDE) + lane);
-                        og[g][0] += ws * a.x; og[g][1] += ws * a.y; og[g][2] += ws * a.z; og[g][3] += ws * a.w;
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            if (g >= G) continue;
-            const float inv = lg[g] > 0.f ? 1.f / lg[g] : 0.f;
-            if (lane * 4 < D) {
-                float4 *dst = reinterpret_cast<float4 *>(out + ((size_t)r * H_q + h * G + g) * D) + lane;
-                *dst = make_float4(og[g][0] * inv, og[g][1] * inv, og[g][2] * inv, og[g][3] * inv);
-            }
-            if (lane == 0)
-                lse[(size_t)r * H_q + h * G + g] = lg[g] > 0.f ? (mg[g] + log2f(lg[g])) * kLn2 : -INFINITY;
         }
     }
     SE_PROF_LAP(3)
@@ -471,34 +403,104 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     }
 }
 
-// score_accum[pid,h,t] += sum_g exp2(z2[g] - lse[g]*log2e) for every attended token slot.
+// combine_kernel: one CTA per (request, kv-head) pair, one warp per query head of the group.
+//   1. LSE merge of the pair's split partials (skipped when the pair had a single split, whose
+//      warp already wrote out/lse): m* = max_s m_s, L = sum_s 2^(m_s-m*) l_s,
+//      out = sum_s 2^(m_s-m*) acc_s / L, lse = (m* + log2 L) ln 2.  Lane s fetches (m_s, l_s),
+//      the weights follow from warp reductions, then each lane sums four channels with the
+//      loads of eight splits in flight together.
+//   2. H2O epilogue (zbuf != NULL): score_accum[pid,h,t] += sum_g 2^(z2[g] - lse_g*log2e) for
+//      every attended token slot of the pair.  The slots of a pair are spread over gridDim.y
+//      CTAs; each of them recomputes the pair's lse (the cheap half of the merge), only
+//      blockIdx.y == 0 sums the accumulators and writes out/lse.
+template <int D>
 __global__ void __launch_bounds__(256)
-h2o_kernel(const float *__restrict__ zbuf, const float *__restrict__ lse, const int32_t *__restrict__ page_table,
-           const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ sel_idx,
-           const int32_t *__restrict__ sel_cnt, float *__restrict__ score_accum, int B, int H_kv, int G, int GP,
-           int max_pages, int P_phys, int k_max) {
-    const long long total = (long long)B * H_kv * k_max * kPage;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
-         e += (long long)gridDim.x * blockDim.x) {
-        const int t = (int)(e % kPage);
-        const long long slot = e / kPage;
-        const int i = (int)(slot % k_max);
-        const int pair = (int)(slot / k_max);
-        const int r = pair / H_kv, h = pair % H_kv;
-        if (i >= min(sel_cnt[pair], k_max)) continue;
-        const int len = seq_lens[r];
-        const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
+combine_kernel(const float *__restrict__ partials, const float *__restrict__ zbuf,
+               const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
+               const int32_t *__restrict__ sel_idx, const int32_t *__restrict__ sel_cnt,
+               float *__restrict__ out, float *__restrict__ lse, float *__restrict__ score_accum,
+               int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
+               int max_splits) {
+    constexpr int PSTRIDE = D + 4;
+    __shared__ float s_lse2[8];
+    const int pair = blockIdx.x;
+    const int r = pair / H_kv, h = pair % H_kv;
+    const int H_q = H_kv * G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cnt = min(sel_cnt[pair], k_max);
+    const int len = seq_lens[r];
+    const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
+    const bool nothing = cnt <= 0 || n_r == 0;
+    const int n_split = nothing ? 0 : (cnt + pages_per_split - 1) / pages_per_split;
+    const int g = warp;                               // query head of the group handled by this warp
+    const bool writer = blockIdx.y == 0;
+    if (g < G) {
+        const size_t head = (size_t)r * H_q + h * G + g;
+        if (n_split > 1) {
+            const float *pr0 = partials + head * max_splits * PSTRIDE;
+            float mg = -INFINITY, lg = 0.f;
+            float4 og = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s0 = 0; s0 < n_split; s0 += 32) {
+                const int ns = min(32, n_split - s0);
+                float ms = -INFINITY, ls = 0.f;
+                if (lane < ns) {
+                    ms = __ldcg(pr0 + (size_t)(s0 + lane) * PSTRIDE + D);
+                    ls = __ldcg(pr0 + (size_t)(s0 + lane) * PSTRIDE + D + 1);
+                }
+                float mb = ms;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(kFull, mb, o));
+                const float m_new = fmaxf(mg, mb);
+                const float wl = (ms == -INFINITY) ? 0.f : exp2f(ms - m_new);      // weight of split s0+lane
+                float lb = wl * ls;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) lb += __shfl_xor_sync(kFull, lb, o);
+                const float keep = (mg == -INFINITY) ? 0.f : exp2f(mg - m_new);
+                lg = lg * keep + lb;
+                og.x *= keep; og.y *= keep; og.z *= keep; og.w *= keep;
+                mg = m_new;
+                if (!writer) continue;                    // the other CTAs of the pair only need the lse
+                for (int s = 0; s < ns; s += 8) {
+                    float4 a[8];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        a[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (s + t < ns && lane * 4 < D)
+                            a[t] = __ldcg(reinterpret_cast<const float4 *>(pr0 + (size_t)(s0 + s + t) * PSTRIDE) + lane);
+                    }
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        const float ws = __shfl_sync(kFull, wl, (s + t) & 31);
+                        og.x += ws * a[t].x; og.y += ws * a[t].y; og.z += ws * a[t].z; og.w += ws * a[t].w;
+                    }
+                }
+            }
+            const float inv = lg > 0.f ? 1.f / lg : 0.f;
+            if (writer && lane * 4 < D)
+                reinterpret_cast<float4 *>(out + head * D)[lane] = make_float4(og.x * inv, og.y * inv, og.z * inv, og.w * inv);
+            const float l2 = lg > 0.f ? mg + log2f(lg) : -INFINITY;
+            if (lane == 0) {
+                if (writer) lse[head] = l2 * kLn2;
+                s_lse2[g] = l2;
+            }
+        } else if (lane == 0) {
+            s_lse2[g] = lse[head] * kLog2e;           // written by the decode kernel (single split / nothing)
+        }
+    }
+    if (zbuf == nullptr || nothing) return;
+    __syncthreads();
+    for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < cnt * kPage; e += gridDim.y * blockDim.x) {
+        const int i = e / kPage, t = e % kPage;
         const int b = sel_idx[(size_t)pair * k_max + i];
         if (b < 0 || b >= n_r) continue;
         const int pid = page_table[(size_t)r * max_pages + b];
         if (pid < 0 || pid >= P_phys) continue;
         if (t >= min(kPage, len - b * kPage)) continue;
-        const float *z = zbuf + (size_t)e * GP;
+        const float *z = zbuf + (((size_t)pair * k_max + i) * kPage + t) * GP;
         float add = 0.f;
-        for (int g = 0; g < G; ++g) {
-            const float l2 = lse[(size_t)r * (H_kv * G) + h * G + g] * kLog2e;
-            const float zz = z[g];
-            if (zz != -INFINITY) add += exp2f(zz - l2);
+        for (int gg = 0; gg < G; ++gg) {
+            const float zz = z[gg];
+            if (zz != -INFINITY) add += exp2f(zz - s_lse2[gg]);
         }
         score_accum[((size_t)pid * H_kv + h) * kPage + t] += add;
     }
@@ -554,18 +556,18 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     float *zbuf = score_accum ? reinterpret_cast<float *>(ws + L.zbuf) : nullptr;
     kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
         k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-        reinterpret_cast<float *>(ws + L.partials), reinterpret_cast<uint32_t *>(ws + L.dec_tickets), zbuf,
+        reinterpret_cast<float *>(ws + L.partials), zbuf,
         p.B, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
         effective_scale(p) * kLog2e, reinterpret_cast<uint32_t *>(ws + L.status));
     e = cudaGetLastError();
-    if (e != cudaSuccess || !score_accum) return e;
-    const long long total = (long long)p.B * p.H_kv * p.k_max * kPage;
-    long long blocks = (total + 255) / 256;
-    const long long cap = (long long)device_sm_count() * 8;
-    if (blocks > cap) blocks = cap;
-    h2o_kernel<<<(unsigned)blocks, 256, 0, stream>>>(zbuf, lse, page_table, seq_lens, sel_idx, sel_cnt,
-                                                     score_accum, p.B, p.H_kv, G, GP, p.max_pages,
-                                                     p.num_phys_pages, p.k_max);
+    if (e != cudaSuccess) return e;
+    if (plan.max_splits == 1 && !score_accum) return e;       // every pair is written by one warp
+    // with the H2O epilogue the token slots of a pair (16 per selected page) are spread over
+    // several CTAs, two slots per thread
+    const int slot_ctas = score_accum ? (p.k_max * kPage + 511) / 512 : 1;
+    combine_kernel<D><<<dim3(p.B * p.H_kv, slot_ctas), 256, 0, stream>>>(
+        reinterpret_cast<const float *>(ws + L.partials), zbuf, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
+        score_accum, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits);
     return cudaGetLastError();
 }
 

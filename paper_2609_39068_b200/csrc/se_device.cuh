@@ -17,9 +17,7 @@ constexpr unsigned kFull = 0xffffffffu;
 // from the workspace base, each a multiple of 256).
 // ---------------------------------------------------------------------------------
 struct WorkspaceLayout {
-    size_t status;          // uint32 status word (+ padding)
-    size_t sel_tickets;     // uint32 [B*H_kv]   chunks of a (request, head) pair scored so far
-    size_t dec_tickets;     // uint32 [B*H_kv]   splits of a pair finished so far
+    size_t status;          // 256 bytes: uint32 status word, work-queue counters of the score kernel
     size_t scores;          // float  [B*H_kv*max_pages]
     size_t partials;        // float  [B*H_q*max_splits*(D+2)]
     size_t zbuf;            // float  [B*H_kv*k_max*16*G]  logits kept for the H2O epilogue
