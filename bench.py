@@ -2,9 +2,10 @@
 """Benchmark of the sparse decode-attention hot path.
 
 A *step* is one pass of the whole path over one batch of synthetic requests, per layer:
-``se_meta_update`` (summary of the page holding each request's newest token) ->
-``se_page_select`` (page scores + top-k) -> ``se_sparse_decode`` (split-K attention over the
-selected pages, LSE merge, optional H2O statistic).  The default workload is the
+summary of the page holding each request's newest token -> page scores + top-k
+(``se_page_select_fused`` does both; ``se_meta_update`` + ``se_page_select`` are the separate
+calls) -> ``se_sparse_decode`` (split-K attention over the selected pages, LSE merge, optional
+H2O statistic).  The default workload is the
 continuous-batching mix (config 3: 64 requests, 4096..65536 tokens, 32/8 heads, D=128,
 budget 2048, page tables permuted over one pool); ``--config`` picks another one.
 
@@ -330,6 +331,7 @@ def main():
     call_us = {
         "se_meta_update": time_call(st0.update_meta, iters),
         "se_page_select": time_call(st0.select, iters),
+        "se_page_select_fused": time_call(st0.select_fused, iters),
         "se_sparse_decode": time_call(lambda: st0.decode(u0), iters),
     }
     b0 = bytes_l[0]
@@ -383,7 +385,7 @@ def main():
             cpu_baseline["sample"] += "; one layer timed, x%d layers" % n_layers
 
     if rank == 0:
-        launches_per_step = n_layers * (5 if h2o else 4)
+        launches_per_step = n_layers * 4        # score, top-k, decode, combine (summary update fused into score)
         line = {
             "metric": METRIC, "value": ms_per_step * 1e3, "unit": "us", "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": ms_per_step,

@@ -150,6 +150,21 @@ int se_page_select(const se_params *p, const void *q, const void *meta,
                    void *workspace, void *stream);
 
 /*
+ * se_meta_update(first_tok = NULL) and se_page_select in one call (the decode step's usual order:
+ * the newest token's K is in the cache, its page's summary is stale).  The scoring kernel recomputes
+ * the summary of the page that holds each request's newest token from k_cache - for every
+ * kv-head, over the tokens below the length, exactly as se_meta_update does - uses it for the
+ * score and writes it to `meta`; every other page's summary is read from `meta` as usual.  Saves
+ * the separate kernel of se_meta_update.  Results (meta, sel_idx, sel_cnt) are identical to the
+ * two calls made one after the other.  (Quest summary and score equations, TopK; "new keys update
+ * the extrema of their pages".)
+ */
+int se_page_select_fused(const se_params *p, const void *q, const void *k_cache, void *meta,
+                         const int32_t *page_table, const int32_t *seq_lens,
+                         int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
+                         void *workspace, void *stream);
+
+/*
  * Attention over the tokens of the selected pages (Appendix A, "Attention over Selected
  * Positions"): for every query head a of request r, with T the tokens (below len_r) of
  * the pages sel_idx[r, a/G, 0..sel_cnt),

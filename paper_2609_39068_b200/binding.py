@@ -21,7 +21,8 @@ SE_DEV_BAD_SELECTION = 2
 SE_DEV_WAIT_TIMEOUT = 4
 
 EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_workspace_init", "se_meta_update",
-           "se_page_select", "se_sparse_decode", "se_last_device_status", "se_page_select_static")
+           "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_last_device_status",
+           "se_page_select_static")
 SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -64,11 +65,12 @@ def load(build_if_missing: bool = True):
     lib.se_workspace_init.argtypes = [pp, vp, vp]
     lib.se_meta_update.argtypes = [pp, vp, i32p, i32p, i32p, vp, vp]
     lib.se_page_select.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
+    lib.se_page_select_fused.argtypes = [pp, vp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_sparse_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, fp, fp, fp, vp, vp]
     lib.se_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
-    for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_sparse_decode",
-                 "se_last_device_status", "se_page_select_static"):
+    for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
+                 "se_sparse_decode", "se_last_device_status", "se_page_select_static"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -145,6 +147,19 @@ def se_page_select(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel
                                  _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_page_select")
 
 
+def se_page_select_fused(p, q, k_cache, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,
+                         workspace) -> None:
+    _check(load().se_page_select_fused(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                       _ptr(k_cache, torch.bfloat16, "k_cache"),
+                                       _ptr(meta, torch.bfloat16, "meta"),
+                                       _ptr(page_table, torch.int32, "page_table"),
+                                       _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens),
+                                       _ptr(sel_idx, torch.int32, "sel_idx"),
+                                       _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                       _ptr(workspace, torch.uint8, "workspace"), _stream()),
+           "se_page_select_fused")
+
+
 def se_sparse_decode(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
                      workspace, score_accum=None) -> None:
     _check(load().se_sparse_decode(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
@@ -214,10 +229,19 @@ class DecodeState:
                          self.w.seq_lens, self.sel_idx, self.sel_cnt, self.out, self.lse,
                          self.workspace, score_accum=score_accum)
 
-    def step(self, score_accum=None):
-        """One decode step of the layer: newest-page summary, selection, attention."""
-        self.update_meta()
-        self.select()
+    def select_fused(self, budget: Optional[int] = None):
+        se_page_select_fused(self.p, self.w.q, self.w.k_cache, self.meta, self.w.page_table, self.w.seq_lens,
+                             self.w.budget if budget is None else budget, self.sel_idx, self.sel_cnt,
+                             self.workspace)
+
+    def step(self, score_accum=None, fused: bool = True):
+        """One decode step of the layer: newest-page summary, selection, attention.  ``fused``
+        folds the summary update into the scoring kernel (se_page_select_fused)."""
+        if fused:
+            self.select_fused()
+        else:
+            self.update_meta()
+            self.select()
         self.decode(score_accum)
 
     def status(self) -> int:

@@ -146,7 +146,26 @@ int se_page_select(const se_params *p, const void *q, const void *meta, const in
     const int k_pages = budget_tokens / kPage;
     if (k_pages + p->sink_pages + p->recent_pages > p->k_max) return SE_ERR_INVALID_ARG;
     const WorkspaceLayout L = make_layout(*p);
-    cudaError_t e = launch_page_select(*p, q, meta, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
+    cudaError_t e = launch_page_select(*p, q, meta, nullptr, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
+                                       workspace, L, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_page_select_fused(const se_params *p, const void *q, const void *k_cache, void *meta,
+                         const int32_t *page_table, const int32_t *seq_lens, int32_t budget_tokens,
+                         int32_t *sel_idx, int32_t *sel_cnt, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!q || !k_cache || !meta || !page_table || !seq_lens || !sel_idx || !sel_cnt || !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(meta) || !aligned16(page_table) ||
+        !aligned16(seq_lens) || !aligned16(sel_idx) || !aligned16(sel_cnt) || !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    if (budget_tokens < kPage) return SE_ERR_INVALID_ARG;
+    const int k_pages = budget_tokens / kPage;
+    if (k_pages + p->sink_pages + p->recent_pages > p->k_max) return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_page_select(*p, q, meta, k_cache, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
                                        workspace, L, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
 }

@@ -2,6 +2,7 @@
 // with bounded waits, bf16 unpacking, packed fp32 FMA, and the transposing warp reduction.
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -90,6 +91,16 @@ __device__ __forceinline__ float2 bf16x2_to_f2(uint32_t w) {
 
 __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
     return __ffma2_rn(a, b, c);
+}
+
+// min / max of two packed bf16 pairs (exact; -0 orders below +0)
+__device__ __forceinline__ uint32_t bmin2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&r);
+}
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&r);
 }
 
 // Order-preserving map fp32 -> uint32 (larger float <=> larger key).

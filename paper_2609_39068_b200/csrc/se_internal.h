@@ -27,7 +27,9 @@ cudaError_t launch_meta_update(const se_params &p, const void *k_cache, const in
                                const int32_t *seq_lens, const int32_t *first_tok, void *meta,
                                cudaStream_t stream);
 
-cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta,
+// k_cache != nullptr: the summary of the page holding each request's newest token is recomputed
+// from K inside the scoring kernel (and written back to `meta`) instead of being read
+cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta, const void *k_cache,
                                const int32_t *page_table, const int32_t *seq_lens, int k_pages,
                                int32_t *sel_idx, int32_t *sel_cnt, void *workspace,
                                const WorkspaceLayout &L, cudaStream_t stream);

@@ -4,22 +4,11 @@
 // One warp per (request, logical page, kv-head).  A K page of one head is a contiguous
 // [16, D] bf16 tile; a row is read with 16-byte loads by D/8 lanes, several rows per warp
 // pass, and the row groups are folded with shuffles.  min/max of bf16 pairs is exact.
-#include <cuda_bf16.h>
-
 #include "se_internal.h"
 
 namespace se {
 
 namespace {
-
-__device__ __forceinline__ uint32_t bmin2(uint32_t a, uint32_t b) {
-    __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
-    return *reinterpret_cast<uint32_t *>(&r);
-}
-__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
-    __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
-    return *reinterpret_cast<uint32_t *>(&r);
-}
 
 template <int D>
 __global__ void __launch_bounds__(256)

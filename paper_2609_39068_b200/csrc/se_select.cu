@@ -39,13 +39,14 @@ struct ScoreCfg {
 
 struct Batch {
     int r, h, b0, n_r;      // request, kv-head, first logical page, pages of the request
+    int len;                // tokens of the request
     int unit;               // flat unit index this batch belongs to (-1 = end of stream)
     int k;                  // batch number inside the unit
 };
 
 // Flat unit u -> (request, head, first page); prefix[r] = units before request r.
 __device__ __forceinline__ bool decode_unit(int u, int total_units, const int *prefix, const int *npages,
-                                            int B, int H_kv, Batch &d) {
+                                            const int *lens, int B, int H_kv, Batch &d) {
     if (u >= total_units) {
         d.unit = -1;
         return false;
@@ -60,6 +61,7 @@ __device__ __forceinline__ bool decode_unit(int u, int total_units, const int *p
     d.h = local % H_kv;
     d.b0 = (local / H_kv) * kUnitPages;
     d.n_r = npages[lo];
+    d.len = lens[lo];
     d.unit = u;
     d.k = 0;
     return true;
@@ -67,17 +69,18 @@ __device__ __forceinline__ bool decode_unit(int u, int total_units, const int *p
 
 template <int D>
 __global__ void __launch_bounds__(kScoreWarps * 32)
-score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
-             const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
+score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t *__restrict__ k_cache,
+             uint8_t *meta_out, const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
              float *__restrict__ scores, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
              uint32_t *status) {
     using C = ScoreCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    // layout: [buffers: warps*2*BUF] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints]
+    // layout: [buffers: warps*2*BUF] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints] [lens: B ints]
     uint8_t *bufs = smem_raw;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)kScoreWarps * 2 * C::BUF);
     int *prefix = reinterpret_cast<int *>(bars + kScoreWarps * 2);
     int *npages = prefix + (B + 1);
+    int *lens = npages + B;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int H_q = H_kv * G;
@@ -93,6 +96,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
                 n = len > 0 ? (len + kPage - 1) / kPage : 0;
                 if (n > max_pages) n = max_pages;
                 npages[r] = n;
+                lens[r] = len;
             }
             int u = ((n + kUnitPages - 1) / kUnitPages) * H_kv;
             int inc = u;
@@ -166,7 +170,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
             return;
         }
         const int u = __shfl_sync(kFull, pending_unit, 0);
-        if (decode_unit(u, total_units, prefix, npages, B, H_kv, d)) request_unit();
+        if (decode_unit(u, total_units, prefix, npages, lens, B, H_kv, d)) request_unit();
     };
     // every warp checks out once; the last one leaves the counters at zero for the next launch
     auto check_out = [&]() {
@@ -187,27 +191,70 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ meta,
             pid = __ldg(page_table + (size_t)d.r * max_pages + d.b0 + lane);
         return pid;
     };
+    // Summary of one K page computed on the spot (fused summary update): the page that holds the
+    // request's newest token may have changed since its summary was stored, so, when the caller
+    // hands in the K cache, that one page per (request, head) is summarised from K here - written
+    // to the summary array and straight into the batch buffer - instead of being copied.
+    auto summarise_page = [&](int pid, int h, int nv, uint32_t dst_smem) {
+        constexpr int LPR = D / 8;           // lanes per token row (16-byte pieces)
+        constexpr int TPP = 32 / LPR;        // token rows per warp pass
+        const int tg = lane / LPR, lr = lane % LPR;
+        const uint4 *kp = reinterpret_cast<const uint4 *>(k_cache) + ((size_t)pid * H_kv + h) * (kPage * D / 8);
+        uint4 mn = make_uint4(0x7f807f80u, 0x7f807f80u, 0x7f807f80u, 0x7f807f80u);   // +inf pairs
+        uint4 mx = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // -inf pairs
+#pragma unroll
+        for (int i = 0; i < kPage / TPP; ++i) {
+            const int t = i * TPP + tg;
+            if (t < nv) {
+                const uint4 w = __ldg(kp + t * LPR + lr);
+                mn.x = bmin2(mn.x, w.x); mn.y = bmin2(mn.y, w.y); mn.z = bmin2(mn.z, w.z); mn.w = bmin2(mn.w, w.w);
+                mx.x = bmax2(mx.x, w.x); mx.y = bmax2(mx.y, w.y); mx.z = bmax2(mx.z, w.z); mx.w = bmax2(mx.w, w.w);
+            }
+        }
+#pragma unroll
+        for (int m = LPR; m < 32; m <<= 1) {
+            mn.x = bmin2(mn.x, __shfl_xor_sync(kFull, mn.x, m)); mn.y = bmin2(mn.y, __shfl_xor_sync(kFull, mn.y, m));
+            mn.z = bmin2(mn.z, __shfl_xor_sync(kFull, mn.z, m)); mn.w = bmin2(mn.w, __shfl_xor_sync(kFull, mn.w, m));
+            mx.x = bmax2(mx.x, __shfl_xor_sync(kFull, mx.x, m)); mx.y = bmax2(mx.y, __shfl_xor_sync(kFull, mx.y, m));
+            mx.z = bmax2(mx.z, __shfl_xor_sync(kFull, mx.z, m)); mx.w = bmax2(mx.w, __shfl_xor_sync(kFull, mx.w, m));
+        }
+        uint4 *gp = reinterpret_cast<uint4 *>(meta_out) + ((size_t)pid * H_kv + h) * (2 * D / 8);
+        if (tg < 2) {
+            const uint4 val = tg == 0 ? mn : mx;
+            gp[tg * LPR + lr] = val;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst_smem + (tg * LPR + lr) * 16),
+                         "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+        }
+    };
     // issue the copies of one batch into buffer `slot`; returns this lane's physical page (or -1)
     auto issue = [&](const Batch &d, int slot, int pid) -> int {
         if (pid >= P_phys) {
             atomicOr(status, SE_DEV_BAD_PAGE_ID);
             pid = -1;
         }
-        const unsigned valid = __ballot_sync(kFull, pid >= 0);
+        int fresh = -1;                        // lane of the page to summarise from K, if any
+        if (k_cache != nullptr) {
+            const int last = d.n_r - 1 - d.b0;
+            if (last >= 0 && last < kPB && __shfl_sync(kFull, pid, last) >= 0) fresh = last;
+        }
+        const unsigned valid = __ballot_sync(kFull, pid >= 0 && lane != fresh);
         const uint32_t bar = bar0 + slot * 8;
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)__popc(valid) * C::PHB);
         __syncwarp();
-        if (pid >= 0) {
+        if (pid >= 0 && lane != fresh) {
             const uint8_t *src = meta + ((size_t)pid * H_kv + d.h) * C::PHB;
             bulk_g2s(buf0 + slot * C::BUF + lane * C::PITCH, src, C::PHB, bar);
         }
+        if (fresh >= 0)
+            summarise_page(__shfl_sync(kFull, pid, fresh), d.h, min(kPage, d.len - (d.n_r - 1) * kPage),
+                           buf0 + slot * C::BUF + fresh * C::PITCH);
         return pid;
     };
 
     // Three batches are live: `cur` is computed, `nxt` is in flight, `nn` has only its page-table
     // entries on the way, so that its copies can be issued the moment a buffer frees up.
     Batch cur, nxt, nn;
-    decode_unit(gw, total_units, prefix, npages, B, H_kv, cur);
+    decode_unit(gw, total_units, prefix, npages, lens, B, H_kv, cur);
     if (cur.unit < 0) {
         check_out();
         return;
@@ -541,11 +588,12 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
 }
 
 template <int D>
-cudaError_t launch_score(const se_params &p, const void *q, const void *meta, const int32_t *page_table,
-                         const int32_t *seq_lens, float *scores, uint32_t *status, cudaStream_t stream) {
+cudaError_t launch_score(const se_params &p, const void *q, const void *meta, const void *k_cache,
+                         const int32_t *page_table, const int32_t *seq_lens, float *scores, uint32_t *status,
+                         cudaStream_t stream) {
     using C = ScoreCfg<D>;
     const size_t smem = (size_t)kScoreWarps * 2 * C::BUF + kScoreWarps * 2 * 8 +
-                        (size_t)(2 * p.B + 1) * sizeof(int);
+                        (size_t)(3 * p.B + 1) * sizeof(int);
     auto kern = score_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -558,14 +606,15 @@ cudaError_t launch_score(const se_params &p, const void *q, const void *meta, co
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
     kern<<<(unsigned)grid, kScoreWarps * 32, smem, stream>>>(
-        (const uint16_t *)q, (const uint8_t *)meta, page_table, seq_lens, scores, p.B, p.H_kv,
+        (const uint16_t *)q, (const uint8_t *)meta, (const uint8_t *)k_cache, (uint8_t *)const_cast<void *>(meta),
+        page_table, seq_lens, scores, p.B, p.H_kv,
         p.H_q / p.H_kv, p.max_pages, p.num_phys_pages, effective_scale(p), status);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta,
+cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta, const void *k_cache,
                                const int32_t *page_table, const int32_t *seq_lens, int k_pages,
                                int32_t *sel_idx, int32_t *sel_cnt, void *workspace,
                                const WorkspaceLayout &L, cudaStream_t stream) {
@@ -573,8 +622,8 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     float *scores = reinterpret_cast<float *>(ws + L.scores);
     uint32_t *status = reinterpret_cast<uint32_t *>(ws + L.status);
     cudaError_t e = (p.D == 128)
-                        ? launch_score<128>(p, q, meta, page_table, seq_lens, scores, status, stream)
-                        : launch_score<64>(p, q, meta, page_table, seq_lens, scores, status, stream);
+                        ? launch_score<128>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream)
+                        : launch_score<64>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream);
     if (e != cudaSuccess) return e;
     const int pairs = p.B * p.H_kv;
 #define SE_TOPK(THREADS, KPT)                                                                         \
@@ -655,7 +704,7 @@ extern "C" int se_page_select_static(const se_params *p, const void *q, const vo
     L.status = 0;
     L.scores = 256;
     L.total = need;
-    cudaError_t e = se::launch_page_select(*p, q, meta, page_table, seq_lens, budget_tokens / se::kPage,
+    cudaError_t e = se::launch_page_select(*p, q, meta, nullptr, page_table, seq_lens, budget_tokens / se::kPage,
                                            sel_idx, sel_cnt, scratch, L, s);
     if (e != cudaSuccess) return SE_ERR_CUDA;
     if (dev_status &&

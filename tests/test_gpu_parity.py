@@ -185,6 +185,34 @@ def test_incremental_summary_update_matches_rebuild():
             assert touched == (b >= 2), (r, b)
 
 
+@pytest.mark.parametrize("D,G", [(128, 4), (64, 2), (128, 7)])
+def test_fused_summary_update_equals_separate_calls(D, G):
+    """se_page_select_fused = se_meta_update (newest page) + se_page_select, bit for bit."""
+    w_cpu = wl.build("fused", 845, 0, [161, 320, 49, 16, 1, 0, 2000], 2 * G, 2, D, 96, "cpu",
+                     permute_pool=True, prune_fraction=0.1, poison_tail=True)
+    w = w_cpu.to("cuda")
+    short = (w.seq_lens - 1).clamp(min=0).contiguous()
+    ft = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    states = []
+    for fused in (False, True):
+        st = binding.DecodeState(w)
+        binding.se_meta_update(st.p, w.k_cache, w.page_table, short, st.meta, first_tok=ft)   # stale summaries
+        if fused:
+            st.select_fused()
+        else:
+            st.update_meta()
+            st.select()
+        st.decode()
+        torch.cuda.synchronize()
+        assert st.status() == 0
+        states.append(st)
+    a, b = states
+    assert torch.equal(a.meta.view(torch.int16), b.meta.view(torch.int16))
+    assert torch.equal(a.sel_idx, b.sel_idx) and torch.equal(a.sel_cnt, b.sel_cnt)
+    assert torch.equal(a.out, b.out) and torch.equal(a.lse, b.lse)
+    compare(w_cpu, b)
+
+
 def test_summary_signed_zero_and_masking():
     w_cpu = wl.build("zero", 850, 0, [20], 2, 1, 64, 32, "cpu", poison_tail=True)
     w_cpu.k_cache[0, 0, 0, 0] = 0.0
