@@ -219,6 +219,24 @@ int se_page_select_static(const se_params *p, const void *q, const void *meta,
                           int32_t *dev_status, void *stream);
 
 /*
+ * The two halves of se_sparse_decode as separate calls (same arguments, same workspace): first
+ * se_sparse_decode_splits - the split-K attention kernel; pairs held by a single worker get their
+ * final out/lse, the others leave partial results in the workspace - then se_combine - the
+ * log-sum-exp merge of the partials and, with score_accum, the H2O epilogue.  Calling one after
+ * the other on the same stream is exactly se_sparse_decode; they exist so that a profiler or a
+ * benchmark can time the two kernels apart.
+ */
+int se_sparse_decode_splits(const se_params *p, const void *q, const void *k_cache,
+                            const void *v_cache, const int32_t *page_table,
+                            const int32_t *seq_lens, const int32_t *sel_idx,
+                            const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                            void *workspace, void *stream);
+int se_combine(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+               const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+               const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+               void *workspace, void *stream);
+
+/*
  * Copies the device status word (an OR of SE_DEV_* bits, 0 = clean) to *host_out and
  * clears it.  Synchronises `stream`; the only entry point that does.
  */

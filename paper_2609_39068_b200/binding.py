@@ -21,7 +21,8 @@ SE_DEV_BAD_SELECTION = 2
 SE_DEV_WAIT_TIMEOUT = 4
 
 EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_workspace_init", "se_meta_update",
-           "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_last_device_status",
+           "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
+           "se_last_device_status",
            "se_page_select_static")
 SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
@@ -67,10 +68,13 @@ def load(build_if_missing: bool = True):
     lib.se_page_select.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_page_select_fused.argtypes = [pp, vp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_sparse_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, fp, fp, fp, vp, vp]
+    lib.se_sparse_decode_splits.argtypes = lib.se_sparse_decode.argtypes
+    lib.se_combine.argtypes = lib.se_sparse_decode.argtypes
     lib.se_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
-                 "se_sparse_decode", "se_last_device_status", "se_page_select_static"):
+                 "se_sparse_decode", "se_sparse_decode_splits", "se_combine", "se_last_device_status",
+                 "se_page_select_static"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -161,8 +165,8 @@ def se_page_select_fused(p, q, k_cache, meta, page_table, seq_lens, budget_token
 
 
 def se_sparse_decode(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-                     workspace, score_accum=None) -> None:
-    _check(load().se_sparse_decode(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                     workspace, score_accum=None, entry="se_sparse_decode") -> None:
+    _check(getattr(load(), entry)(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
                                    _ptr(k_cache, torch.bfloat16, "k_cache"),
                                    _ptr(v_cache, torch.bfloat16, "v_cache"),
                                    _ptr(page_table, torch.int32, "page_table"),
@@ -170,7 +174,15 @@ def se_sparse_decode(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_
                                    _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
                                    _ptr(out, torch.float32, "out"), _ptr(lse, torch.float32, "lse"),
                                    _ptr(score_accum, torch.float32, "score_accum"),
-                                   _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_sparse_decode")
+                                   _ptr(workspace, torch.uint8, "workspace"), _stream()), entry)
+
+
+def se_sparse_decode_splits(*args, **kw) -> None:
+    se_sparse_decode(*args, entry="se_sparse_decode_splits", **kw)
+
+
+def se_combine(*args, **kw) -> None:
+    se_sparse_decode(*args, entry="se_combine", **kw)
 
 
 def se_page_select_static(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,
@@ -224,10 +236,10 @@ class DecodeState:
         se_page_select(self.p, self.w.q, self.meta, self.w.page_table, self.w.seq_lens,
                        self.w.budget if budget is None else budget, self.sel_idx, self.sel_cnt, self.workspace)
 
-    def decode(self, score_accum=None):
+    def decode(self, score_accum=None, entry="se_sparse_decode"):
         se_sparse_decode(self.p, self.w.q, self.w.k_cache, self.w.v_cache, self.w.page_table,
                          self.w.seq_lens, self.sel_idx, self.sel_cnt, self.out, self.lse,
-                         self.workspace, score_accum=score_accum)
+                         self.workspace, score_accum=score_accum, entry=entry)
 
     def select_fused(self, budget: Optional[int] = None):
         se_page_select_fused(self.p, self.w.q, self.w.k_cache, self.meta, self.w.page_table, self.w.seq_lens,

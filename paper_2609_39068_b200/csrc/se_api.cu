@@ -170,10 +170,10 @@ int se_page_select_fused(const se_params *p, const void *q, const void *k_cache,
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
 }
 
-int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
-                     const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
-                     const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                     void *workspace, void *stream) {
+static int sparse_decode_stages(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                                const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+                                const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                                void *workspace, int stages, void *stream) {
     int rc = validate(p);
     if (rc != SE_OK) return rc;
     if (!q || !k_cache || !v_cache || !page_table || !seq_lens || !sel_idx || !sel_cnt || !out ||
@@ -185,9 +185,33 @@ int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, con
         return SE_ERR_MISALIGNED;
     const WorkspaceLayout L = make_layout(*p);
     cudaError_t e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens, sel_idx,
-                                         sel_cnt, out, lse, score_accum, workspace, L,
+                                         sel_cnt, out, lse, score_accum, workspace, L, stages,
                                          static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                     const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+                     const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                     void *workspace, void *stream) {
+    return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
+                                score_accum, workspace, 3, stream);
+}
+
+int se_sparse_decode_splits(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                            const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+                            const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                            void *workspace, void *stream) {
+    return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
+                                score_accum, workspace, 1, stream);
+}
+
+int se_combine(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+               const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+               const int32_t *sel_cnt, float *out, float *lse, float *score_accum, void *workspace,
+               void *stream) {
+    return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
+                                score_accum, workspace, 2, stream);
 }
 
 int se_last_device_status(void *workspace, void *stream, int32_t *host_out) {

@@ -541,19 +541,21 @@ template <int D>
 cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache, const void *v_cache,
                           const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
                           const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                          void *workspace, const WorkspaceLayout &L, cudaStream_t stream) {
+                          void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream) {
     using C = DecCfg<D>;
     const DecodePlan plan = make_decode_plan(p);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
+    const int G = p.H_q / p.H_kv, GP = next_pow2(G);
+    float *zbuf = score_accum ? reinterpret_cast<float *>(ws + L.zbuf) : nullptr;
+    cudaError_t e = cudaSuccess;
+    if (stages & 1) {
     CUtensorMap k_map, v_map;
     if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
     const size_t smem = (size_t)kDecWarps * C::WARP_SMEM + (size_t)kDecWarps * C::NSTAGE * 8 +
                         (size_t)kDecWarps * 2 * kChunk * sizeof(int) + 1024;
     auto kern = decode_kernel<D>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const int G = p.H_q / p.H_kv, GP = next_pow2(G);
-    float *zbuf = score_accum ? reinterpret_cast<float *>(ws + L.zbuf) : nullptr;
     kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
         k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
         reinterpret_cast<float *>(ws + L.partials), zbuf,
@@ -561,6 +563,8 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
         effective_scale(p) * kLog2e, reinterpret_cast<uint32_t *>(ws + L.status));
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    }
+    if (!(stages & 2)) return e;
     if (plan.max_splits == 1 && !score_accum) return e;       // every pair is written by one warp
     // with the H2O epilogue the token slots of a pair (16 per selected page) are spread over
     // several CTAs, two slots per thread
@@ -585,11 +589,11 @@ cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *
                                  const void *v_cache, const int32_t *page_table,
                                  const int32_t *seq_lens, const int32_t *sel_idx,
                                  const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                                 void *workspace, const WorkspaceLayout &L, cudaStream_t stream) {
+                                 void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream) {
     return (p.D == 128) ? launch_decode<128>(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                                             out, lse, score_accum, workspace, L, stream)
+                                             out, lse, score_accum, workspace, L, stages, stream)
                         : launch_decode<64>(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                                            out, lse, score_accum, workspace, L, stream);
+                                            out, lse, score_accum, workspace, L, stages, stream);
 }
 
 }  // namespace se

@@ -38,6 +38,7 @@ cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *
                                  const void *v_cache, const int32_t *page_table,
                                  const int32_t *seq_lens, const int32_t *sel_idx,
                                  const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                                 void *workspace, const WorkspaceLayout &L, cudaStream_t stream);
+                                 void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream);
+// stages: 1 = split attention kernel, 2 = combine kernel (merge + H2O epilogue), 3 = both
 
 }  // namespace se

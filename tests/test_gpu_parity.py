@@ -265,6 +265,20 @@ def test_two_runs_are_bit_identical_and_split_invariant():
     assert (st2.lse - l1).abs().max().item() <= 1e-5
 
 
+def test_split_and_combine_calls_equal_the_single_call():
+    w_cpu = wl.build("two", 875, 0, [5000, 300, 9000], 8, 2, 128, 1024, "cpu", permute_pool=True,
+                     with_score_accum=True)
+    w, st, u = run_gpu(w_cpu, accum=True)
+    o1, l1 = st.out.clone(), st.lse.clone()
+    st.out.fill_(float("nan"))
+    st.lse.fill_(float("nan"))
+    u2 = w.score_accum.clone()
+    st.decode(u2, entry="se_sparse_decode_splits")
+    st.decode(u2, entry="se_combine")
+    torch.cuda.synchronize()
+    assert torch.equal(o1, st.out) and torch.equal(l1, st.lse) and torch.equal(u, u2)
+
+
 def test_h2o_accumulation_small():
     w_cpu = wl.build("h2o", 880, 0, [700, 1300, 90], 8, 2, 128, 256, "cpu", permute_pool=True,
                      with_score_accum=True, poison_tail=True)
