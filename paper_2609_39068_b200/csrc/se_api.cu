@@ -75,7 +75,7 @@ WorkspaceLayout make_layout(const se_params &p) {
     const int GP = next_pow2(G);
     size_t off = 0;
     L.status = off;      off += 256;
-    L.scores = off;      off += align256(pairs * (size_t)p.max_pages * 4);
+    L.scores = off;      off += align256(pairs * (size_t)score_pitch(p) * 4);
     L.partials = off;    off += align256((size_t)p.B * p.H_q * plan.max_splits * (p.D + 4) * 4);
     L.zbuf = off;        off += align256(pairs * (size_t)p.k_max * kPage * GP * 4);
     L.total = off;

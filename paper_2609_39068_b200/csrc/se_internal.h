@@ -21,6 +21,8 @@ int  device_sm_count();
 DecodePlan make_decode_plan(const se_params &p);
 WorkspaceLayout make_layout(const se_params &p);
 float effective_scale(const se_params &p);
+// floats per (request, kv-head) row of the score scratch: rows start 16-byte aligned
+inline int score_pitch(const se_params &p) { return (p.max_pages + 3) & ~3; }
 
 // kernels' launchers; each returns a cudaError_t from the launch
 cudaError_t launch_meta_update(const se_params &p, const void *k_cache, const int32_t *page_table,

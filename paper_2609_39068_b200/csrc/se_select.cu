@@ -15,9 +15,10 @@
 //                and accumulate in fp32.  An earlier plain-FMA version of this kernel was
 //                issue-bound at 64 % of the copy bandwidth (57 warp instructions per page
 //                summary); this one needs 3.
-// topk_kernel    one CTA per (request, kv-head): most-significant-digit radix select over
-//                order-preserving integer keys held in registers, then a page-ordered
-//                compaction, so equal scores go to the lower page and the list is ascending.
+// topk_kernel    one CTA per (request, kv-head): order-preserving integer keys held in registers,
+//                threshold by a histogram over the keys' span plus a brute-force ranking of the
+//                crossing bin, then a page-ordered compaction, so equal scores go to the lower
+//                page and the list is ascending.
 #include "se_internal.h"
 
 namespace se {
@@ -71,7 +72,7 @@ template <int D>
 __global__ void __launch_bounds__(kScoreWarps * 32)
 score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t *__restrict__ k_cache,
              uint8_t *meta_out, const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
-             float *__restrict__ scores, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
+             float *__restrict__ scores, int pitch, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
              uint32_t *status) {
     using C = ScoreCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -308,7 +309,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
         const int pid_lo = __shfl_sync(kFull, pid_cur, gid);
         const int pid_hi = __shfl_sync(kFull, pid_cur, gid + 8);
         if (tid4 == 0) {
-            float *dst = scores + ((size_t)cur.r * H_kv + cur.h) * max_pages + cur.b0;
+            float *dst = scores + ((size_t)cur.r * H_kv + cur.h) * pitch + cur.b0;
             if (cur.b0 + gid < cur.n_r) dst[gid] = (pid_lo >= 0) ? s_lo * scale : ninf;
             if (cur.b0 + gid + 8 < cur.n_r) dst[gid + 8] = (pid_hi >= 0) ? s_hi * scale : ninf;
         }
@@ -337,57 +338,61 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
 }
 
 // ---------------------------------------------------------------------------------
-// top-k: one CTA of 256 threads per (request, kv-head); thread t holds keys t, t+256, ...
-// in registers.  Radix select with 8-bit digits (shared-memory histogram, double buffered, one
-// CTA barrier per digit, every warp locates the crossing digit on its own), then a page-ordered
-// compaction with one more barrier.
+// top-k: one CTA per (request, kv-head).  Thread t holds a run of consecutive pages in registers
+// (as order-preserving integer keys), so thread order is page order.  The k-th largest key is
+// found by one 2048-bin histogram over the span [kmin, kmax] of the request's keys; the bin
+// that holds it usually has a handful of keys, which are ranked by brute force (a further
+// histogram level over the bin's span serves crowded bins).  The result is a threshold
+// (key, page): a page is taken when its key is above the threshold key, or equal to it and
+// the page not above the threshold page - equal scores go to the lower page.  One prefix sum
+// over the per-thread counts then gives every thread the position of its pages in the
+// ascending output list.
 // ---------------------------------------------------------------------------------
 #ifndef SE_TOPK_MARK
 #define SE_TOPK_MARK(i)          // hook for an external timing probe; empty in the library
 #endif
+constexpr int kTopkBins = 2048;
+constexpr int kTopkBinBits = 11;
+constexpr int kTopkList = 32;        // bins with up to this many keys are ranked by brute force
 
-// Exclusive prefix over `entries` (multiple of 32, <= 256) ints in shared memory, computed by the
-// calling warp alone and written back in place.  Every warp of the CTA may run it on the same
-// array at the same time: they all write the same values.
-template <int ENTRIES>
-__device__ __forceinline__ int warp_scan_inplace(int *a, int lane) {
-    constexpr int EPL = ENTRIES / 32;
-    int v[EPL], sum = 0;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-        v[e] = a[lane * EPL + e];
-        sum += v[e];
-    }
-    int inc = sum;
+// Exclusive prefix of one int per thread over the CTA (thread order); `tot` is a shared array
+// of at least 32 ints that no other scan is using between the surrounding barriers.
+template <int NW>
+__device__ __forceinline__ int cta_excl_scan(int v, int *tot, int lane, int warp) {
+    int inc = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int t = __shfl_up_sync(kFull, inc, o);
         if (lane >= o) inc += t;
     }
-    const int total = __shfl_sync(kFull, inc, 31);
-    int run = inc - sum;
-    __syncwarp();
+    if (lane == 31) tot[warp] = inc;
+    __syncthreads();
+    const int wt = lane < NW ? tot[lane] : 0;
+    int winc = wt;
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-        a[lane * EPL + e] = run;
-        run += v[e];
+    for (int o = 1; o < NW; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, winc, o);
+        if (lane >= o) winc += t;
     }
-    __syncwarp();
-    return total;
+    return __shfl_sync(kFull, winc - wt, warp) + inc - v;
 }
 
-// kTopkThreads threads per CTA, KPT keys per thread held in registers (n <= kTopkThreads*KPT).
-template <int kTopkThreads, int KPT, bool kForced>
-__global__ void __launch_bounds__(kTopkThreads, (kTopkThreads * KPT <= 4096 && kTopkThreads <= 512) ? 1024 / kTopkThreads : 1)
-topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_lens, int H_kv,
+// THREADS threads per CTA, up to KPT (a multiple of 4) keys per thread: n <= THREADS*KPT.
+template <int THREADS, int KPT, bool kForced>
+__global__ void __launch_bounds__(THREADS)
+topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restrict__ seq_lens, int H_kv,
             int max_pages, int k_pages, int k_max, int sink_pages, int recent_pages,
             int32_t *__restrict__ sel_idx, int32_t *__restrict__ sel_cnt) {
-    constexpr int kTopkWarps = kTopkThreads / 32;
-    constexpr int ENTRIES = KPT * kTopkWarps;          // (tile, warp) cells of the compaction
-    static_assert(ENTRIES % 32 == 0 && ENTRIES <= 1024, "compaction cells");
-    __shared__ int s_red[4][kTopkWarps];
-    __shared__ int s_hist[2][256];
-    __shared__ int s_cnt[2][ENTRIES];
+    constexpr int NW = THREADS / 32;
+    constexpr int BPT = kTopkBins / THREADS;           // histogram bins per thread
+    static_assert(KPT % 4 == 0 && KPT <= 32 && BPT >= 1, "top-k shape");
+    __shared__ __align__(16) int s_hist[kTopkBins];    // indexed by 2047 - digit: prefix = keys above
+    __shared__ int s_tot[4][32];
+    __shared__ int s_red[4][NW];
+    __shared__ int s_res[6];
+    __shared__ uint32_t s_lkey[kTopkList];
+    __shared__ int s_lpage[kTopkList];
+    __shared__ int s_ln;
     SE_TOPK_MARK(9);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair = blockIdx.x;
@@ -395,40 +400,50 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     const int len = seq_lens[r];
     int n = len > 0 ? (len + kPage - 1) / kPage : 0;
     if (n > max_pages) n = max_pages;
-    const int n_full = n;                                     // pages the request's length spans
-    if (n > KPT * kTopkThreads) n = KPT * kTopkThreads;       // cannot happen: the launcher picks KPT from max_pages
-    const float *row = scores + (size_t)pair * max_pages;
+    if (n > KPT * THREADS) n = KPT * THREADS;          // cannot happen: the launcher picks KPT from max_pages
     int32_t *out = sel_idx + (size_t)pair * k_max;
-    const unsigned lt_mask = (1u << lane) - 1u;
-    const int tiles = (n + kTopkThreads - 1) / kTopkThreads;
 
-    // key j of thread t is page j*256 + t (tile-major, so (tile, thread) order is page order)
+    // thread t owns pages [t*kpe, (t+1)*kpe): kpe is the smallest multiple of 4 that covers the request
+    const int kpe = min(KPT, (((n + THREADS - 1) / THREADS) + 3) & ~3);
+    const int base = tid * kpe;
+    const float4 *row4 = reinterpret_cast<const float4 *>(scores + (size_t)pair * pitch);
     uint32_t keys[KPT];
+    uint32_t forcedmask = 0;         // pages taken regardless of their score; they do not compete
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const int i = j * kTopkThreads + tid;
-        uint32_t key = (i < n) ? f32_key(__ldg(row + i)) : kKeyAbsent;
-        // forced pages (sink / recent) leave the competition and are taken unconditionally
-        if (kForced && key != kKeyAbsent && (i < sink_pages || i >= n_full - recent_pages)) key = kKeyForced;
-        keys[j] = key;
+    for (int j4 = 0; j4 < KPT / 4; ++j4) {
+        const int i = base + 4 * j4;
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (4 * j4 < kpe && i < n) v = __ldg(row4 + (i >> 2));
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float ev = c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
+            uint32_t key = (i + c < n) ? f32_key(ev) : kKeyAbsent;         // absent pages score -inf
+            if (kForced && key != kKeyAbsent && (i + c < sink_pages || i + c >= n - recent_pages)) {
+                forcedmask |= 1u << (4 * j4 + c);
+                key = kKeyAbsent;
+            }
+            keys[4 * j4 + c] = key;
+        }
     }
     SE_TOPK_MARK(0);
+#pragma unroll
+    for (int e = 0; e < BPT; ++e) s_hist[tid * BPT + e] = 0;
+    if (tid == 0) s_ln = 0;
 
-    // ---- present pages, and the range of their keys
+    // ---- candidates, forced pages, and the span of the candidates' keys
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-    int present = 0, forced = 0;          // candidates / forced pages
+    int present = 0, forced = kForced ? __popc(forcedmask) : 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const bool ok = keys[j] != kKeyAbsent && (!kForced || keys[j] != kKeyForced);
+        const bool ok = keys[j] != kKeyAbsent;
         present += ok;
-        if (kForced) forced += keys[j] == kKeyForced;
         kmin = ok ? min(kmin, keys[j]) : kmin;
         kmax = ok ? max(kmax, keys[j]) : kmax;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         present += __shfl_xor_sync(kFull, present, o);
-        forced += __shfl_xor_sync(kFull, forced, o);
+        if (kForced) forced += __shfl_xor_sync(kFull, forced, o);
         kmin = min(kmin, __shfl_xor_sync(kFull, kmin, o));
         kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
     }
@@ -438,12 +453,11 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
         s_red[2][warp] = (int)kmax;
         s_red[3][warp] = forced;
     }
-    if (tid < 256) s_hist[0][tid] = 0;
     __syncthreads();
     present = 0;
     forced = 0;
 #pragma unroll
-    for (int w = 0; w < kTopkWarps; ++w) {
+    for (int w = 0; w < NW; ++w) {
         present += s_red[0][w];
         forced += s_red[3][w];
         kmin = min(kmin, (uint32_t)s_red[1][w]);
@@ -453,136 +467,158 @@ topk_kernel(const float *__restrict__ scores, const int32_t *__restrict__ seq_le
     const int k_eff = min(min(k_pages, k_max - forced), present);      // candidates to take
     SE_TOPK_MARK(1);
 
-    // ---- radix select of the k_eff-th largest key.  All present keys share the bits above the
-    // highest bit in which kmin and kmax differ, so the digits start there (scores of one
-    // request typically share sign, exponent and a few mantissa bits).
-    uint32_t prefix = 0;          // bits decided so far, lower bits zero
-    int remaining = k_eff;        // how many still to take among keys matching the prefix
-    bool ge_mode = false;         // take every key >= prefix (no ties to break)
-    if (k_eff > 0) {
-        if (k_eff == present) {               // everything present is wanted
-            prefix = kmin;
-            ge_mode = true;
-        } else if (kmin == kmax) {            // all equal: ties only
-            prefix = kmax;
-        } else {
-            int hi = 32 - __clz(kmin ^ kmax);                   // undecided low bits
-            prefix = (hi >= 32) ? 0u : (kmax >> hi) << hi;
-            int par = 0;
-            while (hi > 0 && !ge_mode) {
-                const int w = hi < 8 ? hi : 8;
-                const int shift = hi - w;
-                int *hist = s_hist[par];
-                // the digits are spread after the range narrowing, so plain shared-memory atomics
-                // rarely collide; tiles past the request's length are skipped altogether
-#pragma unroll
-                for (int j = 0; j < KPT; ++j) {
-                    if (j < tiles) {
-                        const uint32_t key = keys[j];
-                        const bool active = key != kKeyAbsent && (!kForced || key != kKeyForced) &&
-                                            ((hi >= 32) || ((key >> hi) == (prefix >> hi)));
-                        if (active) atomicAdd(&hist[(key >> shift) & ((1u << w) - 1u)], 1);
-                    }
-                }
-                if (tid < 256) s_hist[par ^ 1][tid] = 0;   // the other buffer serves the next digit
-                __syncthreads();
-                // every warp finds the digit d with  #(digits > d) < remaining <= #(digits >= d)
-                // on its own: lane l owns digits 8l..8l+7, higher lanes hold higher digits
-                int loc[8], sum = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    loc[j] = hist[lane * 8 + j];
-                    sum += loc[j];
-                }
-                int suf = sum;              // inclusive suffix sum over lanes
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int t = __shfl_down_sync(kFull, suf, o);
-                    if (lane + o < 32) suf += t;
-                }
-                const int above_lane = suf - sum;
-                const bool mine = above_lane < remaining && remaining <= suf;
-                int digit = 0, above_d = 0, inbin = 0;
-                if (mine) {
-                    int above = above_lane;
-#pragma unroll
-                    for (int j = 7; j >= 0; --j) {
-                        if (above < remaining && remaining <= above + loc[j]) {
-                            digit = lane * 8 + j;
-                            above_d = above;
-                            inbin = loc[j];
-                        }
-                        above += loc[j];
-                    }
-                }
-                const int owner = __ffs(__ballot_sync(kFull, mine)) - 1;
-                digit = __shfl_sync(kFull, digit, owner);
-                above_d = __shfl_sync(kFull, above_d, owner);
-                inbin = __shfl_sync(kFull, inbin, owner);
-                prefix |= (uint32_t)digit << shift;
-                remaining -= above_d;
-                if (inbin == remaining) ge_mode = true;      // the whole bin is taken
-                hi = shift;
-                par ^= 1;
-                SE_TOPK_MARK(2);
-            }
-        }
-    }
-    SE_TOPK_MARK(3);
-
     if (k_eff + forced == 0) {
-        for (int i = tid; i < k_max; i += kTopkThreads) out[i] = -1;
+        for (int i = tid; i < k_max; i += THREADS) out[i] = -1;
         if (tid == 0) sel_cnt[pair] = 0;
         return;
     }
-    if (k_eff == 0) {             // only forced pages: nothing competes
-        ge_mode = true;
-        prefix = kKeyForced;
-    }
-    // ---- ordered compaction: keys > T are taken; keys == T are taken in page order until `need`
-    // of them are in; in ge_mode every key >= T is taken.
-    const uint32_t T = prefix;
-    uint32_t takemask = 0, eqmask = 0;
+
+    // ---- threshold (T_key, T_page): taken <=> key > T_key || (key == T_key && page <= T_page)
+    uint32_t T_key = 0xffffffffu;
+    int T_page = -1;                         // k_eff == 0: nothing competes
+    int remaining = k_eff;                   // still to take among the keys inside the current span
+    bool ties = false;                       // the keys equal to T_key are taken in page order
+    if (k_eff > 0 && k_eff == present) {     // every candidate is wanted
+        T_key = kmin;
+        T_page = 0x7fffffff;
+    } else if (k_eff > 0 && kmin == kmax) {  // all equal
+        T_key = kmin;
+        ties = true;
+    } else if (k_eff > 0) {
+        uint32_t lo = kmin;                              // the current span is [lo, lo + span)
+        uint32_t span = kmax - kmin + 1u;
+        int width = 32 - __clz(kmax - kmin);             // span <= 2^width
+        for (int level = 0;; ++level) {
+            const int sh = width > kTopkBinBits ? width - kTopkBinBits : 0;
+            if (level > 0) {
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const bool valid = keys[j] != kKeyAbsent && (!kForced || keys[j] != kKeyForced);
-        const bool gt = (kForced && keys[j] == kKeyForced) || (valid && (ge_mode ? (keys[j] >= T) : (keys[j] > T)));
-        const bool eq = valid && !ge_mode && (keys[j] == T);
-        takemask |= (uint32_t)gt << j;
-        eqmask |= (uint32_t)eq << j;
-    }
-    if (!ge_mode) {                            // rank the ties (CTA-uniform branch)
+                for (int e = 0; e < BPT; ++e) s_hist[tid * BPT + e] = 0;
+                __syncthreads();
+            }
+            // keys spread over the bins nearly evenly, so plain shared-memory atomics rarely collide
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
-            if (lane == 0) s_cnt[1][j * kTopkWarps + warp] = __popc(b);
+            for (int j = 0; j < KPT; ++j) {
+                if ((j & ~3) < kpe) {
+                    const uint32_t d = keys[j] - lo;
+                    if (d < span) atomicAdd(&s_hist[(kTopkBins - 1) - (int)(d >> sh)], 1);
+                }
+            }
+            __syncthreads();
+            SE_TOPK_MARK(2);
+            // the bin b with  #(keys in bins above b) < remaining <= #(keys in bins above or in b)
+            int loc[BPT], sum = 0;
+#pragma unroll
+            for (int e = 0; e < BPT; ++e) {
+                loc[e] = s_hist[tid * BPT + e];
+                sum += loc[e];
+            }
+            const int excl = cta_excl_scan<NW>(sum, s_tot[level & 1], lane, warp);
+            if (excl < remaining && remaining <= excl + sum) {
+                int run = excl;
+#pragma unroll
+                for (int e = 0; e < BPT; ++e) {
+                    if (run < remaining && remaining <= run + loc[e]) {
+                        s_res[0] = tid * BPT + e;
+                        s_res[1] = run;
+                        s_res[2] = loc[e];
+                    }
+                    run += loc[e];
+                }
+            }
+            __syncthreads();
+            SE_TOPK_MARK(3);
+            const int digit = (kTopkBins - 1) - s_res[0];
+            const int inbin = s_res[2];
+            remaining -= s_res[1];
+            lo += (uint32_t)digit << sh;
+            span = 1u << sh;
+            width = sh;
+            T_key = lo;
+            if (inbin == remaining) {            // the whole bin is taken
+                T_page = 0x7fffffff;
+                break;
+            }
+            if (sh == 0) {                       // the bin is one key value: ties
+                ties = true;
+                break;
+            }
+            if (inbin <= kTopkList) {
+                // few keys left: collect them and rank each against the others
+#pragma unroll
+                for (int j = 0; j < KPT; ++j) {
+                    if ((j & ~3) < kpe) {
+                        const uint32_t d = keys[j] - lo;
+                        if (d < span) {
+                            const int pos = atomicAdd(&s_ln, 1);
+                            if (pos < kTopkList) {
+                                s_lkey[pos] = keys[j];
+                                s_lpage[pos] = base + j;
+                            }
+                        }
+                    }
+                }
+                __syncthreads();
+                SE_TOPK_MARK(6);
+                if (tid < inbin) {
+                    const uint32_t mk = s_lkey[tid];
+                    const int mp = s_lpage[tid];
+                    int rank = 0;                // keys of the bin that come before mine
+                    for (int i = 0; i < inbin; ++i) {
+                        const uint32_t ok = s_lkey[i];
+                        rank += (ok > mk) || (ok == mk && s_lpage[i] < mp);
+                    }
+                    if (rank == remaining - 1) {
+                        s_res[3] = (int)mk;
+                        s_res[4] = mp;
+                    }
+                }
+                __syncthreads();
+                SE_TOPK_MARK(7);
+                T_key = (uint32_t)s_res[3];
+                T_page = s_res[4];
+                break;
+            }
+        }
+    }
+    if (ties) {
+        // T_page = the remaining-th page, in page order, among the keys equal to T_key
+        int cnt = 0;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) cnt += keys[j] == T_key;
+        const int excl = cta_excl_scan<NW>(cnt, s_tot[2], lane, warp);
+        if (excl < remaining && remaining <= excl + cnt) {
+            int run = excl;
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) {
+                if (keys[j] == T_key) {
+                    ++run;
+                    if (run == remaining) s_res[5] = base + j;
+                }
+            }
         }
         __syncthreads();
-        warp_scan_inplace<ENTRIES>(s_cnt[1], lane);
-#pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            const unsigned b = __ballot_sync(kFull, (eqmask >> j) & 1u);
-            const int rank = s_cnt[1][j * kTopkWarps + warp] + __popc(b & lt_mask);
-            if (((eqmask >> j) & 1u) && rank < remaining) takemask |= 1u << j;
-        }
+        T_page = s_res[5];
     }
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
-        if (lane == 0) s_cnt[0][j * kTopkWarps + warp] = __popc(b);
-    }
-    __syncthreads();
-    warp_scan_inplace<ENTRIES>(s_cnt[0], lane);
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        if (j < tiles) {
-            const unsigned b = __ballot_sync(kFull, (takemask >> j) & 1u);
-            const int pos = s_cnt[0][j * kTopkWarps + warp] + __popc(b & lt_mask);
-            if (((takemask >> j) & 1u) && pos < k_max) out[pos] = j * kTopkThreads + tid;
-        }
-    }
+
     SE_TOPK_MARK(4);
-    for (int i = k_eff + forced + tid; i < k_max; i += kTopkThreads) out[i] = -1;
+    // ---- ordered compaction
+    uint32_t takemask = forcedmask;
+    const int jT = T_page - base;            // page <= T_page  <=>  j <= jT
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const bool take = keys[j] > T_key || (keys[j] == T_key && j <= jT);
+        takemask |= (uint32_t)take << j;
+    }
+    int pos = cta_excl_scan<NW>(__popc(takemask), s_tot[3], lane, warp);
+    SE_TOPK_MARK(8);
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        if ((takemask >> j) & 1u) {
+            if (pos < k_max) out[pos] = base + j;
+            ++pos;
+        }
+    }
+    for (int i = k_eff + forced + tid; i < k_max; i += THREADS) out[i] = -1;
     if (tid == 0) sel_cnt[pair] = k_eff + forced;
     SE_TOPK_MARK(5);
 }
@@ -607,7 +643,7 @@ cudaError_t launch_score(const se_params &p, const void *q, const void *meta, co
     if (grid < 1) grid = 1;
     kern<<<(unsigned)grid, kScoreWarps * 32, smem, stream>>>(
         (const uint16_t *)q, (const uint8_t *)meta, (const uint8_t *)k_cache, (uint8_t *)const_cast<void *>(meta),
-        page_table, seq_lens, scores, p.B, p.H_kv,
+        page_table, seq_lens, scores, score_pitch(p), p.B, p.H_kv,
         p.H_q / p.H_kv, p.max_pages, p.num_phys_pages, effective_scale(p), status);
     return cudaGetLastError();
 }
@@ -630,11 +666,13 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     do {                                                                                              \
         if (p.sink_pages || p.recent_pages)                                                           \
             topk_kernel<THREADS, KPT, true><<<pairs, THREADS, 0, stream>>>(                           \
-                scores, seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, p.sink_pages, p.recent_pages, \
+                scores, score_pitch(p), seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, p.sink_pages,      \
+                p.recent_pages,                                                                       \
                 sel_idx, sel_cnt);                                                                    \
         else                                                                                          \
             topk_kernel<THREADS, KPT, false><<<pairs, THREADS, 0, stream>>>(                          \
-                scores, seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, 0, 0, sel_idx, sel_cnt);     \
+                scores, score_pitch(p), seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, 0, 0, sel_idx,     \
+                sel_cnt);                                                                             \
     } while (0)
     // short requests: fewer keys per thread; long ones: more threads, so the per-thread chains stay short
     if (p.max_pages <= 1024) SE_TOPK(256, 4);
@@ -690,8 +728,8 @@ extern "C" int se_page_select_static(const se_params *p, const void *q, const vo
     if ((bits & 15u) || (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return SE_ERR_MISALIGNED;
     if (budget_tokens < se::kPage || budget_tokens / se::kPage + p->sink_pages + p->recent_pages > p->k_max)
         return SE_ERR_INVALID_ARG;
-    // scratch layout: [status word, padded to 256 bytes][fp32 scores, B*H_kv*max_pages]
-    const size_t need = 256 + (size_t)p->B * p->H_kv * p->max_pages * sizeof(float);
+    // scratch layout: [status word, padded to 256 bytes][fp32 scores, B*H_kv rows of max_pages rounded up to 4]
+    const size_t need = 256 + (size_t)p->B * p->H_kv * se::score_pitch(*p) * sizeof(float);
     if (need > SE_STATIC_SCRATCH_BYTES) return SE_ERR_SCRATCH_TOO_SMALL;
     void *scratch = nullptr;
     const int rc = static_scratch(&scratch);
