@@ -196,21 +196,26 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     // request's newest token may have changed since its summary was stored, so, when the caller
     // hands in the K cache, that one page per (request, head) is summarised from K here - written
     // to the summary array and straight into the batch buffer - instead of being copied.
-    auto summarise_page = [&](int pid, int h, int nv, uint32_t dst_smem) {
-        constexpr int LPR = D / 8;           // lanes per token row (16-byte pieces)
-        constexpr int TPP = 32 / LPR;        // token rows per warp pass
-        const int tg = lane / LPR, lr = lane % LPR;
+    // The K page is fetched into registers when its batch is issued and reduced when the batch is
+    // consumed, one buffer later, so the warp does not sit out the load.
+    constexpr int LPR = D / 8;               // lanes per token row (16-byte pieces)
+    constexpr int TPP = 32 / LPR;            // token rows per warp pass
+    constexpr int KROWS = kPage / TPP;       // 16-byte pieces of the page per lane
+    const int tg = lane / LPR, lr = lane % LPR;
+    auto fetch_page = [&](uint4 (&w)[KROWS], int pid, int h, int nv) {
         const uint4 *kp = reinterpret_cast<const uint4 *>(k_cache) + ((size_t)pid * H_kv + h) * (kPage * D / 8);
-        uint4 mn = make_uint4(0x7f807f80u, 0x7f807f80u, 0x7f807f80u, 0x7f807f80u);   // +inf pairs
-        uint4 mx = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // -inf pairs
 #pragma unroll
-        for (int i = 0; i < kPage / TPP; ++i) {
+        for (int i = 0; i < KROWS; ++i) {
             const int t = i * TPP + tg;
-            if (t < nv) {
-                const uint4 w = __ldg(kp + t * LPR + lr);
-                mn.x = bmin2(mn.x, w.x); mn.y = bmin2(mn.y, w.y); mn.z = bmin2(mn.z, w.z); mn.w = bmin2(mn.w, w.w);
-                mx.x = bmax2(mx.x, w.x); mx.y = bmax2(mx.y, w.y); mx.z = bmax2(mx.z, w.z); mx.w = bmax2(mx.w, w.w);
-            }
+            w[i] = __ldg(kp + (t < nv ? t : 0) * LPR + lr);      // rows past the length repeat row 0
+        }
+    };
+    auto reduce_page = [&](const uint4 (&w)[KROWS], int pid, int h, uint32_t dst_smem) {
+        uint4 mn = w[0], mx = w[0];
+#pragma unroll
+        for (int i = 1; i < KROWS; ++i) {
+            mn.x = bmin2(mn.x, w[i].x); mn.y = bmin2(mn.y, w[i].y); mn.z = bmin2(mn.z, w[i].z); mn.w = bmin2(mn.w, w[i].w);
+            mx.x = bmax2(mx.x, w[i].x); mx.y = bmax2(mx.y, w[i].y); mx.z = bmax2(mx.z, w[i].z); mx.w = bmax2(mx.w, w[i].w);
         }
 #pragma unroll
         for (int m = LPR; m < 32; m <<= 1) {
@@ -227,6 +232,8 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
                          "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
         }
     };
+    uint4 kpend[KROWS];                      // K page on its way for the batch in buffer pend_slot
+    int pend_slot = -1, pend_pid = 0, pend_h = 0, pend_lane = 0;
     // issue the copies of one batch into buffer `slot`; returns this lane's physical page (or -1)
     auto issue = [&](const Batch &d, int slot, int pid) -> int {
         if (pid >= P_phys) {
@@ -246,9 +253,21 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             const uint8_t *src = meta + ((size_t)pid * H_kv + d.h) * C::PHB;
             bulk_g2s(buf0 + slot * C::BUF + lane * C::PITCH, src, C::PHB, bar);
         }
-        if (fresh >= 0)
-            summarise_page(__shfl_sync(kFull, pid, fresh), d.h, min(kPage, d.len - (d.n_r - 1) * kPage),
-                           buf0 + slot * C::BUF + fresh * C::PITCH);
+        if (fresh >= 0) {
+            const int fpid = __shfl_sync(kFull, pid, fresh);
+            const int nv = min(kPage, d.len - (d.n_r - 1) * kPage);
+            if (pend_slot < 0) {
+                fetch_page(kpend, fpid, d.h, nv);
+                pend_slot = slot;
+                pend_pid = fpid;
+                pend_h = d.h;
+                pend_lane = fresh;
+            } else {                          // both buffers hold a newest page (very short requests)
+                uint4 w[KROWS];
+                fetch_page(w, fpid, d.h, nv);
+                reduce_page(w, fpid, d.h, buf0 + slot * C::BUF + fresh * C::PITCH);
+            }
+        }
         return pid;
     };
 
@@ -289,6 +308,11 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             break;
         }
         phases ^= (1u << slot);
+        if (pend_slot == slot) {
+            reduce_page(kpend, pend_pid, pend_h, buf0 + slot * C::BUF + pend_lane * C::PITCH);
+            pend_slot = -1;
+            __syncwarp();
+        }
 
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         const uint32_t a_base = buf0 + slot * C::BUF + lm_off;
