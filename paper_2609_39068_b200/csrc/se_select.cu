@@ -21,6 +21,25 @@
 //                page and the list is ascending.
 #include "se_internal.h"
 
+// Optional per-warp phase timing for development builds (-DSE_SCORE_PROFILE); compiled out of the
+// library otherwise.
+#ifdef SE_SCORE_PROFILE
+__device__ long long g_score_prof[8 * 4096];
+__device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define SP_DECL long long prof_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long prof_t_ = clock64(); const long long prof_t0_ = prof_t_; prof_[5] = gtimer();
+#define SP_LAP(i) { const long long t_ = clock64(); prof_[i] += t_ - prof_t_; prof_t_ = t_; }
+#define SP_ADD(i, v) { prof_[i] += (v); }
+#define SP_STORE(w) { if ((threadIdx.x & 31) == 0 && (w) < 4096) { prof_[7] = clock64() - prof_t0_; prof_[6] = gtimer(); for (int i_ = 0; i_ < 8; ++i_) g_score_prof[(w) * 8 + i_] = prof_[i_]; } }
+extern "C" int se_debug_score_profile(long long *host_out, int n_warps) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_score_prof, sizeof(long long) * 8 * n_warps);
+}
+#else
+#define SP_DECL
+#define SP_LAP(i)
+#define SP_ADD(i, v)
+#define SP_STORE(w)
+#endif
+
 namespace se {
 
 namespace {
@@ -41,13 +60,22 @@ struct ScoreCfg {
 struct Batch {
     int r, h, b0, n_r;      // request, kv-head, first logical page, pages of the request
     int len;                // tokens of the request
-    int unit;               // flat unit index this batch belongs to (-1 = end of stream)
-    int k;                  // batch number inside the unit
+    int unit;               // ticket this batch was handed out under (-1 = end of stream)
+    int k, kend;            // batch number inside the 64-page unit, and where this hand-out ends
 };
 
-// Flat unit u -> (request, head, first page); prefix[r] = units before request r.
-__device__ __forceinline__ bool decode_unit(int u, int total_units, const int *prefix, const int *npages,
+// Ticket t -> (request, head, first page).  Units of 64 pages are numbered request-major, head
+// fastest; prefix[r] = units before request r.  The first `big` tickets are whole units; the
+// tickets after that are single 16-page batches of the remaining units, so that the warps run
+// dry within one batch of each other instead of one unit.
+__device__ __forceinline__ bool decode_unit(int t, int total_units, int big, const int *prefix, const int *npages,
                                             const int *lens, int B, int H_kv, Batch &d) {
+    int u = t, k0 = 0, kend = kNBU;
+    if (t >= big) {
+        u = big + (t - big) / kNBU;
+        k0 = (t - big) % kNBU;
+        kend = k0 + 1;
+    }
     if (u >= total_units) {
         d.unit = -1;
         return false;
@@ -60,11 +88,12 @@ __device__ __forceinline__ bool decode_unit(int u, int total_units, const int *p
     const int local = u - prefix[lo];
     d.r = lo;
     d.h = local % H_kv;
-    d.b0 = (local / H_kv) * kUnitPages;
+    d.b0 = (local / H_kv) * kUnitPages + k0 * kPB;
     d.n_r = npages[lo];
     d.len = lens[lo];
-    d.unit = u;
-    d.k = 0;
+    d.unit = t;
+    d.k = k0;
+    d.kend = kend;
     return true;
 }
 
@@ -75,6 +104,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
              float *__restrict__ scores, int pitch, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
              uint32_t *status) {
     using C = ScoreCfg<D>;
+    SP_DECL
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // layout: [buffers: warps*2*BUF] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints] [lens: B ints]
     uint8_t *bufs = smem_raw;
@@ -118,6 +148,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     }
     __syncthreads();
     const int total_units = prefix[B];
+    const int big_units = total_units - total_units / 8;      // the last eighth goes out batch by batch
     const int gw = blockIdx.x * kScoreWarps + warp;
     const int tw = gridDim.x * kScoreWarps;
 
@@ -165,13 +196,13 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     // advance a descriptor to the next batch of this warp's stream
     auto next_batch = [&](Batch &d) {
         if (d.unit < 0) return;
-        if (d.k + 1 < kNBU && d.b0 + kPB < d.n_r) {
+        if (d.k + 1 < d.kend && d.b0 + kPB < d.n_r) {
             d.k += 1;
             d.b0 += kPB;
             return;
         }
         const int u = __shfl_sync(kFull, pending_unit, 0);
-        if (decode_unit(u, total_units, prefix, npages, lens, B, H_kv, d)) request_unit();
+        if (decode_unit(u, total_units, big_units, prefix, npages, lens, B, H_kv, d)) request_unit();
     };
     // every warp checks out once; the last one leaves the counters at zero for the next launch
     auto check_out = [&]() {
@@ -274,7 +305,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     // Three batches are live: `cur` is computed, `nxt` is in flight, `nn` has only its page-table
     // entries on the way, so that its copies can be issued the moment a buffer frees up.
     Batch cur, nxt, nn;
-    decode_unit(gw, total_units, prefix, npages, lens, B, H_kv, cur);
+    decode_unit(gw, total_units, big_units, prefix, npages, lens, B, H_kv, cur);
     if (cur.unit < 0) {
         check_out();
         return;
@@ -282,16 +313,15 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     request_unit();
     uint32_t phases = 0u;            // parity bit per buffer
     int slot = 0;
-    int pid_cur = issue(cur, 0, load_pids(cur));
-    load_qraw(cur);
-    convert_q();
     nxt = cur;
     next_batch(nxt);
-    int pid_nxt = -1;
-    if (nxt.unit >= 0) {
-        pid_nxt = issue(nxt, 1, load_pids(nxt));
-        if (nxt.r != cur.r || nxt.h != cur.h) load_qraw(nxt);
-    }
+    int pid_cur = load_pids(cur);
+    int pid_nxt = load_pids(nxt);            // both look-ups and q in flight before the first copy goes out
+    load_qraw(cur);
+    pid_cur = issue(cur, 0, pid_cur);
+    if (nxt.unit >= 0) pid_nxt = issue(nxt, 1, pid_nxt);
+    convert_q();
+    if (nxt.unit >= 0 && (nxt.r != cur.r || nxt.h != cur.h)) load_qraw(nxt);
     nn = nxt;
     next_batch(nn);
     int pid_nn = load_pids(nn);
@@ -301,6 +331,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     // {first | second 16-byte piece of the k16 step}
     const uint32_t lm_off = (uint32_t)(((lane & 7) + 8 * ((lane >> 3) & 1)) * C::PITCH + (lane >> 4) * 16);
 
+    SP_LAP(0)
     while (cur.unit >= 0) {
         // wait for the current buffer
         if (!mbar_wait(bar0 + slot * 8, (phases >> slot) & 1u)) {
@@ -308,6 +339,8 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             break;
         }
         phases ^= (1u << slot);
+        SP_LAP(1)
+        SP_ADD(4, 1)
         if (pend_slot == slot) {
             reduce_page(kpend, pend_pid, pend_h, buf0 + slot * C::BUF + pend_lane * C::PITCH);
             pend_slot = -1;
@@ -338,6 +371,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             if (cur.b0 + gid + 8 < cur.n_r) dst[gid + 8] = (pid_hi >= 0) ? s_hi * scale : ninf;
         }
         __syncwarp();        // every lane is done reading the buffer before it is refilled
+        SP_LAP(2)
 
         // refill the buffer just consumed with `nn` (its page-table entries arrived long ago)
         if (nn.unit >= 0) pid_nn = issue(nn, slot, pid_nn);
@@ -352,7 +386,9 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
         next_batch(nn);
         pid_nn = load_pids(nn);
         slot ^= 1;
+        SP_LAP(3)
     }
+    SP_STORE(gw)
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // give the copy that may still be in flight a bounded chance to land before leaving
