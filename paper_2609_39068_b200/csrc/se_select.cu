@@ -439,7 +439,7 @@ __device__ __forceinline__ int cta_excl_scan(int v, int *tot, int lane, int warp
 
 // THREADS threads per CTA, up to KPT (a multiple of 4) keys per thread: n <= THREADS*KPT.
 template <int THREADS, int KPT, bool kForced>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)
 topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restrict__ seq_lens, int H_kv,
             int max_pages, int k_pages, int k_max, int sink_pages, int recent_pages,
             int32_t *__restrict__ sel_idx, int32_t *__restrict__ sel_cnt) {
@@ -619,23 +619,23 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
                 }
                 __syncthreads();
                 SE_TOPK_MARK(6);
-                if (tid < inbin) {
-                    const uint32_t mk = s_lkey[tid];
-                    const int mp = s_lpage[tid];
-                    int rank = 0;                // keys of the bin that come before mine
+                // every warp ranks the (at most 32) collected keys on its own: lane i holds entry i,
+                // the entry that `remaining - 1` others precede is the threshold
+                {
+                    const bool has = lane < inbin;
+                    const uint32_t mk = has ? s_lkey[lane] : 0u;
+                    const int mp = has ? s_lpage[lane] : 0x7fffffff;
+                    int rank = 0;
                     for (int i = 0; i < inbin; ++i) {
-                        const uint32_t ok = s_lkey[i];
-                        rank += (ok > mk) || (ok == mk && s_lpage[i] < mp);
+                        const uint32_t ok = __shfl_sync(kFull, mk, i);
+                        const int op = __shfl_sync(kFull, mp, i);
+                        rank += (ok > mk) || (ok == mk && op < mp);
                     }
-                    if (rank == remaining - 1) {
-                        s_res[3] = (int)mk;
-                        s_res[4] = mp;
-                    }
+                    const int owner = __ffs(__ballot_sync(kFull, has && rank == remaining - 1)) - 1;
+                    T_key = __shfl_sync(kFull, mk, owner);
+                    T_page = __shfl_sync(kFull, mp, owner);
                 }
-                __syncthreads();
                 SE_TOPK_MARK(7);
-                T_key = (uint32_t)s_res[3];
-                T_page = s_res[4];
                 break;
             }
         }
@@ -671,14 +671,29 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
     }
     int pos = cta_excl_scan<NW>(__popc(takemask), s_tot[3], lane, warp);
     SE_TOPK_MARK(8);
+    const int total = k_eff + forced;
+    if (k_max <= kTopkBins) {
+        // the list is put together in shared memory (the histogram is no longer needed) and
+        // written out with coalesced stores, padding included
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        if ((takemask >> j) & 1u) {
-            if (pos < k_max) out[pos] = base + j;
-            ++pos;
+        for (int j = 0; j < KPT; ++j) {
+            if ((takemask >> j) & 1u) {
+                if (pos < k_max) s_hist[pos] = base + j;
+                ++pos;
+            }
         }
+        __syncthreads();
+        for (int i = tid; i < k_max; i += THREADS) out[i] = i < total ? s_hist[i] : -1;
+    } else {
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            if ((takemask >> j) & 1u) {
+                if (pos < k_max) out[pos] = base + j;
+                ++pos;
+            }
+        }
+        for (int i = total + tid; i < k_max; i += THREADS) out[i] = -1;
     }
-    for (int i = k_eff + forced + tid; i < k_max; i += THREADS) out[i] = -1;
     if (tid == 0) sel_cnt[pair] = k_eff + forced;
     SE_TOPK_MARK(5);
 }
