@@ -332,6 +332,8 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 for (int nt = 0; nt < C::NTILES; ++nt) {
                     o_acc[nt][0] *= corr;
                     o_acc[nt][1] *= corr;
+                    o_acc[nt][2] *= corr;
+                    o_acc[nt][3] *= corr;
                 }
                 m_run = m_new;
             }
@@ -339,7 +341,10 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
 #pragma unroll
             for (int e = 0; e < 4; ++e) p[e] = exp2f(z[e] - m_run);    // exp2(-inf) = 0 for masked tokens
             l_run += (p[0] + p[1]) + (p[2] + p[3]);
-            // P as the A operand, split into two bf16 terms so that p_hi + p_lo carries 16 bits
+            // P as the A operand, split into two bf16 terms so that p_hi + p_lo carries 16 bits.  The
+            // group has at most 8 heads, so rows 8-15 of the m16 tile are free: p_hi goes into rows
+            // 0-7 and p_lo into rows 8-15, and one MMA yields both products (accumulator elements
+            // 0,1 and 2,3 of this lane); they are added when the unit ends.
             const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
             const float2 f0 = bf16x2_to_f2(ph0), f1 = bf16x2_to_f2(ph1);
             const uint32_t pl0 = pack_bf16(p[0] - f0.x, p[1] - f0.y), pl1 = pack_bf16(p[2] - f1.x, p[3] - f1.y);
@@ -351,10 +356,8 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 const int chunk = 2 * (c2 & 3) + v_chunk_add;
                 uint32_t v00, v01, v10, v11;     // {chunk c: tok 0-7, tok 8-15}, {chunk c+1: ...}
                 ldmatrix_x4_trans(Vs + hf * kTileBytes + v_row * 128 + ((chunk ^ (v_row & 7)) << 4), v00, v01, v10, v11);
-                mma_bf16_16816(o_acc[2 * c2], ph0, 0u, ph1, 0u, v00, v01);
-                mma_bf16_16816(o_acc[2 * c2], pl0, 0u, pl1, 0u, v00, v01);
-                mma_bf16_16816(o_acc[2 * c2 + 1], ph0, 0u, ph1, 0u, v10, v11);
-                mma_bf16_16816(o_acc[2 * c2 + 1], pl0, 0u, pl1, 0u, v10, v11);
+                mma_bf16_16816(o_acc[2 * c2], ph0, pl0, ph1, pl1, v00, v01);
+                mma_bf16_16816(o_acc[2 * c2 + 1], ph0, pl0, ph1, pl1, v10, v11);
             }
             __syncwarp();     // all lanes are done with this stage before it is refilled
             ++ce;
@@ -368,6 +371,11 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         // ---- the four lanes of a head hold disjoint token columns: fold their l
         l_run += __shfl_xor_sync(kFull, l_run, 1);
         l_run += __shfl_xor_sync(kFull, l_run, 2);
+#pragma unroll
+        for (int nt = 0; nt < C::NTILES; ++nt) {        // p_hi and p_lo products
+            o_acc[nt][0] += o_acc[nt][2];
+            o_acc[nt][1] += o_acc[nt][3];
+        }
 
         if (n_split == 1) {
             if (head_ok) {
