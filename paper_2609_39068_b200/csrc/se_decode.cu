@@ -62,11 +62,12 @@ struct DecCfg {
     static constexpr int PSTRIDE = D + 4;                      // floats per partial row
 };
 
-// TMA: 2-D tile (x = channel, y = row of the [pages*heads*16, D] view) -> shared memory.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+// TMA: one page = 3-D box (64 channels, 16 token rows, D/64 channel halves) of the cache viewed as
+// [half][row][64 channels]; it lands as D/64 swizzled 16x128-byte tiles, one after the other.
+__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap *map, int y, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(y), "r"(0), "r"(bar)
         : "memory");
 }
 
@@ -94,7 +95,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)kDecWarps * C::WARP_SMEM) + warp * C::NSTAGE;
     if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(smem_u32(&bars[s]), 2 * C::HALVES);
+        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(smem_u32(&bars[s]), 2);
         mbar_fence_init();
     }
     __syncwarp();
@@ -193,18 +194,16 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         ce = 0;
         pe = 0;
     };
-    // called between pages, when no stage is being read: fill every free stage.  One lane per
-    // 16x64 tile arms the stage's barrier with its own byte count and issues its tensor copy (the
-    // barrier expects one arrival per tile, so the lanes need no ordering among themselves).
+    // called between pages, when no stage is being read: fill every free stage.  Lane 0 fetches the
+    // K page, lane 1 the V page; each arms the stage's barrier with its own byte count (the barrier
+    // expects two arrivals, so the lanes need no ordering between themselves).
     auto top_up = [&]() {
         while (pe < n_ent && pe < ce + C::NSTAGE) {
-            if (lane < 2 * C::HALVES) {
+            if (lane < 2) {
                 const uint32_t bar = bar0 + stage_i * 8;
-                const int y = ent_y[pe];
-                const int hf = lane >> 1;
-                const uint32_t dst = ring0 + stage_i * C::STAGEB + (lane & 1) * C::PAGEB + hf * kTileBytes;
-                mbar_expect_tx(bar, kTileBytes);
-                tma_load_2d(dst, (lane & 1) ? &v_map : &k_map, hf * 64, y, bar);
+                const uint32_t dst = ring0 + stage_i * C::STAGEB + lane * C::PAGEB;
+                mbar_expect_tx(bar, C::PAGEB);
+                tma_load_page(dst, lane ? &v_map : &k_map, ent_y[pe], bar);
             }
             stage_i = (stage_i + 1 == C::NSTAGE) ? 0 : stage_i + 1;
             ++pe;
@@ -532,15 +531,17 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// The cache viewed as a 2-D bf16 tensor [P_phys*H_kv*16 rows, D channels]; box = 16 rows x 64 channels.
+// The cache viewed as a 3-D bf16 tensor [D/64 halves][P_phys*H_kv*16 rows][64 channels] (the half
+// index is the slowest box dimension although its stride, 128 bytes, is the smaller one);
+// box = 64 channels x 16 rows x all halves = one page of one head.
 bool make_page_map(CUtensorMap *map, const void *base, const se_params &p) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)p.D, (cuuint64_t)p.num_phys_pages * p.H_kv * kPage};
-    const cuuint64_t strides[1] = {(cuuint64_t)p.D * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    const cuuint64_t dims[3] = {64, (cuuint64_t)p.num_phys_pages * p.H_kv * kPage, (cuuint64_t)(p.D / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)p.D * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kPage, (cuuint32_t)(p.D / 64)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
