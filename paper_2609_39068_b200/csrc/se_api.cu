@@ -47,16 +47,20 @@ float effective_scale(const se_params &p) {
 
 int decode_warps_per_cta();
 
-// Split-K geometry: every (request, kv-head) pair is cut into the same number of splits, as many
-// as the persistent warps of the grid can take in one round (one unit per warp), so that no warp
-// carries two pairs and every warp has the same number of pages.
+// Split-K geometry: every (request, kv-head) pair is cut into the same number of splits.  With two
+// or more pairs per SM the pairs themselves fill the machine (a few warps per SM, each with a deep
+// copy pipeline, already saturate HBM) and splitting would only add the merge; below that, as many
+// splits as the persistent warps of the grid can take in one round (one unit per warp).
 DecodePlan make_decode_plan(const se_params &p) {
     DecodePlan plan;
     const int warps_per_cta = decode_warps_per_cta();
     const long long pairs = (long long)p.B * p.H_kv;
     const long long warps = (long long)kAssumedSMs * warps_per_cta;
     long long splits = warps / pairs;
-    if (splits < 1) splits = 1;
+#ifndef SE_X_NOSPLIT_PAIRS_PER_SM
+#define SE_X_NOSPLIT_PAIRS_PER_SM 2
+#endif
+    if (splits < 1 || pairs >= (long long)SE_X_NOSPLIT_PAIRS_PER_SM * kAssumedSMs) splits = 1;
     if (splits > p.k_max) splits = p.k_max;
     const int pps = (int)((p.k_max + splits - 1) / splits);
     plan.pages_per_split = pps;

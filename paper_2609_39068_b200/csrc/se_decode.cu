@@ -55,10 +55,15 @@ struct DecCfg {
     static constexpr int HALVES = D / 64;                      // 64-channel tiles per page
     static constexpr int PAGEB = kPage * D * 2;                // bytes of one K (or V) page
     static constexpr int STAGEB = 2 * PAGEB;                   // K tiles then V tiles
-    static constexpr int NSTAGE = (D == 128) ? 3 : 4;
+    static constexpr int MAXST = 8;                            // most stages one warp can hold
+    // Stages a CTA shares out among its busy warps.  More copies in flight than this made the
+    // kernel slower, not faster (measured: 24 pages in flight per SM lose 3 % against 16 to 20).
+#ifndef SE_X_CTA_STAGES
+#define SE_X_CTA_STAGES 20
+#endif
+    static constexpr int CTA_STAGES = SE_X_CTA_STAGES * (128 / D);
     static constexpr int KSTEPS = D / 16;
     static constexpr int NTILES = D / 8;                       // n8 tiles of the output
-    static constexpr int WARP_SMEM = NSTAGE * STAGEB;
     static constexpr int PSTRIDE = D + 4;                      // floats per partial row
 };
 
@@ -91,11 +96,16 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     // tiles must sit on 1024-byte boundaries for the 128-byte swizzle pattern
     uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint8_t *ring = smem_al + (size_t)warp * C::WARP_SMEM;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)kDecWarps * C::WARP_SMEM) + warp * C::NSTAGE;
+    // The CTA's stages are shared out among the warps that have work: warp w of this CTA is busy iff
+    // its first unit w*gridDim.x + blockIdx.x exists, so the busy warps are the lowest ones.  Every
+    // busy warp gets the same number of stages (warps with unequal pipelines finish apart).
+    int busy = (B * H_kv * max_splits - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    busy = busy < 1 ? 1 : (busy > kDecWarps ? kDecWarps : busy);
+    const int nstage = warp < busy ? min(C::MAXST, C::CTA_STAGES / busy) : 0;
+    uint8_t *ring = smem_al + (size_t)(warp * nstage) * C::STAGEB;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB) + warp * C::MAXST;
     if (lane == 0) {
-#pragma unroll
-        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(smem_u32(&bars[s]), 2);
+        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 2);
         mbar_fence_init();
     }
     __syncwarp();
@@ -132,7 +142,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     // look-ups, across pair boundaries.
     //   ent_y    row of the page's first token in the [pages*heads*16, D] view of the cache
     //   ent_info valid tokens (bits 0-4) | selection index i (bits 5-16) | slot - chunk_base (bits 17-23)
-    int *ent_y = reinterpret_cast<int *>(smem_al + (size_t)kDecWarps * C::WARP_SMEM + kDecWarps * C::NSTAGE * 8) +
+    int *ent_y = reinterpret_cast<int *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8) +
                  warp * 2 * kChunk;
     int *ent_info = ent_y + kChunk;
     int chunk_base = 0, chunk_end = 0;           // slots [chunk_base, chunk_end) are in the list
@@ -198,14 +208,14 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     // K page, lane 1 the V page; each arms the stage's barrier with its own byte count (the barrier
     // expects two arrivals, so the lanes need no ordering between themselves).
     auto top_up = [&]() {
-        while (pe < n_ent && pe < ce + C::NSTAGE) {
+        while (pe < n_ent && pe < ce + nstage) {
             if (lane < 2) {
                 const uint32_t bar = bar0 + stage_i * 8;
                 const uint32_t dst = ring0 + stage_i * C::STAGEB + lane * C::PAGEB;
                 mbar_expect_tx(bar, C::PAGEB);
                 tma_load_page(dst, lane ? &v_map : &k_map, ent_y[pe], bar);
             }
-            stage_i = (stage_i + 1 == C::NSTAGE) ? 0 : stage_i + 1;
+            stage_i = (stage_i + 1 == nstage) ? 0 : stage_i + 1;
             ++pe;
         }
     };
@@ -286,7 +296,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             SE_PROF_ADD(5, 1)
             const uint32_t Ks = ring0 + stage_c * C::STAGEB;
             const uint32_t Vs = Ks + C::PAGEB;
-            stage_c = (stage_c + 1 == C::NSTAGE) ? 0 : stage_c + 1;
+            stage_c = (stage_c + 1 == nstage) ? 0 : stage_c + 1;
 
             // ---- S^T[head, token] = Q . K^T : two n8 tiles (tokens 0-7, 8-15)
             float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -406,7 +416,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // bounded wait for whatever this warp still has in flight before the CTA can retire
-        for (int s = 0; s < C::NSTAGE; ++s) mbar_wait(bar0 + s * 8, (phases >> s) & 1u);
+        for (int s = 0; s < nstage; ++s) mbar_wait(bar0 + s * 8, (phases >> s) & 1u);
     }
 }
 
@@ -560,7 +570,7 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     if (stages & 1) {
     CUtensorMap k_map, v_map;
     if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
-    const size_t smem = (size_t)kDecWarps * C::WARP_SMEM + (size_t)kDecWarps * C::NSTAGE * 8 +
+    const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
                         (size_t)kDecWarps * 2 * kChunk * sizeof(int) + 1024;
     auto kern = decode_kernel<D>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
