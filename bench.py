@@ -42,8 +42,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
 # capture summarised in profiles/ (null until a capture of that workload exists)
 NCU_TRAFFIC_BYTES = {
-    # profiles/decode_kernel_config3_b24.md: 205.57 MB for 24576 tiles, scaled to 65536 tiles
-    "config3_contbatch_b64_mix": 548.2e6,
+    # profiles/full_capture_config3_b24.md: 201.91 MB read for 24576 tiles, scaled to 65536 tiles,
+    # plus the 1.06 MB of out/lse a full-size launch writes (it writes no partials: one split)
+    "config3_contbatch_b64_mix": 539.5e6,
 }
 
 
@@ -388,7 +389,10 @@ def main():
             cpu_baseline["sample"] += "; one layer timed, x%d layers" % n_layers
 
     if rank == 0:
-        launches_per_step = n_layers * 4        # score, top-k, decode, combine (summary update fused into score)
+        # score, top-k, decode (summary update fused into score); the merge kernel runs only when
+        # the pairs are split or the H2O epilogue is on
+        merges = binding.se_decode_num_splits(states[0].p) > 1 or h2o
+        launches_per_step = n_layers * (3 + int(merges))
         line = {
             "metric": METRIC, "value": ms_per_step * 1e3, "unit": "us", "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": ms_per_step,

@@ -101,6 +101,14 @@ const char *se_strerror(int code);
 size_t se_workspace_bytes(const se_params *p);
 
 /*
+ * Split-K geometry se_sparse_decode uses for `p` (host, pure): the number of splits every
+ * (request, kv-head) pair is cut into, or 0 if `p` is invalid.  1 means every pair is attended by
+ * one worker, which writes out/lse itself; the merge kernel then only runs for the H2O epilogue.
+ * Informational: lets a caller count kernel launches or size its own tooling.
+ */
+int se_decode_num_splits(const se_params *p);
+
+/*
  * Zeroes the control block (status word, work-queue counters) at the head of the
  * workspace.  Required once after allocation; the kernels leave the counters at zero
  * when they finish, so it need not be repeated.

@@ -20,7 +20,8 @@ SE_DEV_BAD_PAGE_ID = 1
 SE_DEV_BAD_SELECTION = 2
 SE_DEV_WAIT_TIMEOUT = 4
 
-EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_workspace_init", "se_meta_update",
+EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_decode_num_splits", "se_workspace_init",
+           "se_meta_update",
            "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
            "se_last_device_status",
            "se_page_select_static")
@@ -63,6 +64,7 @@ def load(build_if_missing: bool = True):
     lib.se_strerror.argtypes = [ctypes.c_int]
     lib.se_workspace_bytes.restype = ctypes.c_size_t
     lib.se_workspace_bytes.argtypes = [pp]
+    lib.se_decode_num_splits.argtypes = [pp]
     lib.se_workspace_init.argtypes = [pp, vp, vp]
     lib.se_meta_update.argtypes = [pp, vp, i32p, i32p, i32p, vp, vp]
     lib.se_page_select.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
@@ -117,6 +119,10 @@ def se_strerror(code: int) -> str:
 
 def se_workspace_bytes(p: SeParams) -> int:
     return int(load().se_workspace_bytes(ctypes.byref(p)))
+
+
+def se_decode_num_splits(p: SeParams) -> int:
+    return int(load().se_decode_num_splits(ctypes.byref(p)))
 
 
 def se_workspace_init(p: SeParams, workspace: torch.Tensor) -> None:

@@ -113,6 +113,11 @@ size_t se_workspace_bytes(const se_params *p) {
     return make_layout(*p).total;
 }
 
+int se_decode_num_splits(const se_params *p) {
+    if (validate(p) != SE_OK) return 0;
+    return make_decode_plan(*p).max_splits;
+}
+
 int se_workspace_init(const se_params *p, void *workspace, void *stream) {
     int rc = validate(p);
     if (rc != SE_OK) return rc;

@@ -47,6 +47,15 @@ def test_workspace_bytes_is_pure_and_monotone():
     assert binding.se_workspace_bytes(p2) > n1
 
 
+def test_decode_split_plan():
+    # few pairs: split so that every persistent warp has a unit; two or more pairs per SM: no split
+    few = binding.make_params(8, 32, 8, 128, 2048, 16384, 128)
+    many = binding.make_params(64, 32, 8, 128, 4096, 140000, 128)
+    assert binding.se_decode_num_splits(few) > 1
+    assert binding.se_decode_num_splits(many) == 1
+    assert binding.se_decode_num_splits(binding.make_params(8, 32, 8, 96, 2048, 16384, 128)) == 0
+
+
 @pytest.mark.parametrize("kw", [
     dict(D=96), dict(page_size=32), dict(H_q=36), dict(H_q=72), dict(B=0), dict(k_max=0),
     dict(k_max=5000), dict(max_pages=0), dict(num_phys_pages=0), dict(sm_scale=-1.0),
