@@ -13,7 +13,8 @@ The five steps can be called one by one so that each CUDA stage is checkable on 
     out, lse  = attend(...)              softmax attention over the selected tokens
                                          (+ H2O accumulated attention mass, in place)
 
-``decode_step`` chains them the way one decode step of the engine does.
+``decode_step`` chains them the way one decode step of the engine does.  ``h2o_retain`` /
+``h2o_compact`` are the consumer of the H2O statistic: the retained set and the eviction.
 """
 from __future__ import annotations
 
@@ -175,6 +176,43 @@ def attend(q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
                              _p(sel_cnt, ctypes.c_int32), _p(out, ctypes.c_double),
                              _p(lse, ctypes.c_double), _p(u_accum, ctypes.c_double))
     return out, lse
+
+
+def h2o_retain(u_accum, page_table, seq_lens, budget, recent, page_size=16):
+    """H2O retained set per (request, kv-head): returns (keep_idx [B,H_kv,budget] int32, ascending
+    token positions, -1 padded; keep_cnt [B,H_kv]).  ``u_accum`` [P,H_kv,p] float64."""
+    u_accum = np.ascontiguousarray(u_accum, dtype=np.float64)
+    P_, H_kv, p = u_accum.shape
+    assert p == page_size
+    page_table = _i32(page_table)
+    seq_lens = _i32(seq_lens)
+    B, max_pages = page_table.shape
+    keep_idx = np.full((B, H_kv, int(budget)), -1, dtype=np.int32)
+    keep_cnt = np.zeros((B, H_kv), dtype=np.int32)
+    _load().se_oracle_h2o_retain(B, H_kv, p, max_pages, int(budget), int(recent),
+                                 _p(u_accum, ctypes.c_double), _p(page_table, ctypes.c_int32),
+                                 _p(seq_lens, ctypes.c_int32), _p(keep_idx, ctypes.c_int32),
+                                 _p(keep_cnt, ctypes.c_int32))
+    return keep_idx, keep_cnt
+
+
+def h2o_compact(k_cache, v_cache, u_accum, page_table, keep_idx, keep_cnt):
+    """Eviction as slot compaction.  Returns new copies (k_cache, v_cache, u_accum, new_lens)."""
+    k = _u16(k_cache).copy()
+    v = _u16(v_cache).copy()
+    u = np.ascontiguousarray(u_accum, dtype=np.float64).copy()
+    P_, H_kv, p, D = k.shape
+    page_table = _i32(page_table)
+    keep_idx = _i32(keep_idx)
+    keep_cnt = _i32(keep_cnt)
+    B, max_pages = page_table.shape
+    budget = keep_idx.shape[2]
+    new_lens = np.zeros((B,), dtype=np.int32)
+    _load().se_oracle_h2o_compact(B, H_kv, D, p, max_pages, P_, budget, _p(k, ctypes.c_uint16),
+                                  _p(v, ctypes.c_uint16), _p(u, ctypes.c_double),
+                                  _p(page_table, ctypes.c_int32), _p(keep_idx, ctypes.c_int32),
+                                  _p(keep_cnt, ctypes.c_int32), _p(new_lens, ctypes.c_int32))
+    return k, v, u, new_lens
 
 
 def decode_step(q, k_cache, v_cache, page_table, seq_lens, budget, meta=None,

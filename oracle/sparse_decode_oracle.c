@@ -14,6 +14,8 @@
  *   se_oracle_topk     TopK_b(s; A)                    (Appendix A, notation table)
  *   se_oracle_attend   attention over selected tokens  (Appendix A, selected-attention eq.)
  *                      + H2O accumulated score         (Appendix A, H2O score eq.)
+ *   se_oracle_h2o_retain   H2O retained set R = W u TopK(u; A \ W)   (Appendix A, H2O retention eq.)
+ *   se_oracle_h2o_compact  eviction: retained tokens moved to the front of the request's cache
  *
  * Conventions (0-based everywhere; the paper's positions are 1-based):
  *   logical page b of request r holds tokens [b*p, min(len_r, (b+1)*p)); its physical
@@ -25,6 +27,9 @@
  * score, equality with a token logit on single-token pages, unit-vector closed forms,
  * argsort brute force for top-k, equality with dense attention when every page is
  * selected, log-sum-exp against a library routine, the unit sum of attention mass.
+ * For the H2O retention: the paper's budget-4 / two-recent-tokens example, argsort brute force,
+ * the "a token that leaves the window competes on its score" scenario, and equality of attention
+ * over the retained tokens before and after compaction.
  * Parity with the authors' own code is unpinned: the paper prints no numbers for
  * this path, and the reduction of a GQA group to one per-kv-head score (max) is a
  * convention of this build.
@@ -286,4 +291,107 @@ void se_oracle_attend(int B, int H_q, int H_kv, int D, int p, int max_pages, int
         }
         free(z);
     }
+}
+
+/*
+ * H2O retained set (Appendix A, "H2O: Accumulated Scores and Online Eviction", retention equation).
+ * For request r (len_r tokens, token j in logical page j/p, slot j%p) and kv-head h:
+ *     A = the tokens of the request whose page has a physical page,
+ *     W = the tokens of A among the last w = min(recent, budget) positions of the request,
+ *     R = W  u  TopK_{budget-|W|}(u; A \ W)      (all of A \ W if it has fewer members),
+ * where u[pid,h,t] is the accumulated score of the token stored in slot t of physical page pid.
+ * Equal scores are ordered by lower position.  keep_idx[r,h,:] lists R in ascending token
+ * position, padded with -1 up to `budget` entries; keep_cnt[r,h] = |R| (the same for every head
+ * of a request, since it only depends on |A|).
+ *   u [P, H_kv, p] (double)   keep_idx [B, H_kv, budget]   keep_cnt [B, H_kv]
+ */
+typedef struct { double u; int pos; } tok_t;
+
+static int tok_cmp(const void *x, const void *y) {
+    const tok_t *a = (const tok_t *)x, *b = (const tok_t *)y;
+    if (a->u > b->u) return -1;
+    if (a->u < b->u) return 1;
+    return (a->pos > b->pos) - (a->pos < b->pos);
+}
+
+void se_oracle_h2o_retain(int B, int H_kv, int p, int max_pages, int budget, int recent,
+                          const double *u, const int32_t *page_table, const int32_t *seq_lens,
+                          int32_t *keep_idx, int32_t *keep_cnt) {
+    const int w = recent < budget ? recent : budget;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int r = 0; r < B; ++r)
+        for (int h = 0; h < H_kv; ++h) {
+            int len = seq_lens[r];
+            if (len > max_pages * p) len = max_pages * p;
+            if (len < 0) len = 0;
+            int32_t *row = keep_idx + ((size_t)r * H_kv + h) * budget;
+            for (int i = 0; i < budget; ++i) row[i] = -1;
+            tok_t *cand = (tok_t *)malloc(sizeof(tok_t) * (size_t)(len > 0 ? len : 1));
+            int *kept = (int *)malloc(sizeof(int) * (size_t)(budget > 0 ? budget : 1));
+            int n_cand = 0, n_kept = 0;
+            for (int j = 0; j < len; ++j) {
+                const int pid = page_table[(size_t)r * max_pages + j / p];
+                if (pid < 0) continue;                       /* not in A */
+                if (j >= len - w) {                          /* protected recent window */
+                    kept[n_kept++] = j;
+                } else {
+                    cand[n_cand].u = u[((size_t)pid * H_kv + h) * p + j % p];
+                    cand[n_cand].pos = j;
+                    ++n_cand;
+                }
+            }
+            int k = budget - n_kept;
+            if (k > n_cand) k = n_cand;
+            qsort(cand, (size_t)n_cand, sizeof(tok_t), tok_cmp);
+            for (int i = 0; i < k; ++i) kept[n_kept++] = cand[i].pos;
+            qsort(kept, (size_t)n_kept, sizeof(int), int_cmp);
+            for (int i = 0; i < n_kept; ++i) row[i] = kept[i];
+            keep_cnt[(size_t)r * H_kv + h] = n_kept;
+            free(cand);
+            free(kept);
+        }
+}
+
+/*
+ * Eviction as slot compaction: for every request r and kv-head h the retained tokens
+ * keep_idx[r,h,0..cnt) move, in order, to token positions 0..cnt-1 of the request: K, V and the
+ * accumulated score of position i become those of position keep_idx[r,h,i] ("the scores of
+ * retained entries persist").  Everything is gathered from a snapshot of the caches, so the
+ * result does not depend on the order of the moves.  new_lens[r] = cnt (the heads of a request
+ * must agree on it; the first ceil(cnt/p) logical pages of the request must be present).
+ * Slots past the new length keep whatever they held.
+ *   k_cache, v_cache [P, H_kv, p, D] bf16 bits (in/out)   u [P, H_kv, p] (in/out)
+ */
+void se_oracle_h2o_compact(int B, int H_kv, int D, int p, int max_pages, int P, int budget,
+                           uint16_t *k_cache, uint16_t *v_cache, double *u,
+                           const int32_t *page_table, const int32_t *keep_idx,
+                           const int32_t *keep_cnt, int32_t *new_lens) {
+    const size_t n_kv = (size_t)P * H_kv * p * D, n_u = (size_t)P * H_kv * p;
+    uint16_t *k0 = (uint16_t *)malloc(n_kv * sizeof(uint16_t));
+    uint16_t *v0 = (uint16_t *)malloc(n_kv * sizeof(uint16_t));
+    double *u0 = (double *)malloc(n_u * sizeof(double));
+    memcpy(k0, k_cache, n_kv * sizeof(uint16_t));
+    memcpy(v0, v_cache, n_kv * sizeof(uint16_t));
+    memcpy(u0, u, n_u * sizeof(double));
+    for (int r = 0; r < B; ++r) {
+        for (int h = 0; h < H_kv; ++h) {
+            const int cnt = keep_cnt[(size_t)r * H_kv + h];
+            const int32_t *row = keep_idx + ((size_t)r * H_kv + h) * budget;
+            for (int i = 0; i < cnt; ++i) {
+                const int j = row[i];
+                const int pid_d = page_table[(size_t)r * max_pages + i / p];
+                const int pid_s = page_table[(size_t)r * max_pages + j / p];
+                if (pid_d < 0 || pid_s < 0) continue;        /* precondition violated: leave alone */
+                const size_t d = ((size_t)pid_d * H_kv + h) * p + i % p;
+                const size_t sidx = ((size_t)pid_s * H_kv + h) * p + j % p;
+                memcpy(k_cache + d * D, k0 + sidx * D, (size_t)D * sizeof(uint16_t));
+                memcpy(v_cache + d * D, v0 + sidx * D, (size_t)D * sizeof(uint16_t));
+                u[d] = u0[sidx];
+            }
+        }
+        new_lens[r] = keep_cnt[(size_t)r * H_kv];
+    }
+    free(k0);
+    free(v0);
+    free(u0);
 }
