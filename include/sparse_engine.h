@@ -245,6 +245,40 @@ int se_combine(const se_params *p, const void *q, const void *k_cache, const voi
                void *workspace, void *stream);
 
 /*
+ * H2O retained set (Appendix A, "H2O: Accumulated Scores and Online Eviction", retention
+ * equation).  For request r (seq_lens[r] tokens; token j lives in slot j % 16 of logical page
+ * j / 16) and kv-head h, with u = score_accum as maintained by se_sparse_decode:
+ *     A = the request's tokens whose logical page is present (page_table >= 0),
+ *     W = the tokens of A among the last min(recent_tokens, budget_tokens) positions,
+ *     R = W  u  TopK_{budget - |W|}(u; A \ W)       (all of A \ W if it has fewer members);
+ * equal scores go to the lower position.  keep_idx[r,h,:] ([B, H_kv, budget_tokens] int32, device)
+ * receives R in ascending token position, padded with -1; keep_cnt[r,h] = |R| (the same for every
+ * head of a request).  Reads score_accum, page_table, seq_lens; writes only keep_idx / keep_cnt.
+ * 1 <= budget_tokens <= 2^20.  Scores must be finite.  Asynchronous on `stream`,
+ * allocates nothing; bad page ids are reported through the workspace's status word.
+ */
+int se_h2o_retain(const se_params *p, const float *score_accum, const int32_t *page_table,
+                  const int32_t *seq_lens, int32_t budget_tokens, int32_t recent_tokens,
+                  int32_t *keep_idx, int32_t *keep_cnt, void *workspace, void *stream);
+
+/*
+ * H2O eviction as slot compaction ("KV outside R is evicted, while the scores of retained entries
+ * persist"): for every (request, kv-head) the retained tokens keep_idx[r,h,0..keep_cnt) move, in
+ * order, to token positions 0..keep_cnt-1 of the request - K row, V row and accumulated score of
+ * position i become those of position keep_idx[r,h,i] - and new_seq_lens[r] = keep_cnt[r,0].
+ * In place: k_cache, v_cache and score_accum are read and written; slots past the new length keep
+ * what they held.  Requirements: keep_idx rows ascending (as se_h2o_retain writes them), the heads
+ * of a request agree on keep_cnt, the request's first ceil(cnt/16) logical pages are present, and
+ * no physical page is shared between requests.  Page summaries (meta) of the touched pages are
+ * stale afterwards: rebuild them with se_meta_update(first_tok = 0) before the next page
+ * selection.  budget_tokens is the row length of keep_idx.  Invalid rows (a source before its
+ * destination, absent or out-of-range pages) are skipped and reported through the status word.
+ */
+int se_h2o_compact(const se_params *p, void *k_cache, void *v_cache, float *score_accum,
+                   const int32_t *page_table, const int32_t *keep_idx, const int32_t *keep_cnt,
+                   int32_t budget_tokens, int32_t *new_seq_lens, void *workspace, void *stream);
+
+/*
  * Copies the device status word (an OR of SE_DEV_* bits, 0 = clean) to *host_out and
  * clears it.  Synchronises `stream`; the only entry point that does.
  */

@@ -23,7 +23,7 @@ SE_DEV_WAIT_TIMEOUT = 4
 EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_decode_num_splits", "se_workspace_init",
            "se_meta_update",
            "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
-           "se_last_device_status",
+           "se_last_device_status", "se_h2o_retain", "se_h2o_compact",
            "se_page_select_static")
 SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
@@ -73,10 +73,12 @@ def load(build_if_missing: bool = True):
     lib.se_sparse_decode_splits.argtypes = lib.se_sparse_decode.argtypes
     lib.se_combine.argtypes = lib.se_sparse_decode.argtypes
     lib.se_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.se_h2o_retain.argtypes = [pp, fp, i32p, i32p, ctypes.c_int32, ctypes.c_int32, i32p, i32p, vp, vp]
+    lib.se_h2o_compact.argtypes = [pp, vp, vp, fp, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp]
     lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
                  "se_sparse_decode", "se_sparse_decode_splits", "se_combine", "se_last_device_status",
-                 "se_page_select_static"):
+                 "se_h2o_retain", "se_h2o_compact", "se_decode_num_splits", "se_page_select_static"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -204,6 +206,26 @@ def se_page_select_static(p, q, meta, page_table, seq_lens, budget_tokens, sel_i
                                         _ptr(sel_cnt, torch.int32, "sel_cnt"),
                                         _ptr(dev_status, torch.int32, "dev_status"), _stream()),
            "se_page_select_static")
+
+
+def se_h2o_retain(p, score_accum, page_table, seq_lens, budget_tokens, recent_tokens, keep_idx, keep_cnt,
+                  workspace) -> None:
+    _check(load().se_h2o_retain(ctypes.byref(p), _ptr(score_accum, torch.float32, "score_accum"),
+                                _ptr(page_table, torch.int32, "page_table"),
+                                _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens), int(recent_tokens),
+                                _ptr(keep_idx, torch.int32, "keep_idx"), _ptr(keep_cnt, torch.int32, "keep_cnt"),
+                                _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_h2o_retain")
+
+
+def se_h2o_compact(p, k_cache, v_cache, score_accum, page_table, keep_idx, keep_cnt, new_seq_lens,
+                   workspace) -> None:
+    _check(load().se_h2o_compact(ctypes.byref(p), _ptr(k_cache, torch.bfloat16, "k_cache"),
+                                 _ptr(v_cache, torch.bfloat16, "v_cache"),
+                                 _ptr(score_accum, torch.float32, "score_accum"),
+                                 _ptr(page_table, torch.int32, "page_table"),
+                                 _ptr(keep_idx, torch.int32, "keep_idx"), _ptr(keep_cnt, torch.int32, "keep_cnt"),
+                                 int(keep_idx.shape[-1]), _ptr(new_seq_lens, torch.int32, "new_seq_lens"),
+                                 _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_h2o_compact")
 
 
 def se_last_device_status(workspace) -> int:

@@ -223,6 +223,43 @@ int se_combine(const se_params *p, const void *q, const void *k_cache, const voi
                                 score_accum, workspace, 2, stream);
 }
 
+int se_h2o_retain(const se_params *p, const float *score_accum, const int32_t *page_table,
+                  const int32_t *seq_lens, int32_t budget_tokens, int32_t recent_tokens, int32_t *keep_idx,
+                  int32_t *keep_cnt, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!score_accum || !page_table || !seq_lens || !keep_idx || !keep_cnt || !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(score_accum) || !aligned16(page_table) || !aligned16(seq_lens) || !aligned16(keep_idx) ||
+        !aligned16(keep_cnt) || !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    if (budget_tokens < 1 || budget_tokens > (1 << 20) || recent_tokens < 0) return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_h2o_retain(*p, score_accum, page_table, seq_lens, budget_tokens, recent_tokens, keep_idx,
+                                      keep_cnt, reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + L.status),
+                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_h2o_compact(const se_params *p, void *k_cache, void *v_cache, float *score_accum,
+                   const int32_t *page_table, const int32_t *keep_idx, const int32_t *keep_cnt,
+                   int32_t budget_tokens, int32_t *new_seq_lens, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!k_cache || !v_cache || !score_accum || !page_table || !keep_idx || !keep_cnt || !new_seq_lens || !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(score_accum) || !aligned16(page_table) ||
+        !aligned16(keep_idx) || !aligned16(keep_cnt) || !aligned16(new_seq_lens) || !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    if (budget_tokens < 1 || budget_tokens > (1 << 20)) return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_h2o_compact(*p, k_cache, v_cache, score_accum, page_table, keep_idx, keep_cnt, budget_tokens,
+                                       new_seq_lens,
+                                       reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + L.status),
+                                       static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
 int se_last_device_status(void *workspace, void *stream, int32_t *host_out) {
     if (!workspace || !host_out) return SE_ERR_NULL_POINTER;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

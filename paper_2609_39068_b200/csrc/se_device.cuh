@@ -112,6 +112,28 @@ __device__ __forceinline__ uint32_t f32_key(float f) {
 constexpr uint32_t kKeyAbsent = 0x007fffffu;   // f32_key(-inf): below every finite score
 constexpr uint32_t kKeyForced = 0xffffffffu;   // marks a page that is selected regardless of its score
 
+// Exclusive prefix of one int per thread over the CTA (thread order); `tot` is a shared array
+// of at least 32 ints that no other scan is using between the surrounding barriers.
+template <int NW>
+__device__ __forceinline__ int cta_excl_scan(int v, int *tot, int lane, int warp) {
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) tot[warp] = inc;
+    __syncthreads();
+    const int wt = lane < NW ? tot[lane] : 0;
+    int winc = wt;
+#pragma unroll
+    for (int o = 1; o < NW; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, winc, o);
+        if (lane >= o) winc += t;
+    }
+    return __shfl_sync(kFull, winc - wt, warp) + inc - v;
+}
+
 // ---------------------------------------------------------------------------------
 // warp-level matrix helpers (bf16 inputs, fp32 accumulation)
 // ---------------------------------------------------------------------------------

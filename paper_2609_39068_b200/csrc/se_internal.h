@@ -41,6 +41,13 @@ cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *
                                  const int32_t *seq_lens, const int32_t *sel_idx,
                                  const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
                                  void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream);
+// H2O retention (retained positions per (request, kv-head)) and eviction (in-place compaction)
+cudaError_t launch_h2o_retain(const se_params &p, const float *score_accum, const int32_t *page_table,
+                              const int32_t *seq_lens, int budget, int recent, int32_t *keep_idx,
+                              int32_t *keep_cnt, uint32_t *status, cudaStream_t stream);
+cudaError_t launch_h2o_compact(const se_params &p, void *k_cache, void *v_cache, float *score_accum,
+                               const int32_t *page_table, const int32_t *keep_idx, const int32_t *keep_cnt,
+                               int budget, int32_t *new_lens, uint32_t *status, cudaStream_t stream);
 // stages: 1 = split attention kernel, 2 = combine kernel (merge + H2O epilogue), 3 = both
 
 }  // namespace se

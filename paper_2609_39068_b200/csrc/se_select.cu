@@ -415,28 +415,6 @@ constexpr int kTopkBins = 2048;
 constexpr int kTopkBinBits = 11;
 constexpr int kTopkList = 32;        // bins with up to this many keys are ranked by brute force
 
-// Exclusive prefix of one int per thread over the CTA (thread order); `tot` is a shared array
-// of at least 32 ints that no other scan is using between the surrounding barriers.
-template <int NW>
-__device__ __forceinline__ int cta_excl_scan(int v, int *tot, int lane, int warp) {
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(kFull, inc, o);
-        if (lane >= o) inc += t;
-    }
-    if (lane == 31) tot[warp] = inc;
-    __syncthreads();
-    const int wt = lane < NW ? tot[lane] : 0;
-    int winc = wt;
-#pragma unroll
-    for (int o = 1; o < NW; o <<= 1) {
-        const int t = __shfl_up_sync(kFull, winc, o);
-        if (lane >= o) winc += t;
-    }
-    return __shfl_sync(kFull, winc - wt, warp) + inc - v;
-}
-
 // THREADS threads per CTA, up to KPT (a multiple of 4) keys per thread: n <= THREADS*KPT.
 template <int THREADS, int KPT, bool kForced>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS)

@@ -251,6 +251,14 @@ def config5(device="cpu", layer: int = 0, B: int = 128, lo: int = 8192, hi: int 
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
 
 
+def h2o_evict_workload(device="cpu", B: int = 64, cached: int = 5120, budget: int = 4096) -> Workload:
+    """Periodic decode eviction of an H2O cache: B=64 concurrent requests, each 1024 tokens over its
+    4096-token budget (the paper's settings evict every 1024 decode steps), 32/8 heads, D=128,
+    pages dealt from a permuted pool, accumulated scores |N(0,1)|."""
+    return build("h2o_evict_b64_5120to4096", 6, 0, [cached] * B, 32, 8, 128, budget, device,
+                 permute_pool=True, with_score_accum=True)
+
+
 def sub_workload(w: Workload, rows, device="cpu") -> Workload:
     """The requests ``rows`` of ``w`` with their pages gathered into a compact pool of their
     own (physical ids renumbered, aliasing preserved).  Pure data movement: it lets a few
