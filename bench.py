@@ -48,6 +48,10 @@ NCU_TRAFFIC_BYTES = {
 }
 
 
+# dram bytes of one h2o_compact_kernel launch on the 64-request eviction workload (profiles/)
+H2O_NCU_TRAFFIC_BYTES = 2055e6        # 770.7 MB at 24 requests, scaled by the request count
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -208,6 +212,9 @@ def main():
                     help="override the number of requests (configs 3-5; for small profiling captures)")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls directly instead of a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="decode", choices=["decode", "h2o_evict"],
+                    help="decode = the sparse decode step (the headline); h2o_evict = one H2O eviction "
+                         "(retained set + in-place compaction) of 64 requests, 5120 -> 4096 tokens")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -216,6 +223,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     n_layers = args.layers or (28 if args.config == 5 else 1)
 
+    if args.workload == "h2o_evict":
+        if rank == 0:                        # the eviction step has no multi-GPU leg of its own
+            run_h2o_evict(args, local_rank)
+        return
     if args.impl == "reference":
         if rank == 0:
             run_reference(args, n_layers)
@@ -428,6 +439,126 @@ def main():
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
+
+
+def h2o_oracle_time(w, budget, recent, n_sample=8):
+    """The oracle's retained set + compaction on a few requests, scaled to the batch by request count."""
+    import oracle
+    rows = list(range(0, w.B, max(1, w.B // n_sample)))[:n_sample]
+    sub = wl.sub_workload(w, rows, "cpu")
+    k, v = wl.bf16_bits(sub.k_cache), wl.bf16_bits(sub.v_cache)
+    u = sub.score_accum.numpy().astype(np.float64)
+    pt, sl = sub.page_table.numpy(), sub.seq_lens.numpy()
+    times = []
+    for _ in range(3):
+        t0 = time.perf_counter()
+        idx, cnt = oracle.h2o_retain(u, pt, sl, budget, recent)
+        oracle.h2o_compact(k, v, u, pt, idx, cnt)
+        times.append(time.perf_counter() - t0)
+    best, scale = min(times), w.B / float(len(rows))
+    return dict(value=best * scale * 1e6, unit="us", cores=oracle.num_threads(), kind="oracle",
+                sample="%d of %d requests, retained set (OpenMP over pairs) + compaction (one thread), best of 3 "
+                       "= %.1f ms, scaled x%.1f by request count" % (len(rows), w.B, best * 1e3, scale))
+
+
+def run_h2o_evict(args, local_rank):
+    """One H2O eviction step: se_h2o_retain + se_h2o_compact on 64 requests that are 1024 tokens over
+    their 4096-token budget (recent ratio 0.2).  The scores are restored (untimed) before every step,
+    so every step evicts the same tokens; K/V values do not influence the work."""
+    budget, recent = 4096, 819
+    if args.impl == "reference":
+        dev = "cuda" if torch.cuda.is_available() else "cpu"
+        w = wl.h2o_evict_workload(dev) if dev == "cuda" else wl.h2o_evict_workload(dev, B=8)
+        cb = h2o_oracle_time(w, budget, recent)
+        print(json.dumps({
+            "impl": "reference", "metric": "h2o_evict_us_per_step", "value": cb["value"], "unit": "us",
+            "n_gpus": args.gpus, "steps": 3, "warmup": 0, "ms_per_step": cb["value"] / 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name}, "cpu_baseline": cb,
+            "e2e": {"value": cb["value"], "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    from paper_2609_39068_b200 import binding
+    binding.load()
+    w = wl.h2o_evict_workload(dev, B=args.batch or 64)
+    p = binding.make_params(w.B, w.H_q, w.H_kv, w.D, w.max_pages, w.num_phys_pages, 1)
+    ws = binding.alloc_workspace(p, dev)
+    keep_idx = torch.empty((w.B, w.H_kv, budget), dtype=torch.int32, device=dev)
+    keep_cnt = torch.empty((w.B, w.H_kv), dtype=torch.int32, device=dev)
+    new_lens = torch.empty((w.B,), dtype=torch.int32, device=dev)
+    u0 = w.score_accum.clone()
+    lens_pin = w.seq_lens.cpu().pin_memory()
+    out_pin = torch.empty((w.B,), dtype=torch.int32).pin_memory()
+
+    def retain():
+        binding.se_h2o_retain(p, w.score_accum, w.page_table, w.seq_lens, budget, recent, keep_idx, keep_cnt, ws)
+
+    def compact():
+        binding.se_h2o_compact(p, w.k_cache, w.v_cache, w.score_accum, w.page_table, keep_idx, keep_cnt,
+                               new_lens, ws)
+
+    def timed(fns, iters, e2e=False):
+        tot = 0.0
+        for _ in range(iters):
+            w.score_accum.copy_(u0)                      # untimed: same eviction every step
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if e2e:
+                w.seq_lens.copy_(lens_pin, non_blocking=True)
+            for fn in fns:
+                fn()
+            if e2e:
+                out_pin.copy_(new_lens, non_blocking=True)
+            b.record()
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        return tot / iters * 1e3
+
+    K = min(args.steps, 200)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    timed([retain, compact], args.warmup)
+    t0 = time.perf_counter()
+    step_us = timed([retain, compact], K)
+    t1 = time.perf_counter()
+    w.score_accum.copy_(u0)
+    retain()
+    retain_us = timed([retain], 50)
+    compact_us = timed([compact], 50)                    # keep_idx of the step above, scores restored each time
+    e2e_us = timed([retain, compact], 50, e2e=True)
+    sampler.stop()
+    status = binding.se_last_device_status(ws)
+    if status:
+        raise SystemExit("device status %d" % status)
+    # algorithmic bytes: every destination page that holds a moved token is read and written once
+    ki = keep_idx.cpu().numpy().reshape(-1, budget)
+    moved_tok = ki != np.arange(budget)[None, :]
+    moved_pages = int(moved_tok.reshape(ki.shape[0], budget // 16, 16).any(axis=2).sum())
+    row_bytes = 2 * w.D * 2 + 4                          # K row + V row + score
+    compact_bytes = moved_pages * 16 * row_bytes * 2 + ki.size * 4
+    retain_bytes = int(w.seq_lens.sum().item()) * w.H_kv * 4 + ki.size * 4
+    peak, peak_kind = measured_peak()
+    cb = None if args.no_cpu_baseline else h2o_oracle_time(w, budget, recent)
+    gbs = compact_bytes / (compact_us * 1e-6) / 1e9
+    print(json.dumps({
+        "metric": "h2o_evict_us_per_step", "value": step_us, "unit": "us", "n_gpus": 1, "steps": K,
+        "warmup": args.warmup, "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H_kv": w.H_kv, "D": w.D, "cached_tokens": 5120,
+                   "budget_tokens": budget, "recent_tokens": recent, "moved_pages": moved_pages,
+                   "l2": "inputs larger than L2 (%d MB moved per step)" % (compact_bytes // 10**6)},
+        "calls_us": {"se_h2o_retain": retain_us, "se_h2o_compact": compact_us},
+        "algorithmic_bytes": {"se_h2o_retain": retain_bytes, "se_h2o_compact": compact_bytes},
+        "roofline": {"bound": "hbm", "kernel": "h2o_compact_kernel (se_h2o_compact)", "achieved": gbs, "peak": peak,
+                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": gbs / peak,
+                     "traffic": H2O_NCU_TRAFFIC_BYTES if w.B == 64 else None,
+                     "algorithmic_bytes": compact_bytes},
+        "clocks": sampler.summary(t0, t1),
+        "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": w.B * 4, "d2h_bytes_per_step": w.B * 4},
+        "gpu_launches": 2 * K, "cpu_baseline": cb}))
 
 
 def run_reference(args, n_layers):
