@@ -215,6 +215,69 @@ def h2o_compact(k_cache, v_cache, u_accum, page_table, keep_idx, keep_cnt):
     return k, v, u, new_lens
 
 
+def token_scores(q, k_cache, page_table, seq_lens, page_size=16, sm_scale=None):
+    """Observation-layer selector: returns (s [B, max_pages*p] = max over query heads of the logit,
+    present [B, max_pages*p] bool)."""
+    q = _u16(q)
+    k_cache = _u16(k_cache)
+    B, H_q, D = q.shape
+    _, H_kv, p, _ = k_cache.shape
+    assert p == page_size
+    page_table = _i32(page_table)
+    seq_lens = _i32(seq_lens)
+    max_pages = page_table.shape[1]
+    s = np.zeros((B, max_pages * p), dtype=np.float64)
+    present = np.zeros((B, max_pages * p), dtype=np.uint8)
+    scale = default_scale(D) if sm_scale is None else float(sm_scale)
+    _load().se_oracle_token_scores(B, H_q, H_kv, D, p, max_pages, ctypes.c_double(scale),
+                                   _p(q, ctypes.c_uint16), _p(k_cache, ctypes.c_uint16),
+                                   _p(page_table, ctypes.c_int32), _p(seq_lens, ctypes.c_int32),
+                                   _p(s, ctypes.c_double), _p(present, ctypes.c_uint8))
+    return s, present.astype(bool)
+
+
+def token_topk(s, present, seq_lens, budget, recent=0, n_out=None):
+    """Returns (tok_idx [B, n_out] ascending / -1 padded, tok_cnt [B], theta [B])."""
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    pres = np.ascontiguousarray(present, dtype=np.uint8)
+    B, n_max = s.shape
+    seq_lens = _i32(seq_lens)
+    if n_out is None:
+        n_out = int(budget) + int(recent)
+    tok_idx = np.full((B, n_out), -1, dtype=np.int32)
+    tok_cnt = np.zeros((B,), dtype=np.int32)
+    theta = np.zeros((B,), dtype=np.float64)
+    _load().se_oracle_token_topk(B, n_max, int(n_out), int(budget), int(recent), _p(s, ctypes.c_double),
+                                 _p(pres, ctypes.c_uint8), _p(seq_lens, ctypes.c_int32),
+                                 _p(tok_idx, ctypes.c_int32), _p(tok_cnt, ctypes.c_int32),
+                                 _p(theta, ctypes.c_double))
+    return tok_idx, tok_cnt, theta
+
+
+def token_attend(q, k_cache, v_cache, page_table, seq_lens, tok_idx, tok_cnt, page_size=16, sm_scale=None):
+    """Attention of every query head over one token set per request: (out [B,H_q,D], lse [B,H_q])."""
+    q = _u16(q)
+    k_cache = _u16(k_cache)
+    v_cache = _u16(v_cache)
+    B, H_q, D = q.shape
+    _, H_kv, p, _ = k_cache.shape
+    assert p == page_size
+    page_table = _i32(page_table)
+    seq_lens = _i32(seq_lens)
+    tok_idx = _i32(tok_idx)
+    tok_cnt = _i32(tok_cnt)
+    max_pages = page_table.shape[1]
+    out = np.zeros((B, H_q, D), dtype=np.float64)
+    lse = np.zeros((B, H_q), dtype=np.float64)
+    scale = default_scale(D) if sm_scale is None else float(sm_scale)
+    _load().se_oracle_token_attend(B, H_q, H_kv, D, p, max_pages, tok_idx.shape[1], ctypes.c_double(scale),
+                                   _p(q, ctypes.c_uint16), _p(k_cache, ctypes.c_uint16),
+                                   _p(v_cache, ctypes.c_uint16), _p(page_table, ctypes.c_int32),
+                                   _p(seq_lens, ctypes.c_int32), _p(tok_idx, ctypes.c_int32),
+                                   _p(tok_cnt, ctypes.c_int32), _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    return out, lse
+
+
 def decode_step(q, k_cache, v_cache, page_table, seq_lens, budget, meta=None,
                 page_size=16, sm_scale=None, u_accum=None, k_max=None, sink_pages=0, recent_pages=0):
     """One decode step: summary of the newest page, scores, top-k, attention."""

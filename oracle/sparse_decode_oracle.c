@@ -16,6 +16,9 @@
  *                      + H2O accumulated score         (Appendix A, H2O score eq.)
  *   se_oracle_h2o_retain   H2O retained set R = W u TopK(u; A \ W)   (Appendix A, H2O retention eq.)
  *   se_oracle_h2o_compact  eviction: retained tokens moved to the front of the request's cache
+ *   se_oracle_token_scores observation-layer selector s(j) = max_a z_j^(a)   (Appendix A, OmniKV selection eq.)
+ *   se_oracle_token_topk   J = TopK_b(s; [i]) plus the always-kept recent tokens
+ *   se_oracle_token_attend attention of every head over one token set per request (OmniKV reuse eq.)
  *
  * Conventions (0-based everywhere; the paper's positions are 1-based):
  *   logical page b of request r holds tokens [b*p, min(len_r, (b+1)*p)); its physical
@@ -394,4 +397,138 @@ void se_oracle_h2o_compact(int B, int H_kv, int D, int p, int max_pages, int P, 
     free(k0);
     free(v0);
     free(u0);
+}
+
+/*
+ * Observation-layer selector (Appendix A, "OmniKV: Selection Reuse across Layers", selection
+ * equation): for request r and token j < len_r whose page is present,
+ *     s[r,j] = max over all query heads a of  z_j^(a) = sm_scale * sum_c q[r,a,c] k[j,g(a),c];
+ * tokens that are absent (or lie past the length) get present = 0 and s = 0.
+ *   s [B, max_pages*p]   present [B, max_pages*p]
+ */
+void se_oracle_token_scores(int B, int H_q, int H_kv, int D, int p, int max_pages, double sm_scale,
+                            const uint16_t *q, const uint16_t *k_cache, const int32_t *page_table,
+                            const int32_t *seq_lens, double *s, uint8_t *present) {
+    const int G = H_q / H_kv, n_max = max_pages * p;
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < B; ++r) {
+        int len = seq_lens[r];
+        if (len > n_max) len = n_max;
+        for (int j = 0; j < n_max; ++j) {
+            s[(size_t)r * n_max + j] = 0.0;
+            present[(size_t)r * n_max + j] = 0;
+            if (j >= len) continue;
+            const int pid = page_table[(size_t)r * max_pages + j / p];
+            if (pid < 0) continue;
+            double best = -INFINITY;
+            for (int a = 0; a < H_q; ++a) {
+                const uint16_t *qa = q + ((size_t)r * H_q + a) * D;
+                const uint16_t *kt = k_cache + ((((size_t)pid * H_kv + a / G) * p) + j % p) * D;
+                double z = 0.0;
+                for (int c = 0; c < D; ++c) z += bf16_to_f64(qa[c]) * bf16_to_f64(kt[c]);
+                z *= sm_scale;
+                if (z > best) best = z;
+            }
+            s[(size_t)r * n_max + j] = best;
+            present[(size_t)r * n_max + j] = 1;
+        }
+    }
+}
+
+/*
+ * Token selection of an observation layer: J = TopK_b(s; present tokens), equal scores to the
+ * lower position; the last `recent` positions of the request (when present) are always in the
+ * result and do not count against b (the paper's OmniKV settings list "selected" and "recent"
+ * tokens separately).  tok_idx[r,:] = the set in ascending position, -1 padded to n_out entries;
+ * theta[r] = the score of the last token taken by rank (NaN if none competes).
+ */
+void se_oracle_token_topk(int B, int n_max, int n_out, int budget, int recent, const double *s,
+                          const uint8_t *present, const int32_t *seq_lens, int32_t *tok_idx,
+                          int32_t *tok_cnt, double *theta) {
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < B; ++r) {
+        int len = seq_lens[r];
+        if (len > n_max) len = n_max;
+        if (len < 0) len = 0;
+        int32_t *row = tok_idx + (size_t)r * n_out;
+        for (int i = 0; i < n_out; ++i) row[i] = -1;
+        tok_t *cand = (tok_t *)malloc(sizeof(tok_t) * (size_t)(len > 0 ? len : 1));
+        int *kept = (int *)malloc(sizeof(int) * (size_t)(n_out > 0 ? n_out : 1));
+        int n_cand = 0, n_kept = 0;
+        for (int j = 0; j < len; ++j) {
+            if (!present[(size_t)r * n_max + j]) continue;
+            if (j >= len - recent) {
+                if (n_kept < n_out) kept[n_kept++] = j;
+            } else {
+                cand[n_cand].u = s[(size_t)r * n_max + j];
+                cand[n_cand].pos = j;
+                ++n_cand;
+            }
+        }
+        int k = budget < n_cand ? budget : n_cand;
+        if (k > n_out - n_kept) k = n_out - n_kept;
+        qsort(cand, (size_t)n_cand, sizeof(tok_t), tok_cmp);
+        theta[r] = k > 0 ? cand[k - 1].u : NAN;
+        for (int i = 0; i < k; ++i) kept[n_kept++] = cand[i].pos;
+        qsort(kept, (size_t)n_kept, sizeof(int), int_cmp);
+        for (int i = 0; i < n_kept; ++i) row[i] = kept[i];
+        tok_cnt[r] = n_kept;
+        free(cand);
+        free(kept);
+    }
+}
+
+/*
+ * Attention of a sparse layer that reuses an observation layer's token set (Appendix A, OmniKV
+ * reuse equation): every query head a of request r attends the tokens tok_idx[r,0..tok_cnt[r])
+ * of this layer's own cache,
+ *     out = sum_{j in I} alpha_j v_j^(g(a)),  alpha = softmax over I of sm_scale * q_a . k_j^(g(a)),
+ * lse = ln sum_{j in I} exp(z_j).  Tokens whose page is absent or that lie past the length are
+ * skipped; an empty set gives out = 0, lse = -inf.
+ */
+void se_oracle_token_attend(int B, int H_q, int H_kv, int D, int p, int max_pages, int n_out,
+                            double sm_scale, const uint16_t *q, const uint16_t *k_cache,
+                            const uint16_t *v_cache, const int32_t *page_table, const int32_t *seq_lens,
+                            const int32_t *tok_idx, const int32_t *tok_cnt, double *out, double *lse) {
+    const int G = H_q / H_kv;
+#pragma omp parallel for schedule(dynamic)
+    for (int ra = 0; ra < B * H_q; ++ra) {
+        const int r = ra / H_q, a = ra % H_q, h = a / G;
+        const int cnt = tok_cnt[r], len = seq_lens[r];
+        const uint16_t *qa = q + (size_t)ra * D;
+        double *o = out + (size_t)ra * D;
+        double *z = (double *)malloc(sizeof(double) * (size_t)(cnt > 0 ? cnt : 1));
+        double zmax = -INFINITY;
+        for (int c = 0; c < D; ++c) o[c] = 0.0;
+        for (int i = 0; i < cnt; ++i) {
+            const int j = tok_idx[(size_t)r * n_out + i];
+            z[i] = -INFINITY;
+            if (j < 0 || j >= len || j >= max_pages * p) continue;
+            const int pid = page_table[(size_t)r * max_pages + j / p];
+            if (pid < 0) continue;
+            const uint16_t *kt = k_cache + ((((size_t)pid * H_kv + h) * p) + j % p) * D;
+            double acc = 0.0;
+            for (int c = 0; c < D; ++c) acc += bf16_to_f64(qa[c]) * bf16_to_f64(kt[c]);
+            z[i] = acc * sm_scale;
+            if (z[i] > zmax) zmax = z[i];
+        }
+        if (!(zmax > -INFINITY)) {
+            lse[ra] = -INFINITY;
+            free(z);
+            continue;
+        }
+        double denom = 0.0;
+        for (int i = 0; i < cnt; ++i)
+            if (z[i] > -INFINITY) denom += exp(z[i] - zmax);
+        lse[ra] = zmax + log(denom);
+        for (int i = 0; i < cnt; ++i) {
+            if (!(z[i] > -INFINITY)) continue;
+            const int j = tok_idx[(size_t)r * n_out + i];
+            const int pid = page_table[(size_t)r * max_pages + j / p];
+            const uint16_t *vt = v_cache + ((((size_t)pid * H_kv + h) * p) + j % p) * D;
+            const double alpha = exp(z[i] - zmax) / denom;
+            for (int c = 0; c < D; ++c) o[c] += alpha * bf16_to_f64(vt[c]);
+        }
+        free(z);
+    }
 }
