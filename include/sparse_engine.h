@@ -245,6 +245,42 @@ int se_combine(const se_params *p, const void *q, const void *k_cache, const voi
                void *workspace, void *stream);
 
 /*
+ * Selection reuse across layers (Appendix A, "OmniKV: Selection Reuse across Layers").
+ *
+ * se_observe_decode - an observation (filter) layer: se_sparse_decode (normally with every page
+ * selected, i.e. full attention) that also leaves, for every attended token j of request r,
+ *     s[r,j] = max over all query heads a of the logit z_j^(a) = sm_scale * q_a . k_j      (selection eq.)
+ * in tok_keys ([B, 16*max_pages] uint32, device) as the order-preserving integer image of the fp32
+ * score: key = bits ^ 0xffffffff for negative values, bits | 0x80000000 otherwise; 0 = token not
+ * attended.  The call zeroes tok_keys itself (a memset on `stream`) before the kernel runs.
+ *
+ * se_token_select - J = TopK_b(s; attended tokens) per request, equal scores to the lower
+ * position, plus the attended tokens among the request's last recent_tokens positions, which are
+ * always kept and do not count against b (the paper's OmniKV settings list "selected" and
+ * "recent" tokens separately).  tok_idx[r,:] ([B, n_out] int32) receives the set in ascending
+ * position, -1 padded; tok_cnt[r] its size.  budget_tokens + recent_tokens <= n_out <= 2^20.
+ *
+ * se_token_decode - a sparse layer that reuses the set (reuse equation): every query head of
+ * request r attends the tokens tok_idx[r, 0..tok_cnt[r]) of THIS layer's k_cache / v_cache,
+ *     out = sum_j alpha_j v_j,   alpha = softmax over the set,   lse = ln sum_j exp(z_j).
+ * Tokens whose page is absent are skipped; tokens outside [0, seq_lens[r]) are skipped and
+ * reported through the status word; an empty set gives out = 0, lse = -inf.  Needs
+ * ceil(n_out / 16) <= k_max (the workspace holds one partial per 16-token tile group).
+ * All three are asynchronous on `stream` and allocate nothing.
+ */
+int se_observe_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                      const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+                      const int32_t *sel_cnt, float *out, float *lse, uint32_t *tok_keys,
+                      void *workspace, void *stream);
+int se_token_select(const se_params *p, const uint32_t *tok_keys, const int32_t *seq_lens,
+                    int32_t budget_tokens, int32_t recent_tokens, int32_t *tok_idx, int32_t *tok_cnt,
+                    int32_t n_out, void *workspace, void *stream);
+int se_token_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                    const int32_t *page_table, const int32_t *seq_lens, const int32_t *tok_idx,
+                    const int32_t *tok_cnt, int32_t n_out, float *out, float *lse, void *workspace,
+                    void *stream);
+
+/*
  * H2O retained set (Appendix A, "H2O: Accumulated Scores and Online Eviction", retention
  * equation).  For request r (seq_lens[r] tokens; token j lives in slot j % 16 of logical page
  * j / 16) and kv-head h, with u = score_accum as maintained by se_sparse_decode:

@@ -23,7 +23,8 @@ SE_DEV_WAIT_TIMEOUT = 4
 EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_decode_num_splits", "se_workspace_init",
            "se_meta_update",
            "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
-           "se_last_device_status", "se_h2o_retain", "se_h2o_compact",
+           "se_last_device_status", "se_h2o_retain", "se_h2o_compact", "se_observe_decode", "se_token_select",
+           "se_token_decode",
            "se_page_select_static")
 SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
@@ -73,12 +74,16 @@ def load(build_if_missing: bool = True):
     lib.se_sparse_decode_splits.argtypes = lib.se_sparse_decode.argtypes
     lib.se_combine.argtypes = lib.se_sparse_decode.argtypes
     lib.se_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.se_observe_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, fp, fp, vp, vp, vp]
+    lib.se_token_select.argtypes = [pp, vp, i32p, ctypes.c_int32, ctypes.c_int32, i32p, i32p, ctypes.c_int32, vp, vp]
+    lib.se_token_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, ctypes.c_int32, fp, fp, vp, vp]
     lib.se_h2o_retain.argtypes = [pp, fp, i32p, i32p, ctypes.c_int32, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_h2o_compact.argtypes = [pp, vp, vp, fp, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp]
     lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
                  "se_sparse_decode", "se_sparse_decode_splits", "se_combine", "se_last_device_status",
-                 "se_h2o_retain", "se_h2o_compact", "se_decode_num_splits", "se_page_select_static"):
+                 "se_h2o_retain", "se_h2o_compact", "se_decode_num_splits", "se_page_select_static",
+                 "se_observe_decode", "se_token_select", "se_token_decode"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -206,6 +211,44 @@ def se_page_select_static(p, q, meta, page_table, seq_lens, budget_tokens, sel_i
                                         _ptr(sel_cnt, torch.int32, "sel_cnt"),
                                         _ptr(dev_status, torch.int32, "dev_status"), _stream()),
            "se_page_select_static")
+
+
+def se_observe_decode(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse, tok_keys,
+                      workspace) -> None:
+    _check(load().se_observe_decode(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                    _ptr(k_cache, torch.bfloat16, "k_cache"), _ptr(v_cache, torch.bfloat16, "v_cache"),
+                                    _ptr(page_table, torch.int32, "page_table"), _ptr(seq_lens, torch.int32, "seq_lens"),
+                                    _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                    _ptr(out, torch.float32, "out"), _ptr(lse, torch.float32, "lse"),
+                                    _ptr(tok_keys, torch.int32, "tok_keys"),
+                                    _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_observe_decode")
+
+
+def se_token_select(p, tok_keys, seq_lens, budget_tokens, recent_tokens, tok_idx, tok_cnt, workspace) -> None:
+    _check(load().se_token_select(ctypes.byref(p), _ptr(tok_keys, torch.int32, "tok_keys"),
+                                  _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens), int(recent_tokens),
+                                  _ptr(tok_idx, torch.int32, "tok_idx"), _ptr(tok_cnt, torch.int32, "tok_cnt"),
+                                  int(tok_idx.shape[-1]), _ptr(workspace, torch.uint8, "workspace"), _stream()),
+           "se_token_select")
+
+
+def se_token_decode(p, q, k_cache, v_cache, page_table, seq_lens, tok_idx, tok_cnt, out, lse, workspace) -> None:
+    _check(load().se_token_decode(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                  _ptr(k_cache, torch.bfloat16, "k_cache"), _ptr(v_cache, torch.bfloat16, "v_cache"),
+                                  _ptr(page_table, torch.int32, "page_table"), _ptr(seq_lens, torch.int32, "seq_lens"),
+                                  _ptr(tok_idx, torch.int32, "tok_idx"), _ptr(tok_cnt, torch.int32, "tok_cnt"),
+                                  int(tok_idx.shape[-1]), _ptr(out, torch.float32, "out"),
+                                  _ptr(lse, torch.float32, "lse"), _ptr(workspace, torch.uint8, "workspace"),
+                                  _stream()), "se_token_decode")
+
+
+def keys_to_scores(tok_keys):
+    """Inverse of the order-preserving integer image used by se_observe_decode: int32 tensor of keys ->
+    (float32 scores, bool attended)."""
+    k = tok_keys.to(torch.int64) & 0xFFFFFFFF
+    bits = torch.where(k >= 0x80000000, k & 0x7FFFFFFF, (~k) & 0xFFFFFFFF)
+    bits = torch.where(bits >= 0x80000000, bits - (1 << 32), bits).to(torch.int32)
+    return bits.view(torch.float32), k != 0
 
 
 def se_h2o_retain(p, score_accum, page_table, seq_lens, budget_tokens, recent_tokens, keep_idx, keep_cnt,

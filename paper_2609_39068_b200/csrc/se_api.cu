@@ -182,7 +182,7 @@ int se_page_select_fused(const se_params *p, const void *q, const void *k_cache,
 static int sparse_decode_stages(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
                                 const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
                                 const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                                void *workspace, int stages, void *stream) {
+                                uint32_t *tok_keys, void *workspace, int stages, void *stream) {
     int rc = validate(p);
     if (rc != SE_OK) return rc;
     if (!q || !k_cache || !v_cache || !page_table || !seq_lens || !sel_idx || !sel_cnt || !out ||
@@ -193,8 +193,14 @@ static int sparse_decode_stages(const se_params *p, const void *q, const void *k
         !aligned16(lse) || !aligned16(score_accum) || !aligned16(workspace))
         return SE_ERR_MISALIGNED;
     const WorkspaceLayout L = make_layout(*p);
+    if (tok_keys) {
+        if (!aligned16(tok_keys)) return SE_ERR_MISALIGNED;
+        if (cudaMemsetAsync(tok_keys, 0, (size_t)p->B * p->max_pages * kPage * sizeof(uint32_t),
+                            static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return SE_ERR_CUDA;
+    }
     cudaError_t e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens, sel_idx,
-                                         sel_cnt, out, lse, score_accum, workspace, L, stages,
+                                         sel_cnt, out, lse, score_accum, tok_keys, workspace, L, stages,
                                          static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
 }
@@ -204,7 +210,16 @@ int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, con
                      const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
                      void *workspace, void *stream) {
     return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-                                score_accum, workspace, 3, stream);
+                                score_accum, nullptr, workspace, 3, stream);
+}
+
+int se_observe_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                      const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
+                      const int32_t *sel_cnt, float *out, float *lse, uint32_t *tok_keys, void *workspace,
+                      void *stream) {
+    if (!tok_keys) return SE_ERR_NULL_POINTER;
+    return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
+                                nullptr, tok_keys, workspace, 3, stream);
 }
 
 int se_sparse_decode_splits(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
@@ -212,7 +227,7 @@ int se_sparse_decode_splits(const se_params *p, const void *q, const void *k_cac
                             const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
                             void *workspace, void *stream) {
     return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-                                score_accum, workspace, 1, stream);
+                                score_accum, nullptr, workspace, 1, stream);
 }
 
 int se_combine(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
@@ -220,7 +235,45 @@ int se_combine(const se_params *p, const void *q, const void *k_cache, const voi
                const int32_t *sel_cnt, float *out, float *lse, float *score_accum, void *workspace,
                void *stream) {
     return sparse_decode_stages(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-                                score_accum, workspace, 2, stream);
+                                score_accum, nullptr, workspace, 2, stream);
+}
+
+int se_token_select(const se_params *p, const uint32_t *tok_keys, const int32_t *seq_lens, int32_t budget_tokens,
+                    int32_t recent_tokens, int32_t *tok_idx, int32_t *tok_cnt, int32_t n_out, void *workspace,
+                    void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!tok_keys || !seq_lens || !tok_idx || !tok_cnt || !workspace) return SE_ERR_NULL_POINTER;
+    if (!aligned16(tok_keys) || !aligned16(seq_lens) || !aligned16(tok_idx) || !aligned16(tok_cnt) ||
+        !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    if (budget_tokens < 0 || recent_tokens < 0 || n_out < 1 || n_out > (1 << 20) ||
+        (long long)budget_tokens + recent_tokens > n_out)
+        return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_token_select(*p, tok_keys, seq_lens, budget_tokens, recent_tokens, n_out, tok_idx, tok_cnt,
+                                        reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + L.status),
+                                        static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_token_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,
+                    const int32_t *page_table, const int32_t *seq_lens, const int32_t *tok_idx,
+                    const int32_t *tok_cnt, int32_t n_out, float *out, float *lse, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!q || !k_cache || !v_cache || !page_table || !seq_lens || !tok_idx || !tok_cnt || !out || !lse || !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(page_table) ||
+        !aligned16(seq_lens) || !aligned16(tok_idx) || !aligned16(tok_cnt) || !aligned16(out) || !aligned16(lse) ||
+        !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    // the workspace is sized for k_max units per pair; a unit here is a 16-token tile
+    if (n_out < 1 || (n_out + kPage - 1) / kPage > p->k_max) return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaError_t e = launch_token_decode(*p, q, k_cache, v_cache, page_table, seq_lens, tok_idx, tok_cnt, n_out, out,
+                                        lse, workspace, L, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
 }
 
 int se_h2o_retain(const se_params *p, const float *score_accum, const int32_t *page_table,

@@ -88,7 +88,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
               const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
               const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ sel_idx,
               const int32_t *__restrict__ sel_cnt, float *__restrict__ out, float *__restrict__ lse,
-              float *__restrict__ partials, float *__restrict__ zbuf,
+              float *__restrict__ partials, float *__restrict__ zbuf, uint32_t *__restrict__ tok_keys,
               int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
               int max_splits, float scale_log2, uint32_t *status) {
     using C = DecCfg<D>;
@@ -142,9 +142,11 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     // look-ups, across pair boundaries.
     //   ent_y    row of the page's first token in the [pages*heads*16, D] view of the cache
     //   ent_info valid tokens (bits 0-4) | selection index i (bits 5-16) | slot - chunk_base (bits 17-23)
+    //   ent_b    logical page (only read by an observation layer)
     int *ent_y = reinterpret_cast<int *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8) +
-                 warp * 2 * kChunk;
+                 warp * 3 * kChunk;
     int *ent_info = ent_y + kChunk;
+    int *ent_b = ent_info + kChunk;
     int chunk_base = 0, chunk_end = 0;           // slots [chunk_base, chunk_end) are in the list
     int n_ent = 0, ce = 0, pe = 0;               // entries, next to consume, next to issue
 
@@ -153,11 +155,11 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         chunk_end = min(x_end, base + kChunk);
         const int pair0 = base / k_max;
         const int i0 = base - pair0 * k_max;
-        int sl_pid[kChunk / 32], sl_meta[kChunk / 32];
+        int sl_pid[kChunk / 32], sl_meta[kChunk / 32], sl_b[kChunk / 32];
 #pragma unroll
         for (int rep = 0; rep < kChunk / 32; ++rep) {
             const int off = rep * 32 + lane;
-            int pid = -1, meta = 0;
+            int pid = -1, meta = 0, lb = 0;
             if (base + off < chunk_end) {
                 const int dp = (i0 + off) / k_max;
                 const int pair = pair0 + dp;
@@ -173,12 +175,14 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                         atomicOr(status, SE_DEV_BAD_SELECTION);
                     } else {
                         pid = __ldg(page_table + (size_t)r * max_pages + b);
+                        lb = b;
                         meta = min(kPage, len - b * kPage) | (i << 5) | (off << 17) | (hh << 24);
                     }
                 }
             }
             sl_pid[rep] = pid;
             sl_meta[rep] = meta;
+            sl_b[rep] = lb;
         }
         int count = 0;
 #pragma unroll
@@ -196,6 +200,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 const int pos = count + __popc(vm & ((1u << lane) - 1u));
                 ent_y[pos] = (pid * H_kv + (sl_meta[rep] >> 24)) * kPage;
                 ent_info[pos] = sl_meta[rep] & 0x00ffffff;
+                ent_b[pos] = sl_b[rep];
             }
             count += __popc(vm);
         }
@@ -330,6 +335,38 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 zp[(t0 + 8) * GP] = z[2];
                 zp[(t0 + 9) * GP] = z[3];
             }
+            if (tok_keys != nullptr) {
+                // observation layer: s(j) = max over every query head of the logit (Appendix A, OmniKV
+                // selection equation).  Here: max over the group's heads (rows gid), then an atomic
+                // max over the kv-heads on the order-preserving integer image of the score.
+                float m4[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float v = head_ok ? z[e] : -INFINITY;
+                    v = fmaxf(v, __shfl_xor_sync(kFull, v, 4));
+                    v = fmaxf(v, __shfl_xor_sync(kFull, v, 8));
+                    v = fmaxf(v, __shfl_xor_sync(kFull, v, 16));
+                    m4[e] = v;
+                }
+                if (gid == 0) {
+                    uint32_t *kp = tok_keys + (size_t)r * max_pages * kPage + ent_b[ce] * kPage;
+                    if (m4[0] > -INFINITY) atomicMax(kp + t0, f32_key(m4[0] * kLn2));
+                    if (m4[1] > -INFINITY) atomicMax(kp + t0 + 1, f32_key(m4[1] * kLn2));
+                    if (m4[2] > -INFINITY) atomicMax(kp + t0 + 8, f32_key(m4[2] * kLn2));
+                    if (m4[3] > -INFINITY) atomicMax(kp + t0 + 9, f32_key(m4[3] * kLn2));
+                }
+            }
+            if (nv_j < kPage) {
+                // slots past the request's length may hold anything (NaN included): their weights are
+                // zero, so their V rows are cleared in shared memory before the product
+                for (int idx = lane; idx < (kPage - nv_j) * C::HALVES * 8; idx += 32) {
+                    const int row = nv_j + idx / (C::HALVES * 8);
+                    const int rem = idx % (C::HALVES * 8);
+                    const uint32_t addr = Vs + (rem >> 3) * kTileBytes + row * 128 + (rem & 7) * 16;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                }
+                __syncwarp();
+            }
             float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
             pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
             pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
@@ -437,14 +474,15 @@ combine_kernel(const float *__restrict__ partials, const float *__restrict__ zbu
                const int32_t *__restrict__ sel_idx, const int32_t *__restrict__ sel_cnt,
                float *__restrict__ out, float *__restrict__ lse, float *__restrict__ score_accum,
                int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
-               int max_splits) {
+               int max_splits, const int32_t *__restrict__ tok_cnt) {
     constexpr int PSTRIDE = D + 4;
     __shared__ float s_lse2[8];
     const int pair = blockIdx.x;
     const int r = pair / H_kv, h = pair % H_kv;
     const int H_q = H_kv * G;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int cnt = min(sel_cnt[pair], k_max);
+    // token-granular decode (tok_cnt != NULL): the units are 16-token tiles of the request's token list
+    const int cnt = tok_cnt ? min((tok_cnt[r] + kPage - 1) / kPage, k_max) : min(sel_cnt[pair], k_max);
     const int len = seq_lens[r];
     const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
     const bool nothing = cnt <= 0 || n_r == 0;
@@ -559,7 +597,7 @@ bool make_page_map(CUtensorMap *map, const void *base, const se_params &p) {
 template <int D>
 cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache, const void *v_cache,
                           const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
-                          const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                          const int32_t *sel_cnt, float *out, float *lse, float *score_accum, uint32_t *tok_keys,
                           void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream) {
     using C = DecCfg<D>;
     const DecodePlan plan = make_decode_plan(p);
@@ -571,13 +609,13 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     CUtensorMap k_map, v_map;
     if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
     const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
-                        (size_t)kDecWarps * 2 * kChunk * sizeof(int) + 1024;
+                        (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 1024;
     auto kern = decode_kernel<D>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
         k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-        reinterpret_cast<float *>(ws + L.partials), zbuf,
+        reinterpret_cast<float *>(ws + L.partials), zbuf, tok_keys,
         p.B, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
         effective_scale(p) * kLog2e, reinterpret_cast<uint32_t *>(ws + L.status));
     e = cudaGetLastError();
@@ -590,10 +628,311 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     const int slot_ctas = score_accum ? (p.k_max * kPage + 511) / 512 : 1;
     combine_kernel<D><<<dim3(p.B * p.H_kv, slot_ctas), 256, 0, stream>>>(
         reinterpret_cast<const float *>(ws + L.partials), zbuf, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-        score_accum, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits);
+        score_accum, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
+        nullptr);
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------
+// token_decode_kernel: attention of a sparse layer over a token set handed down by an observation
+// layer (Appendix A, OmniKV reuse equation): all kv-heads of request r read the tokens
+// tok_idx[r, 0..tok_cnt[r]) of this layer's own cache.  Same structure as decode_kernel - one
+// (pair, split) unit per warp, stages shared out among the busy warps, MMA on ldmatrix fragments,
+// online softmax - but a tile is 16 tokens from anywhere: 16 K rows and 16 V rows of D*2 bytes,
+// fetched with one 1-D bulk copy each (lanes 0-15 the K rows, lanes 16-31 the V rows) into rows
+// padded by 16 bytes (conflict-free ldmatrix without hardware swizzle).  Tokens that are out of
+// range or whose page is absent are skipped (their columns are masked, their V rows cleared).
+// ---------------------------------------------------------------------------------
+template <int D>
+struct TokCfg {
+    static constexpr int ROWB = D * 2;                         // bytes of one K or V row
+    static constexpr int PITCH = ROWB + 16;
+    static constexpr int TILEB = kPage * PITCH;                // K (or V) rows of one tile
+    static constexpr int STAGEB = 2 * TILEB;
+    static constexpr int MAXST = 8;
+    static constexpr int CTA_STAGES = 20 * (128 / D);
+    static constexpr int KSTEPS = D / 16;
+    static constexpr int NTILES = D / 8;
+    static constexpr int PSTRIDE = D + 4;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDecWarps * 32, 1)
+token_decode_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ k_cache,
+                    const uint8_t *__restrict__ v_cache, const int32_t *__restrict__ page_table,
+                    const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ tok_idx,
+                    const int32_t *__restrict__ tok_cnt, float *__restrict__ out, float *__restrict__ lse,
+                    float *__restrict__ partials, int B, int H_kv, int G, int max_pages, int P_phys, int n_out,
+                    int tiles_per_split, int max_splits, float scale_log2, uint32_t *status) {
+    using C = TokCfg<D>;
+    extern __shared__ __align__(128) uint8_t smem_tok[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_units = B * H_kv * max_splits;
+    int busy = (n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    busy = busy < 1 ? 1 : (busy > kDecWarps ? kDecWarps : busy);
+    const int nstage = warp < busy ? min(C::MAXST, C::CTA_STAGES / busy) : 0;
+    uint8_t *ring = smem_tok + (size_t)(warp * nstage) * C::STAGEB;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_tok + (size_t)C::CTA_STAGES * C::STAGEB) + warp * C::MAXST;
+    int *ent_row = reinterpret_cast<int *>(smem_tok + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8) +
+                   warp * kChunk;
+    if (lane == 0) {
+        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    const uint32_t ring0 = smem_u32(ring);
+    const int H_q = H_kv * G;
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const bool head_ok = gid < G;
+    const int gw = warp * gridDim.x + blockIdx.x;
+    const int warps_total = kDecWarps * gridDim.x;
+    const int k_row = (lane & 7) + 8 * (lane >> 4);
+    const int k_chunk_add = (lane >> 3) & 1;
+    const int v_row = (lane & 7) + 8 * ((lane >> 3) & 1);
+    const int v_chunk_add = lane >> 4;
+    uint32_t phases = 0;
+    int stage_c = 0, stage_i = 0;
+    bool failed = false;
+
+    for (int unit = gw; unit < n_units && !failed; unit += warps_total) {
+        const int pair = unit / max_splits;
+        const int my_split = unit - pair * max_splits;
+        const int r = pair / H_kv, h = pair % H_kv;
+        const int len = min(__ldg(seq_lens + r), max_pages * kPage);
+        int cnt = __ldg(tok_cnt + r);
+        if (cnt > n_out) {
+            if (lane == 0) atomicOr(status, SE_DEV_BAD_SELECTION);
+            cnt = n_out;
+        }
+        const int tiles = cnt > 0 ? (cnt + kPage - 1) / kPage : 0;
+        const int n_split = (tiles + tiles_per_split - 1) / tiles_per_split;
+        if (tiles == 0 || len <= 0) {
+            if (my_split == 0) {
+                for (int g = 0; g < G; ++g) {
+                    float *o = out + ((size_t)r * H_q + h * G + g) * D;
+                    for (int c = lane; c < D; c += 32) o[c] = 0.f;
+                    if (lane == 0) lse[(size_t)r * H_q + h * G + g] = -INFINITY;
+                }
+            }
+            continue;
+        }
+        if (my_split >= n_split) continue;
+        const int e_lo = my_split * tiles_per_split * kPage;                       // entries of this unit
+        const int e_hi = min(cnt, (my_split + 1) * tiles_per_split * kPage);
+
+        uint32_t qa[C::KSTEPS][2];
+        {
+            const uint16_t *src = q + ((size_t)r * H_q + h * G + (head_ok ? gid : 0)) * D + 2 * tid4;
+#pragma unroll
+            for (int s = 0; s < C::KSTEPS; ++s) {
+                const uint32_t w0 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16));
+                const uint32_t w1 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16 + 8));
+                qa[s][0] = head_ok ? w0 : 0u;
+                qa[s][1] = head_ok ? w1 : 0u;
+            }
+        }
+        float o_acc[C::NTILES][4];
+#pragma unroll
+        for (int nt = 0; nt < C::NTILES; ++nt) {
+            o_acc[nt][0] = 0.f; o_acc[nt][1] = 0.f; o_acc[nt][2] = 0.f; o_acc[nt][3] = 0.f;
+        }
+        float m_run = -INFINITY, l_run = 0.f;
+
+        for (int c_lo = e_lo; c_lo < e_hi && !failed; c_lo += kChunk) {
+            // ---- row list of up to kChunk tokens: token -> page table -> row of the [pages*heads*16, D] view
+            const int c_hi = min(e_hi, c_lo + kChunk);
+            const int n_tiles = (c_hi - c_lo + kPage - 1) / kPage;
+#pragma unroll
+            for (int rep = 0; rep < kChunk / 32; ++rep) {
+                const int off = rep * 32 + lane;
+                int row = -1;
+                if (c_lo + off < c_hi) {
+                    const int tok = __ldg(tok_idx + (size_t)r * n_out + c_lo + off);
+                    if (tok < 0 || tok >= len) {
+                        atomicOr(status, SE_DEV_BAD_SELECTION);
+                    } else {
+                        const int pid = __ldg(page_table + (size_t)r * max_pages + (tok >> 4));
+                        if (pid >= P_phys) atomicOr(status, SE_DEV_BAD_PAGE_ID);
+                        else if (pid >= 0) row = (pid * H_kv + h) * kPage + (tok & 15);
+                    }
+                }
+                ent_row[off] = row;
+            }
+            __syncwarp();
+            int ce = 0, pe = 0;                      // tiles of this chunk consumed / issued
+            auto top_up = [&]() {
+                while (pe < n_tiles && pe < ce + nstage) {
+                    const int row = ent_row[pe * kPage + (lane & 15)];
+                    const unsigned vm = __ballot_sync(kFull, row >= 0);
+                    const uint32_t bar = bar0 + stage_i * 8;
+                    if (lane == 0) mbar_expect_tx(bar, (uint32_t)__popc(vm) * C::ROWB);
+                    __syncwarp();
+                    if (row >= 0) {
+                        const uint32_t dst = ring0 + stage_i * C::STAGEB + (lane >> 4) * C::TILEB + (lane & 15) * C::PITCH;
+                        bulk_g2s(dst, (lane < 16 ? k_cache : v_cache) + (size_t)row * C::ROWB, C::ROWB, bar);
+                    }
+                    stage_i = (stage_i + 1 == nstage) ? 0 : stage_i + 1;
+                    ++pe;
+                }
+            };
+            top_up();
+            while (ce < n_tiles) {
+                if (!mbar_wait(bar0 + stage_c * 8, (phases >> stage_c) & 1u)) {
+                    failed = true;
+                    break;
+                }
+                phases ^= (1u << stage_c);
+                const uint32_t Ks = ring0 + stage_c * C::STAGEB;
+                const uint32_t Vs = Ks + C::TILEB;
+                stage_c = (stage_c + 1 == nstage) ? 0 : stage_c + 1;
+                const unsigned vmask = __ballot_sync(kFull, ent_row[ce * kPage + (lane & 15)] >= 0) & 0xffffu;
+                if (vmask == 0u) {                        // nothing to attend in this tile
+                    ++ce;
+                    top_up();
+                    continue;
+                }
+                if (vmask != 0xffffu) {
+                    // skipped tokens: whatever the stage held before must not reach the product
+                    for (int idx = lane; idx < kPage * (C::ROWB / 16); idx += 32) {
+                        const int row = idx / (C::ROWB / 16);
+                        if (!((vmask >> row) & 1u))
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(Vs + row * C::PITCH + (idx % (C::ROWB / 16)) * 16), "r"(0u) : "memory");
+                    }
+                    __syncwarp();
+                }
+                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                float s0b[4] = {0.f, 0.f, 0.f, 0.f}, s1b[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int s = 0; s < C::KSTEPS; ++s) {
+                    uint32_t b00, b01, b10, b11;
+                    ldmatrix_x4(Ks + k_row * C::PITCH + ((2 * s + k_chunk_add) << 4), b00, b01, b10, b11);
+                    if (s & 1) {
+                        mma_bf16_16816(s0b, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                        mma_bf16_16816(s1b, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+                    } else {
+                        mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                        mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+                    }
+                }
+                s0[0] += s0b[0]; s0[1] += s0b[1]; s1[0] += s1b[0]; s1[1] += s1b[1];
+                const int t0 = 2 * tid4;
+                float z[4];
+                z[0] = ((vmask >> t0) & 1u) ? s0[0] * scale_log2 : -INFINITY;
+                z[1] = ((vmask >> (t0 + 1)) & 1u) ? s0[1] * scale_log2 : -INFINITY;
+                z[2] = ((vmask >> (t0 + 8)) & 1u) ? s1[0] * scale_log2 : -INFINITY;
+                z[3] = ((vmask >> (t0 + 9)) & 1u) ? s1[1] * scale_log2 : -INFINITY;
+                float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+                pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
+                pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
+                const float m_new = fmaxf(m_run, pmax);           // finite: the tile has a valid token
+                const float corr = exp2f(m_run - m_new);
+                if (__any_sync(kFull, m_new != m_run)) {
+                    l_run *= corr;
+#pragma unroll
+                    for (int nt = 0; nt < C::NTILES; ++nt) {
+                        o_acc[nt][0] *= corr; o_acc[nt][1] *= corr; o_acc[nt][2] *= corr; o_acc[nt][3] *= corr;
+                    }
+                    m_run = m_new;
+                }
+                float pw[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) pw[e] = exp2f(z[e] - m_run);
+                l_run += (pw[0] + pw[1]) + (pw[2] + pw[3]);
+                const uint32_t ph0 = pack_bf16(pw[0], pw[1]), ph1 = pack_bf16(pw[2], pw[3]);
+                const float2 f0 = bf16x2_to_f2(ph0), f1 = bf16x2_to_f2(ph1);
+                const uint32_t pl0 = pack_bf16(pw[0] - f0.x, pw[1] - f0.y), pl1 = pack_bf16(pw[2] - f1.x, pw[3] - f1.y);
+#pragma unroll
+                for (int c2 = 0; c2 < C::NTILES / 2; ++c2) {
+                    uint32_t v00, v01, v10, v11;
+                    ldmatrix_x4_trans(Vs + v_row * C::PITCH + ((2 * c2 + v_chunk_add) << 4), v00, v01, v10, v11);
+                    mma_bf16_16816(o_acc[2 * c2], ph0, pl0, ph1, pl1, v00, v01);
+                    mma_bf16_16816(o_acc[2 * c2 + 1], ph0, pl0, ph1, pl1, v10, v11);
+                }
+                __syncwarp();
+                ++ce;
+                top_up();
+            }
+        }
+        if (failed) break;
+
+        l_run += __shfl_xor_sync(kFull, l_run, 1);
+        l_run += __shfl_xor_sync(kFull, l_run, 2);
+#pragma unroll
+        for (int nt = 0; nt < C::NTILES; ++nt) {
+            o_acc[nt][0] += o_acc[nt][2];
+            o_acc[nt][1] += o_acc[nt][3];
+        }
+        if (n_split == 1) {
+            if (head_ok) {
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                float *o = out + ((size_t)r * H_q + h * G + gid) * D + 2 * tid4;
+#pragma unroll
+                for (int nt = 0; nt < C::NTILES; ++nt)
+                    *reinterpret_cast<float2 *>(o + nt * 8) = make_float2(o_acc[nt][0] * inv, o_acc[nt][1] * inv);
+                if (tid4 == 0)
+                    lse[(size_t)r * H_q + h * G + gid] = l_run > 0.f ? (m_run + log2f(l_run)) * kLn2 : -INFINITY;
+            }
+            continue;
+        }
+        if (head_ok) {
+            float *pr = partials + (((size_t)r * H_q + h * G + gid) * max_splits + my_split) * C::PSTRIDE;
+#pragma unroll
+            for (int nt = 0; nt < C::NTILES; ++nt)
+                *reinterpret_cast<float2 *>(pr + nt * 8 + 2 * tid4) = make_float2(o_acc[nt][0], o_acc[nt][1]);
+            if (tid4 == 0) {
+                pr[D] = m_run;
+                pr[D + 1] = l_run;
+            }
+        }
+    }
+    if (failed) {
+        if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
+        for (int s = 0; s < nstage; ++s) mbar_wait(bar0 + s * 8, (phases >> s) & 1u);
+    }
+}
+
+template <int D>
+cudaError_t launch_token_decode_t(const se_params &p, const void *q, const void *k_cache, const void *v_cache,
+                                  const int32_t *page_table, const int32_t *seq_lens, const int32_t *tok_idx,
+                                  const int32_t *tok_cnt, int n_out, float *out, float *lse, void *workspace,
+                                  const WorkspaceLayout &L, cudaStream_t stream) {
+    using C = TokCfg<D>;
+    const DecodePlan plan = make_decode_plan(p);        // a unit of the plan = one 16-token tile
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    const int G = p.H_q / p.H_kv, GP = next_pow2(G);
+    const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
+                        (size_t)kDecWarps * kChunk * sizeof(int);
+    auto kern = token_decode_kernel<D>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
+        (const uint16_t *)q, (const uint8_t *)k_cache, (const uint8_t *)v_cache, page_table, seq_lens, tok_idx,
+        tok_cnt, out, lse, reinterpret_cast<float *>(ws + L.partials), p.B, p.H_kv, G, p.max_pages,
+        p.num_phys_pages, n_out, plan.pages_per_split, plan.max_splits, effective_scale(p) * kLog2e,
+        reinterpret_cast<uint32_t *>(ws + L.status));
+    e = cudaGetLastError();
+    if (e != cudaSuccess || plan.max_splits == 1) return e;
+    combine_kernel<D><<<dim3(p.B * p.H_kv, 1), 256, 0, stream>>>(
+        reinterpret_cast<const float *>(ws + L.partials), nullptr, page_table, seq_lens, nullptr, nullptr, out, lse,
+        nullptr, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
+        tok_cnt);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_token_decode(const se_params &p, const void *q, const void *k_cache, const void *v_cache,
+                                const int32_t *page_table, const int32_t *seq_lens, const int32_t *tok_idx,
+                                const int32_t *tok_cnt, int n_out, float *out, float *lse, void *workspace,
+                                const WorkspaceLayout &L, cudaStream_t stream) {
+    return (p.D == 128) ? launch_token_decode_t<128>(p, q, k_cache, v_cache, page_table, seq_lens, tok_idx,
+                                                     tok_cnt, n_out, out, lse, workspace, L, stream)
+                        : launch_token_decode_t<64>(p, q, k_cache, v_cache, page_table, seq_lens, tok_idx,
+                                                    tok_cnt, n_out, out, lse, workspace, L, stream);
+}
+
+namespace {
 }  // namespace
 
 int decode_warps_per_cta() { return kDecWarps; }
@@ -608,11 +947,12 @@ cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *
                                  const void *v_cache, const int32_t *page_table,
                                  const int32_t *seq_lens, const int32_t *sel_idx,
                                  const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                                 void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream) {
+                                 uint32_t *tok_keys, void *workspace, const WorkspaceLayout &L, int stages,
+                                 cudaStream_t stream) {
     return (p.D == 128) ? launch_decode<128>(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                                             out, lse, score_accum, workspace, L, stages, stream)
+                                             out, lse, score_accum, tok_keys, workspace, L, stages, stream)
                         : launch_decode<64>(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                                            out, lse, score_accum, workspace, L, stages, stream);
+                                            out, lse, score_accum, tok_keys, workspace, L, stages, stream);
 }
 
 }  // namespace se

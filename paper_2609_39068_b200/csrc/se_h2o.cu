@@ -1,7 +1,7 @@
 // H2O retention and eviction (Appendix A, "H2O: Accumulated Scores and Online Eviction",
 // retention equation): the consumer of the accumulated scores that se_sparse_decode maintains.
 //
-// h2o_retain_kernel   one CTA per (request, kv-head).  The request's token scores are read page
+// retain_kernel       (H2O form) one CTA per (request, kv-head).  The request's token scores are read page
 //                     row by page row (one thread = one 64-byte row of 16 scores, a chunk = one
 //                     row per thread) as order-preserving integer keys; tokens of the protected
 //                     recent window are kept unconditionally and do not compete.  Pass 1 finds
@@ -24,16 +24,22 @@ namespace se {
 
 namespace {
 
-constexpr int kRetThreads = 256;
 constexpr int kRetBins = 2048;
 constexpr int kRetBinBits = 11;
 constexpr int kRetList = 32;
 
+// kTok == false: H2O retention.  One CTA per (request, kv-head); scores are score_accum rows found
+//   through the page table; the window counts against the budget; rows of `budget` entries.
+// kTok == true: token selection of an observation layer (Appendix A, OmniKV selection equation).
+//   One CTA per request; scores are the integer keys an observation layer left in tok_keys
+//   [B, 16*max_pages] (0 = token not attended); the recent window is kept on top of the budget;
+//   rows of n_out entries.
+template <int kRetThreads, bool kTok>
 __global__ void __launch_bounds__(kRetThreads)
-h2o_retain_kernel(const float *__restrict__ score_accum, const int32_t *__restrict__ page_table,
-                  const int32_t *__restrict__ seq_lens, int H_kv, int max_pages, int P_phys, int budget,
-                  int recent, int32_t *__restrict__ keep_idx, int32_t *__restrict__ keep_cnt,
-                  uint32_t *status) {
+retain_kernel(const float *__restrict__ score_accum, const uint32_t *__restrict__ tok_keys,
+              const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens, int H_kv,
+              int max_pages, int P_phys, int budget, int recent, int n_out, int32_t *__restrict__ keep_idx,
+              int32_t *__restrict__ keep_cnt, uint32_t *status) {
     constexpr int NW = kRetThreads / 32;
     constexpr int BPT = kRetBins / kRetThreads;
     __shared__ __align__(16) int s_hist[kRetBins];     // bin = (kmax' - key) >> shift: prefix = better keys
@@ -45,21 +51,46 @@ h2o_retain_kernel(const float *__restrict__ score_accum, const int32_t *__restri
     __shared__ int s_ln;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair = blockIdx.x;
-    const int r = pair / H_kv, h = pair - r * H_kv;
+    const int r = kTok ? pair : pair / H_kv, h = kTok ? 0 : pair - r * H_kv;
     int n = seq_lens[r];
     if (n > max_pages * kPage) n = max_pages * kPage;
     if (n < 0) n = 0;
-    const int w = min(recent, budget);
+    const int w = kTok ? min(recent, n_out) : min(recent, budget);
     const int wstart = n - w;                           // positions >= wstart form the protected window
     const int npages = (n + kPage - 1) / kPage;
     const int chunks = (npages + kRetThreads - 1) / kRetThreads;
-    int32_t *out = keep_idx + (size_t)pair * budget;
+    int32_t *out = keep_idx + (size_t)pair * n_out;
     int scan_par = 0;
 
     // keys of this thread's page row in chunk c; bit t of winmask = token t is in the window
     auto load_row = [&](int c, uint32_t (&keys)[kPage], uint32_t &winmask) {
         const int b = c * kRetThreads + tid;
         winmask = 0;
+        if (kTok) {
+            if (b >= npages) {
+#pragma unroll
+                for (int t = 0; t < kPage; ++t) keys[t] = kKeyAbsent;
+                return;
+            }
+            const uint4 *src = reinterpret_cast<const uint4 *>(tok_keys + (size_t)r * max_pages * kPage + b * kPage);
+#pragma unroll
+            for (int t4 = 0; t4 < kPage / 4; ++t4) {
+                const uint4 v = __ldg(src + t4);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int t = 4 * t4 + e;
+                    const int pos = b * kPage + t;
+                    const uint32_t x = e == 0 ? v.x : e == 1 ? v.y : e == 2 ? v.z : v.w;
+                    uint32_t key = kKeyAbsent;
+                    if (pos < n && x != 0u) {                // 0 = the observation layer did not attend it
+                        if (pos >= wstart) winmask |= 1u << t;
+                        else key = max(x, kKeyAbsent + 1u);
+                    }
+                    keys[t] = key;
+                }
+            }
+            return;
+        }
         int pid = -1;
         if (b < npages) pid = __ldg(page_table + (size_t)r * max_pages + b);
         if (pid >= P_phys) {
@@ -131,10 +162,12 @@ h2o_retain_kernel(const float *__restrict__ score_accum, const int32_t *__restri
         kmin = min(kmin, (uint32_t)s_red[1][i]);
         kmax = max(kmax, (uint32_t)s_red[2][i]);
     }
-    const int k_take = min(budget - nwin, present);      // competitors that stay
+    nwin = min(nwin, n_out);
+    const int k_take = kTok ? min(min(budget, n_out - nwin), present)     // competitors that stay
+                            : min(budget - nwin, present);
     const int total = k_take + nwin;
     if (total == 0) {
-        for (int i = tid; i < budget; i += kRetThreads) out[i] = -1;
+        for (int i = tid; i < n_out; i += kRetThreads) out[i] = -1;
         if (tid == 0) keep_cnt[pair] = 0;
         return;
     }
@@ -292,7 +325,7 @@ h2o_retain_kernel(const float *__restrict__ score_accum, const int32_t *__restri
 #pragma unroll
         for (int t = 0; t < kPage; ++t) {
             if ((takemask >> t) & 1u) {
-                if (pos < budget) out[pos] = pos0 + t;
+                if (pos < n_out) out[pos] = pos0 + t;
                 ++pos;
             }
         }
@@ -300,7 +333,7 @@ h2o_retain_kernel(const float *__restrict__ score_accum, const int32_t *__restri
         base_out = s_res[3];
         scan_par ^= 1;
     }
-    for (int i = total + tid; i < budget; i += kRetThreads) out[i] = -1;
+    for (int i = total + tid; i < n_out; i += kRetThreads) out[i] = -1;
     if (tid == 0) keep_cnt[pair] = total;
 }
 
@@ -387,9 +420,18 @@ h2o_compact_kernel(uint4 *k_cache, uint4 *v_cache, float *score_accum, const int
 cudaError_t launch_h2o_retain(const se_params &p, const float *score_accum, const int32_t *page_table,
                               const int32_t *seq_lens, int budget, int recent, int32_t *keep_idx,
                               int32_t *keep_cnt, uint32_t *status, cudaStream_t stream) {
-    h2o_retain_kernel<<<p.B * p.H_kv, kRetThreads, 0, stream>>>(score_accum, page_table, seq_lens, p.H_kv,
+    retain_kernel<256, false><<<p.B * p.H_kv, 256, 0, stream>>>(score_accum, nullptr, page_table, seq_lens, p.H_kv,
                                                                  p.max_pages, p.num_phys_pages, budget, recent,
-                                                                 keep_idx, keep_cnt, status);
+                                                                 budget, keep_idx, keep_cnt, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_token_select(const se_params &p, const uint32_t *tok_keys, const int32_t *seq_lens, int budget,
+                                int recent, int n_out, int32_t *tok_idx, int32_t *tok_cnt, uint32_t *status,
+                                cudaStream_t stream) {
+    retain_kernel<1024, true><<<p.B, 1024, 0, stream>>>(nullptr, tok_keys, nullptr, seq_lens, p.H_kv, p.max_pages,
+                                                         p.num_phys_pages, budget, recent, n_out, tok_idx, tok_cnt,
+                                                         status);
     return cudaGetLastError();
 }
 

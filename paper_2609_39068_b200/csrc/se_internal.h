@@ -40,7 +40,10 @@ cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *
                                  const void *v_cache, const int32_t *page_table,
                                  const int32_t *seq_lens, const int32_t *sel_idx,
                                  const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
-                                 void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream);
+                                 uint32_t *tok_keys, void *workspace, const WorkspaceLayout &L, int stages,
+                                 cudaStream_t stream);
+// tok_keys != nullptr: observation layer - [B, 16*max_pages] order-preserving integer images of
+// max-over-heads logits, merged with atomic max (the caller zeroes the array first)
 // H2O retention (retained positions per (request, kv-head)) and eviction (in-place compaction)
 cudaError_t launch_h2o_retain(const se_params &p, const float *score_accum, const int32_t *page_table,
                               const int32_t *seq_lens, int budget, int recent, int32_t *keep_idx,
@@ -48,6 +51,13 @@ cudaError_t launch_h2o_retain(const se_params &p, const float *score_accum, cons
 cudaError_t launch_h2o_compact(const se_params &p, void *k_cache, void *v_cache, float *score_accum,
                                const int32_t *page_table, const int32_t *keep_idx, const int32_t *keep_cnt,
                                int budget, int32_t *new_lens, uint32_t *status, cudaStream_t stream);
+cudaError_t launch_token_select(const se_params &p, const uint32_t *tok_keys, const int32_t *seq_lens, int budget,
+                                int recent, int n_out, int32_t *tok_idx, int32_t *tok_cnt, uint32_t *status,
+                                cudaStream_t stream);
+cudaError_t launch_token_decode(const se_params &p, const void *q, const void *k_cache, const void *v_cache,
+                                const int32_t *page_table, const int32_t *seq_lens, const int32_t *tok_idx,
+                                const int32_t *tok_cnt, int n_out, float *out, float *lse, void *workspace,
+                                const WorkspaceLayout &L, cudaStream_t stream);
 // stages: 1 = split attention kernel, 2 = combine kernel (merge + H2O epilogue), 3 = both
 
 }  // namespace se

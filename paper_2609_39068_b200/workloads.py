@@ -259,6 +259,15 @@ def h2o_evict_workload(device="cpu", B: int = 64, cached: int = 5120, budget: in
                  permute_pool=True, with_score_accum=True)
 
 
+def omnikv_workload(device="cpu", layer: int = 0, B: int = 24, length: int = 32768) -> Workload:
+    """One layer of a selection-reuse step: 24 concurrent requests (the paper's OmniKV concurrency) of
+    32768 tokens, 32/8 heads, D=128, 2048 selected + 32 recent tokens.  Layer 0 plays the observation
+    layer, layers 1.. the sparse layers that reuse its token set; the page table does not depend on
+    ``layer``, q/K/V do."""
+    return build("omnikv_reuse_b24_32k", 7, layer, [length] * B, 32, 8, 128, 2048, device, outliers=True,
+                 permute_pool=True)
+
+
 def sub_workload(w: Workload, rows, device="cpu") -> Workload:
     """The requests ``rows`` of ``w`` with their pages gathered into a compact pool of their
     own (physical ids renumbered, aliasing preserved).  Pure data movement: it lets a few

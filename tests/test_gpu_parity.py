@@ -279,6 +279,25 @@ def test_split_and_combine_calls_equal_the_single_call():
     assert torch.equal(o1, st.out) and torch.equal(l1, st.lse) and torch.equal(u, u2)
 
 
+def test_nan_in_slots_past_the_length_does_not_leak():
+    # slots past a request's length are never initialised by an engine: NaN there must not matter
+    w_cpu = wl.build("nan", 876, 0, [37, 16, 1, 250], 8, 2, 128, 64, "cpu", permute_pool=True,
+                     with_score_accum=True)
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16)
+    for r in range(w_cpu.B):
+        L = int(w_cpu.seq_lens[r])
+        if L % 16:
+            pid = int(w_cpu.page_table[r, (L - 1) // 16])
+            w_cpu.k_cache[pid, :, L % 16:, :] = nan
+            w_cpu.v_cache[pid, :, L % 16:, :] = nan
+    w, st, u = run_gpu(w_cpu, accum=True)
+    assert torch.isfinite(st.out).all() and torch.isfinite(st.lse).all() and torch.isfinite(u).all()
+    finite = w_cpu
+    finite.k_cache = torch.nan_to_num(w_cpu.k_cache.float(), nan=0.0).to(torch.bfloat16)
+    finite.v_cache = torch.nan_to_num(w_cpu.v_cache.float(), nan=0.0).to(torch.bfloat16)
+    compare(finite, st, u_before=w_cpu.score_accum.numpy(), u_after=u.cpu().numpy())
+
+
 def test_h2o_accumulation_small():
     w_cpu = wl.build("h2o", 880, 0, [700, 1300, 90], 8, 2, 128, 256, "cpu", permute_pool=True,
                      with_score_accum=True, poison_tail=True)
