@@ -52,6 +52,10 @@ NCU_TRAFFIC_BYTES = {
 H2O_NCU_TRAFFIC_BYTES = 2055e6        # 770.7 MB at 24 requests, scaled by the request count
 
 
+# dram bytes of one token_decode_kernel launch on the 24-request selection-reuse workload (profiles/)
+OMNIKV_NCU_TRAFFIC_BYTES = None
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -212,9 +216,11 @@ def main():
                     help="override the number of requests (configs 3-5; for small profiling captures)")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls directly instead of a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "h2o_evict"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "h2o_evict", "omnikv_reuse"],
                     help="decode = the sparse decode step (the headline); h2o_evict = one H2O eviction "
-                         "(retained set + in-place compaction) of 64 requests, 5120 -> 4096 tokens")
+                         "(retained set + in-place compaction) of 64 requests, 5120 -> 4096 tokens; "
+                         "omnikv_reuse = one observation layer (full attention + token selection) and four "
+                         "sparse layers reusing its 2048+32 tokens, 24 requests of 32768 tokens")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -223,9 +229,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     n_layers = args.layers or (28 if args.config == 5 else 1)
 
-    if args.workload == "h2o_evict":
-        if rank == 0:                        # the eviction step has no multi-GPU leg of its own
-            run_h2o_evict(args, local_rank)
+    if args.workload in ("h2o_evict", "omnikv_reuse"):
+        if rank == 0:                        # these steps have no multi-GPU leg of their own
+            (run_h2o_evict if args.workload == "h2o_evict" else run_omnikv)(args, local_rank)
         return
     if args.impl == "reference":
         if rank == 0:
@@ -559,6 +565,158 @@ def run_h2o_evict(args, local_rank):
         "clocks": sampler.summary(t0, t1),
         "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": w.B * 4, "d2h_bytes_per_step": w.B * 4},
         "gpu_launches": 2 * K, "cpu_baseline": cb}))
+
+
+def omnikv_oracle_time(layers, budget, recent, n_sample=2):
+    """The oracle's observation layer (scores, full attention, token top-k) + reuse layers on a few requests."""
+    import oracle
+    w0 = layers[0]
+    rows = list(range(0, w0.B, max(1, w0.B // n_sample)))[:n_sample]
+    subs = [wl.sub_workload(w, rows, "cpu") for w in layers]
+    a0 = subs[0]
+    pt, sl = a0.page_table.numpy(), a0.seq_lens.numpy()
+    n_pages = (sl + 15) // 16
+    sel = np.full((a0.B, a0.H_kv, a0.max_pages), -1, np.int32)
+    scnt = np.zeros((a0.B, a0.H_kv), np.int32)
+    for r in range(a0.B):
+        sel[r, :, :n_pages[r]] = np.arange(n_pages[r])
+        scnt[r, :] = n_pages[r]
+    bits = [(wl.bf16_bits(x.q), wl.bf16_bits(x.k_cache), wl.bf16_bits(x.v_cache)) for x in subs]
+    t0 = time.perf_counter()
+    s, present = oracle.token_scores(bits[0][0], bits[0][1], pt, sl)
+    oracle.attend(bits[0][0], bits[0][1], bits[0][2], pt, sl, sel, scnt)
+    idx, cnt, _ = oracle.token_topk(s, present, sl, budget, recent)
+    for q, k, v in bits[1:]:
+        oracle.token_attend(q, k, v, pt, sl, idx, cnt)
+    dt = time.perf_counter() - t0
+    scale = w0.B / float(len(rows))
+    return dict(value=dt * scale * 1e6, unit="us", cores=oracle.num_threads(), kind="oracle",
+                sample="%d of %d requests, one run = %.2f s, scaled x%.1f by request count" % (len(rows), w0.B, dt, scale))
+
+
+def run_omnikv(args, local_rank):
+    """Selection reuse across layers: layer 0 = observation layer (full attention that also scores every
+    token, then the token top-k), layers 1-4 = sparse layers attending the 2048 selected + 32 recent
+    tokens of their own caches.  One step = se_observe_decode + se_token_select + 4 x se_token_decode."""
+    budget, recent, n_sparse = 2048, 32, 4
+    if not torch.cuda.is_available():
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the selection-reuse workload is generated on the GPU"}))
+            return
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B = args.batch or 24
+    layers = [wl.omnikv_workload(dev, layer=l, B=B) for l in range(1 + n_sparse)]
+    if args.impl == "reference":
+        cb = omnikv_oracle_time(layers, budget, recent)
+        print(json.dumps({
+            "impl": "reference", "metric": "omnikv_reuse_us_per_step", "value": cb["value"], "unit": "us",
+            "n_gpus": args.gpus, "steps": 1, "warmup": 0, "ms_per_step": cb["value"] / 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": layers[0].name}, "cpu_baseline": cb,
+            "e2e": {"value": cb["value"], "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+    from paper_2609_39068_b200 import binding
+    binding.load()
+    w0 = layers[0]
+    obs = binding.DecodeState(w0, k_max=w0.max_pages)
+    obs.w = wl.Workload(**{**w0.__dict__, "budget": 16 * w0.max_pages})
+    obs.rebuild_meta()
+    obs.select()                                   # full attention: every present page, selected once
+    n_out = budget + recent
+    keys = torch.zeros((B, 16 * w0.max_pages), dtype=torch.int32, device=dev)
+    tok_idx = torch.empty((B, n_out), dtype=torch.int32, device=dev)
+    tok_cnt = torch.empty((B,), dtype=torch.int32, device=dev)
+    p_tok = binding.make_params(B, w0.H_q, w0.H_kv, w0.D, w0.max_pages, w0.num_phys_pages, (n_out + 15) // 16)
+    ws_tok = binding.alloc_workspace(p_tok, dev)
+    outs = [(torch.empty((B, w0.H_q, w0.D), dtype=torch.float32, device=dev),
+             torch.empty((B, w0.H_q), dtype=torch.float32, device=dev)) for _ in range(n_sparse)]
+
+    def observe():
+        binding.se_observe_decode(obs.p, w0.q, w0.k_cache, w0.v_cache, w0.page_table, w0.seq_lens, obs.sel_idx,
+                                  obs.sel_cnt, obs.out, obs.lse, keys, obs.workspace)
+
+    def select():
+        binding.se_token_select(obs.p, keys, w0.seq_lens, budget, recent, tok_idx, tok_cnt, obs.workspace)
+
+    def reuse(i):
+        w = layers[1 + i]
+        binding.se_token_decode(p_tok, w.q, w.k_cache, w.v_cache, w.page_table, w.seq_lens, tok_idx, tok_cnt,
+                                outs[i][0], outs[i][1], ws_tok)
+
+    def step():
+        observe()
+        select()
+        for i in range(n_sparse):
+            reuse(i)
+
+    q_pin = [w.q.cpu().pin_memory() for w in layers]
+    o_pin = [torch.empty(o.shape, dtype=torch.float32).pin_memory() for o, _ in outs]
+
+    def step_e2e():
+        for w, qp in zip(layers, q_pin):
+            w.q.copy_(qp, non_blocking=True)
+        step()
+        for (o, _), op in zip(outs, o_pin):
+            op.copy_(o, non_blocking=True)
+
+    def timed(fn, iters):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters * 1e3
+
+    K = min(args.steps, 100)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    timed(step, args.warmup)
+    t0 = time.perf_counter()
+    step_us = timed(step, K)
+    t1 = time.perf_counter()
+    calls = {"se_observe_decode": timed(observe, 30), "se_token_select": timed(select, 50),
+             "se_token_decode": timed(lambda: reuse(0), 50)}
+    e2e_us = timed(step_e2e, 30)
+    sampler.stop()
+    for ws in (obs.workspace, ws_tok):
+        if binding.se_last_device_status(ws):
+            raise SystemExit("device status %d" % binding.se_last_device_status(ws))
+    n_tok = int(tok_cnt.sum().item())
+    row = 2 * w0.D * 2
+    qo = B * w0.H_q * (2 * w0.D + 4 * w0.D + 4)
+    tok_bytes = n_tok * w0.H_kv * row + n_tok * 4 + qo
+    obs_bytes = int(obs.sel_cnt.sum().item()) * 16 * row + qo + B * 16 * w0.max_pages * 4
+    peak, peak_kind = measured_peak()
+    gbs = tok_bytes / (calls["se_token_decode"] * 1e-6) / 1e9
+    cb = None if args.no_cpu_baseline else omnikv_oracle_time(layers, budget, recent)
+    splits = binding.se_decode_num_splits(p_tok)
+    print(json.dumps({
+        "metric": "omnikv_reuse_us_per_step", "value": step_us, "unit": "us", "n_gpus": 1, "steps": K,
+        "warmup": args.warmup, "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w0.name, "B": B, "H_q": w0.H_q, "H_kv": w0.H_kv, "D": w0.D, "context_tokens": 32768,
+                   "selected_tokens": budget, "recent_tokens": recent, "observation_layers": 1,
+                   "sparse_layers": n_sparse, "storage_dtype": "bf16",
+                   "l2": "inputs larger than L2 (%d MB read by the observation layer, %d MB per sparse layer)"
+                         % (obs_bytes // 10**6, tok_bytes // 10**6)},
+        "calls_us": calls,
+        "algorithmic_bytes": {"se_observe_decode": obs_bytes, "se_token_decode": tok_bytes},
+        "calls_gbs": {"se_observe_decode": obs_bytes / calls["se_observe_decode"] / 1e3,
+                      "se_token_decode": gbs},
+        "roofline": {"bound": "hbm", "kernel": "token_decode_kernel (se_token_decode)", "achieved": gbs, "peak": peak,
+                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": gbs / peak,
+                     "traffic": OMNIKV_NCU_TRAFFIC_BYTES if B == 24 else None, "algorithmic_bytes": tok_bytes},
+        "clocks": sampler.summary(t0, t1),
+        "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": sum(x.numel() * 2 for x in q_pin),
+                "d2h_bytes_per_step": sum(x.numel() * 4 for x in o_pin)},
+        "gpu_launches": K * (2 + 1 + n_sparse * (1 + int(splits > 1))) + K * int(binding.se_decode_num_splits(obs.p) > 1),
+        "cpu_baseline": cb}))
 
 
 def run_reference(args, n_layers):

@@ -643,6 +643,8 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
 // padded by 16 bytes (conflict-free ldmatrix without hardware swizzle).  Tokens that are out of
 // range or whose page is absent are skipped (their columns are masked, their V rows cleared).
 // ---------------------------------------------------------------------------------
+constexpr int kTokChunk = 512;           // tokens whose rows are looked up at once (32 tiles)
+
 template <int D>
 struct TokCfg {
     static constexpr int ROWB = D * 2;                         // bytes of one K or V row
@@ -674,7 +676,7 @@ token_decode_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ 
     uint8_t *ring = smem_tok + (size_t)(warp * nstage) * C::STAGEB;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_tok + (size_t)C::CTA_STAGES * C::STAGEB) + warp * C::MAXST;
     int *ent_row = reinterpret_cast<int *>(smem_tok + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8) +
-                   warp * kChunk;
+                   warp * kTokChunk;
     if (lane == 0) {
         for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
         mbar_fence_init();
@@ -739,25 +741,29 @@ token_decode_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ 
         }
         float m_run = -INFINITY, l_run = 0.f;
 
-        for (int c_lo = e_lo; c_lo < e_hi && !failed; c_lo += kChunk) {
-            // ---- row list of up to kChunk tokens: token -> page table -> row of the [pages*heads*16, D] view
-            const int c_hi = min(e_hi, c_lo + kChunk);
+        for (int c_lo = e_lo; c_lo < e_hi && !failed; c_lo += kTokChunk) {
+            // ---- row list of up to kTokChunk tokens: token -> page table -> row of the [pages*heads*16, D] view
+            const int c_hi = min(e_hi, c_lo + kTokChunk);
             const int n_tiles = (c_hi - c_lo + kPage - 1) / kPage;
+            // (all token loads first, then all page-table loads: two round trips for the whole chunk)
+            int tk[kTokChunk / 32], pd[kTokChunk / 32];
 #pragma unroll
-            for (int rep = 0; rep < kChunk / 32; ++rep) {
+            for (int rep = 0; rep < kTokChunk / 32; ++rep) {
                 const int off = rep * 32 + lane;
+                tk[rep] = (c_lo + off < c_hi) ? __ldg(tok_idx + (size_t)r * n_out + c_lo + off) : -2;
+            }
+#pragma unroll
+            for (int rep = 0; rep < kTokChunk / 32; ++rep) {
+                pd[rep] = -1;
+                if (tk[rep] >= 0 && tk[rep] < len) pd[rep] = __ldg(page_table + (size_t)r * max_pages + (tk[rep] >> 4));
+            }
+#pragma unroll
+            for (int rep = 0; rep < kTokChunk / 32; ++rep) {
                 int row = -1;
-                if (c_lo + off < c_hi) {
-                    const int tok = __ldg(tok_idx + (size_t)r * n_out + c_lo + off);
-                    if (tok < 0 || tok >= len) {
-                        atomicOr(status, SE_DEV_BAD_SELECTION);
-                    } else {
-                        const int pid = __ldg(page_table + (size_t)r * max_pages + (tok >> 4));
-                        if (pid >= P_phys) atomicOr(status, SE_DEV_BAD_PAGE_ID);
-                        else if (pid >= 0) row = (pid * H_kv + h) * kPage + (tok & 15);
-                    }
-                }
-                ent_row[off] = row;
+                if (tk[rep] != -2 && (tk[rep] < 0 || tk[rep] >= len)) atomicOr(status, SE_DEV_BAD_SELECTION);
+                else if (pd[rep] >= P_phys) atomicOr(status, SE_DEV_BAD_PAGE_ID);
+                else if (pd[rep] >= 0) row = (pd[rep] * H_kv + h) * kPage + (tk[rep] & 15);
+                ent_row[rep * 32 + lane] = row;
             }
             __syncwarp();
             int ce = 0, pe = 0;                      // tiles of this chunk consumed / issued
@@ -902,7 +908,7 @@ cudaError_t launch_token_decode_t(const se_params &p, const void *q, const void 
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     const int G = p.H_q / p.H_kv, GP = next_pow2(G);
     const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
-                        (size_t)kDecWarps * kChunk * sizeof(int);
+                        (size_t)kDecWarps * kTokChunk * sizeof(int);
     auto kern = token_decode_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
