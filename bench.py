@@ -53,7 +53,7 @@ H2O_NCU_TRAFFIC_BYTES = 2055e6        # 770.7 MB at 24 requests, scaled by the r
 
 
 # dram bytes of one token_decode_kernel launch on the 24-request selection-reuse workload (profiles/)
-OMNIKV_NCU_TRAFFIC_BYTES = None
+OMNIKV_NCU_TRAFFIC_BYTES = 209e6     # 69.8 MB at 8 requests, scaled by the request count
 
 
 def measured_peak():
