@@ -57,10 +57,7 @@ DecodePlan make_decode_plan(const se_params &p) {
     const long long pairs = (long long)p.B * p.H_kv;
     const long long warps = (long long)kAssumedSMs * warps_per_cta;
     long long splits = warps / pairs;
-#ifndef SE_X_NOSPLIT_PAIRS_PER_SM
-#define SE_X_NOSPLIT_PAIRS_PER_SM 2
-#endif
-    if (splits < 1 || pairs >= (long long)SE_X_NOSPLIT_PAIRS_PER_SM * kAssumedSMs) splits = 1;
+    if (splits < 1 || pairs >= 2LL * kAssumedSMs) splits = 1;
     if (splits > p.k_max) splits = p.k_max;
     const int pps = (int)((p.k_max + splits - 1) / splits);
     plan.pages_per_split = pps;

@@ -58,10 +58,7 @@ struct DecCfg {
     static constexpr int MAXST = 8;                            // most stages one warp can hold
     // Stages a CTA shares out among its busy warps.  More copies in flight than this made the
     // kernel slower, not faster (measured: 24 pages in flight per SM lose 3 % against 16 to 20).
-#ifndef SE_X_CTA_STAGES
-#define SE_X_CTA_STAGES 20
-#endif
-    static constexpr int CTA_STAGES = SE_X_CTA_STAGES * (128 / D);
+    static constexpr int CTA_STAGES = 20 * (128 / D);
     static constexpr int KSTEPS = D / 16;
     static constexpr int NTILES = D / 8;                       // n8 tiles of the output
     static constexpr int PSTRIDE = D + 4;                      // floats per partial row
@@ -938,8 +935,6 @@ cudaError_t launch_token_decode(const se_params &p, const void *q, const void *k
                                                     tok_cnt, n_out, out, lse, workspace, L, stream);
 }
 
-namespace {
-}  // namespace
 
 int decode_warps_per_cta() { return kDecWarps; }
 

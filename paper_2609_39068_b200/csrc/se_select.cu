@@ -676,6 +676,34 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
     SE_TOPK_MARK(5);
 }
 
+// Dense-layer mode (budget >= context): every present page is selected, so there is nothing to
+// score.  One warp per (request, kv-head) writes the present logical pages in ascending order.
+__global__ void __launch_bounds__(256)
+select_all_kernel(const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens, int pairs,
+                  int H_kv, int max_pages, int k_max, int32_t *__restrict__ sel_idx,
+                  int32_t *__restrict__ sel_cnt) {
+    const int lane = threadIdx.x & 31;
+    const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (pair >= pairs) return;
+    const int r = pair / H_kv;
+    const int len = seq_lens[r];
+    int n = len > 0 ? (len + kPage - 1) / kPage : 0;
+    if (n > max_pages) n = max_pages;
+    int32_t *out = sel_idx + (size_t)pair * k_max;
+    int count = 0;
+    for (int b0 = 0; b0 < n; b0 += 32) {
+        const int b = b0 + lane;
+        const bool ok = b < n && __ldg(page_table + (size_t)r * max_pages + b) >= 0;
+        const unsigned m = __ballot_sync(kFull, ok);
+        const int pos = count + __popc(m & ((1u << lane) - 1u));
+        if (ok && pos < k_max) out[pos] = b;
+        count += __popc(m);
+    }
+    count = min(count, k_max);
+    for (int i = count + lane; i < k_max; i += 32) out[i] = -1;
+    if (lane == 0) sel_cnt[pair] = count;
+}
+
 template <int D>
 cudaError_t launch_score(const se_params &p, const void *q, const void *meta, const void *k_cache,
                          const int32_t *page_table, const int32_t *seq_lens, float *scores, uint32_t *status,
@@ -710,6 +738,17 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     float *scores = reinterpret_cast<float *>(ws + L.scores);
     uint32_t *status = reinterpret_cast<uint32_t *>(ws + L.status);
+    if (k_pages >= p.max_pages && p.k_max >= p.max_pages) {
+        // dense layer: the budget covers any context this shape can hold
+        if (k_cache != nullptr) {           // the fused call still owes the newest page's summary
+            cudaError_t em = launch_meta_update(p, k_cache, page_table, seq_lens, nullptr, const_cast<void *>(meta), stream);
+            if (em != cudaSuccess) return em;
+        }
+        const int pairs_all = p.B * p.H_kv;
+        select_all_kernel<<<(pairs_all + 7) / 8, 256, 0, stream>>>(page_table, seq_lens, pairs_all, p.H_kv,
+                                                                    p.max_pages, p.k_max, sel_idx, sel_cnt);
+        return cudaGetLastError();
+    }
     cudaError_t e = (p.D == 128)
                         ? launch_score<128>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream)
                         : launch_score<64>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream);

@@ -279,6 +279,44 @@ def test_split_and_combine_calls_equal_the_single_call():
     assert torch.equal(o1, st.out) and torch.equal(l1, st.lse) and torch.equal(u, u2)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_dense_layer_mode_selects_every_present_page(fused):
+    # budget >= context: nothing is scored, the selection is every present page in ascending order
+    w_cpu = wl.build("dense", 877, 0, [700, 33, 16, 1, 1200], 8, 2, 128, 64, "cpu", permute_pool=True,
+                     prune_fraction=0.3)
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w, k_max=w.max_pages)
+    st.rebuild_meta()
+    meta_full = st.meta.clone()
+    if fused:
+        st.meta.zero_()
+        st.select_fused(budget=16 * w.max_pages)
+    else:
+        st.select(budget=16 * w.max_pages)
+    torch.cuda.synchronize()
+    a = host_arrays(w_cpu)
+    sel, cnt = st.sel_idx.cpu().numpy(), st.sel_cnt.cpu().numpy()
+    for r in range(w.B):
+        n = (int(a["seq_lens"][r]) + 15) // 16
+        want = [b for b in range(n) if a["page_table"][r, b] >= 0]
+        for h in range(w.H_kv):
+            assert cnt[r, h] == len(want) and sel[r, h, :len(want)].tolist() == want
+            assert np.all(sel[r, h, len(want):] == -1)
+    P = np.zeros((w.B, w.H_kv, w.max_pages))
+    present = a["page_table"] >= 0
+    for r in range(w.B):
+        present[r, (int(a["seq_lens"][r]) + 15) // 16:] = False
+    ref_idx, ref_cnt, _ = oracle.topk_pages(P, present, 16 * w.max_pages, k_max=w.max_pages)
+    assert np.array_equal(ref_idx, sel) and np.array_equal(ref_cnt, cnt)
+    if fused:       # the newest page's summary was still refreshed
+        for r in range(w.B):
+            pid = int(a["page_table"][r, (int(a["seq_lens"][r]) - 1) // 16])
+            assert torch.equal(st.meta[pid], meta_full[pid])
+    st.decode()
+    torch.cuda.synchronize()
+    assert st.status() == 0
+
+
 def test_nan_in_slots_past_the_length_does_not_leak():
     # slots past a request's length are never initialised by an engine: NaN there must not matter
     w_cpu = wl.build("nan", 876, 0, [37, 16, 1, 250], 8, 2, 128, 64, "cpu", permute_pool=True,
