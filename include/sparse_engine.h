@@ -151,7 +151,7 @@ int se_meta_update(const se_params *p, const void *k_cache, const int32_t *page_
  * request are always part of the result when they are present; they are not candidates of the
  * top-k and do not count against the budget, so sel_cnt can reach floor(budget/16) + s + t.
  * Requires 16 <= budget_tokens and floor(budget_tokens/16) + s + t <= k_max.
-  * Dense-layer mode: when budget_tokens / 16 >= max_pages and k_max >= max_pages the budget covers
+ * Dense-layer mode: when budget_tokens / 16 >= max_pages and k_max >= max_pages the budget covers
  * any context of this shape, nothing is scored (meta is not read) and every present page is
  * selected.
  */
