@@ -85,3 +85,26 @@ def test_null_and_misaligned_pointers_are_rejected_before_launch():
     assert lib.se_sparse_decode(ctypes.byref(p), ok, ok, ok, ok, ok, ok, ok, ok, None, None, ok, None) == -3
     assert lib.se_sparse_decode(ctypes.byref(p), ok, ok, ok, ok, ok, ok, ok, ok, ok, odd, ok, None) == -4
     assert lib.se_workspace_init(None, ok, None) == -3
+
+
+def test_h2o_and_token_calls_reject_bad_arguments_before_launch():
+    lib = binding.load()
+    p = binding.make_params(2, 32, 8, 128, 64, 128, 16)
+    pp = ctypes.byref(p)
+    ok, odd = ctypes.c_void_p(4096), ctypes.c_void_p(4100)
+    # H2O retention / eviction
+    assert lib.se_h2o_retain(pp, None, ok, ok, 64, 8, ok, ok, ok, None) == -3
+    assert lib.se_h2o_retain(pp, ok, ok, ok, 0, 8, ok, ok, ok, None) == -1          # empty budget
+    assert lib.se_h2o_retain(pp, ok, ok, ok, 64, -1, ok, ok, ok, None) == -1
+    assert lib.se_h2o_retain(pp, ok, ok, ok, 64, 8, odd, ok, ok, None) == -4
+    assert lib.se_h2o_compact(pp, ok, ok, ok, ok, ok, ok, 64, None, ok, None) == -3
+    assert lib.se_h2o_compact(pp, ok, odd, ok, ok, ok, ok, 64, ok, ok, None) == -4
+    assert lib.se_h2o_compact(pp, ok, ok, ok, ok, ok, ok, 0, ok, ok, None) == -1
+    # selection reuse
+    assert lib.se_observe_decode(pp, ok, ok, ok, ok, ok, ok, ok, ok, ok, None, ok, None) == -3
+    assert lib.se_token_select(pp, ok, ok, 32, 8, ok, ok, 32, ok, None) == -1        # budget + recent > row length
+    assert lib.se_token_select(pp, ok, ok, 32, 8, ok, None, 40, ok, None) == -3
+    assert lib.se_token_decode(pp, ok, ok, ok, ok, ok, ok, ok, 16 * 16 + 1, ok, ok, ok, None) == -1   # > k_max tiles
+    assert lib.se_token_decode(pp, ok, ok, ok, ok, ok, ok, ok, 64, ok, odd, ok, None) == -4
+    bad = binding.make_params(2, 32, 8, 96, 64, 128, 16)
+    assert lib.se_token_decode(ctypes.byref(bad), ok, ok, ok, ok, ok, ok, ok, 64, ok, ok, ok, None) in (-1, -2)
