@@ -726,9 +726,12 @@ def run_reference(args, n_layers):
     if dev == "cpu" and args.config in (3, 4, 5):
         kw = {3: dict(B=4), 4: dict(B=1, length=32768), 5: dict(B=8)}[args.config]
         w = wl.CONFIGS[args.config](dev, **kw)
-        note = "generated on the CPU at reduced batch (%s)" % kw
+        # no GPU to generate the full pool on: a sixteenth of the workload, scaled back up
+        reduced = 16.0
+        note = "generated on the CPU at reduced size (%s), then x%.0f to the full workload" % (kw, reduced)
     else:
         w = wl.CONFIGS[args.config](dev)
+        reduced = 1.0
         note = "full workload generated on the GPU, sample copied to the host"
     order = list(range(0, w.B, max(1, w.B // 16)))[:16]
     sub = wl.sub_workload(w, order, "cpu")
@@ -737,7 +740,7 @@ def run_reference(args, n_layers):
     meta = oracle.quest_meta(k, pt, sl, first_tok=np.zeros(sub.B, np.int32))
     u = None if sub.score_accum is None else sub.score_accum.numpy().astype(np.float64)
     n_all = (w.seq_lens.cpu().numpy() + 15) // 16
-    scale = float(n_all.sum()) / float(((sl + 15) // 16).sum()) * n_layers
+    scale = float(n_all.sum()) / float(((sl + 15) // 16).sum()) * n_layers * reduced
     steps = max(1, min(args.steps, 20))
     warm = max(1, min(args.warmup, 3))
     for _ in range(warm):
