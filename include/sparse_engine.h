@@ -213,8 +213,8 @@ int se_sparse_decode(const se_params *p, const void *q, const void *k_cache,
  *   - no workspace argument; nothing is allocated or freed, by this call or on its behalf;
  *   - dev_status (nullable, 4-byte aligned DEVICE pointer, caller-owned) receives the status
  *     word of this call (SE_DEV_* bits) once the stream reaches that point;
- *   - the shape is limited by the array: 256 + 4*B*H_kv*max_pages bytes must not exceed
- *     SE_STATIC_SCRATCH_BYTES, otherwise SE_ERR_SCRATCH_TOO_SMALL is returned and nothing is
+ *   - the shape is limited by the array: 256 + 4*B*H_kv*P bytes, P = max_pages rounded up to a
+ *     multiple of 4 (score rows start 16-byte aligned), must not exceed SE_STATIC_SCRATCH_BYTES, otherwise SE_ERR_SCRATCH_TOO_SMALL is returned and nothing is
  *     enqueued.
  * The first call on a device looks up the array's device address (a set-up step, done once per
  * device with that device current); make that first call outside any stream capture.
