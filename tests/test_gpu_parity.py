@@ -366,6 +366,19 @@ def test_bad_selection_sets_status_and_is_skipped():
 
 # ---------------------------------------------------------------- the named configurations
 
+def test_maximum_sizes_one_request():
+    # the limits of the build at once: 131072 tokens (8192 pages), k_max = 4096 selected pages, G = 8
+    w = wl.build("max", 878, 0, [131072], 8, 1, 128, 65536, "cuda", permute_pool=True)
+    w_cpu = w.to("cpu")
+    st = binding.DecodeState(w)
+    assert st.k_max == 4096 and w.max_pages == 8192
+    st.rebuild_meta()
+    st.step()
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    compare(w_cpu, st)
+
+
 def test_config1_tiny():
     w_cpu = wl.config1("cpu")
     w, st, _ = run_gpu(w_cpu)
