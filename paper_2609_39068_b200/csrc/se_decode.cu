@@ -79,7 +79,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
-template <int D>
+template <int D, bool kObserve>
 __global__ void __launch_bounds__(kDecWarps * 32, 1)
 decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
               const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
@@ -152,7 +152,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         chunk_end = min(x_end, base + kChunk);
         const int pair0 = base / k_max;
         const int i0 = base - pair0 * k_max;
-        int sl_pid[kChunk / 32], sl_meta[kChunk / 32], sl_b[kChunk / 32];
+        int sl_pid[kChunk / 32], sl_meta[kChunk / 32], sl_b[kObserve ? kChunk / 32 : 1];
 #pragma unroll
         for (int rep = 0; rep < kChunk / 32; ++rep) {
             const int off = rep * 32 + lane;
@@ -179,7 +179,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             }
             sl_pid[rep] = pid;
             sl_meta[rep] = meta;
-            sl_b[rep] = lb;
+            if (kObserve) sl_b[rep] = lb;
         }
         int count = 0;
 #pragma unroll
@@ -197,7 +197,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 const int pos = count + __popc(vm & ((1u << lane) - 1u));
                 ent_y[pos] = (pid * H_kv + (sl_meta[rep] >> 24)) * kPage;
                 ent_info[pos] = sl_meta[rep] & 0x00ffffff;
-                ent_b[pos] = sl_b[rep];
+                if (kObserve) ent_b[pos] = sl_b[rep];
             }
             count += __popc(vm);
         }
@@ -332,7 +332,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 zp[(t0 + 8) * GP] = z[2];
                 zp[(t0 + 9) * GP] = z[3];
             }
-            if (tok_keys != nullptr) {
+            if (kObserve) {
                 // observation layer: s(j) = max over every query head of the logit (Appendix A, OmniKV
                 // selection equation).  Here: max over the group's heads (rows gid), then an atomic
                 // max over the kv-heads on the order-preserving integer image of the score.
@@ -607,7 +607,7 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
     const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
                         (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 1024;
-    auto kern = decode_kernel<D>;
+    auto kern = tok_keys ? decode_kernel<D, true> : decode_kernel<D, false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
