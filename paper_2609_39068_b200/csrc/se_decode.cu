@@ -144,6 +144,12 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                  warp * 3 * kChunk;
     int *ent_info = ent_y + kChunk;
     int *ent_b = ent_info + kChunk;
+    // 16 zero bytes per CTA (behind the page lists)
+    const uint32_t zero_chunk = smem_u32(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8 +
+                                         (size_t)kDecWarps * 3 * kChunk * sizeof(int));
+    if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8 +
+                                                     (size_t)kDecWarps * 3 * kChunk * sizeof(int))[threadIdx.x] = 0u;
+    __syncthreads();
     int chunk_base = 0, chunk_end = 0;           // slots [chunk_base, chunk_end) are in the list
     int n_ent = 0, ce = 0, pe = 0;               // entries, next to consume, next to issue
 
@@ -353,17 +359,6 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                     if (m4[3] > -INFINITY) atomicMax(kp + t0 + 9, f32_key(m4[3] * kLn2));
                 }
             }
-            if (nv_j < kPage) {
-                // slots past the request's length may hold anything (NaN included): their weights are
-                // zero, so their V rows are cleared in shared memory before the product
-                for (int idx = lane; idx < (kPage - nv_j) * C::HALVES * 8; idx += 32) {
-                    const int row = nv_j + idx / (C::HALVES * 8);
-                    const int rem = idx % (C::HALVES * 8);
-                    const uint32_t addr = Vs + (rem >> 3) * kTileBytes + row * 128 + (rem & 7) * 16;
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
-                }
-                __syncwarp();
-            }
             float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
             pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
             pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
@@ -398,7 +393,10 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 const int hf = c2 >> 2;
                 const int chunk = 2 * (c2 & 3) + v_chunk_add;
                 uint32_t v00, v01, v10, v11;     // {chunk c: tok 0-7, tok 8-15}, {chunk c+1: ...}
-                ldmatrix_x4_trans(Vs + hf * kTileBytes + v_row * 128 + ((chunk ^ (v_row & 7)) << 4), v00, v01, v10, v11);
+                // token rows past the request's length may hold anything (NaN included) and their
+                // weights are zero: their lanes read a zeroed chunk instead
+                const uint32_t va = Vs + hf * kTileBytes + v_row * 128 + ((chunk ^ (v_row & 7)) << 4);
+                ldmatrix_x4_trans(v_row < nv_j ? va : zero_chunk, v00, v01, v10, v11);
                 mma_bf16_16816(o_acc[2 * c2], ph0, pl0, ph1, pl1, v00, v01);
                 mma_bf16_16816(o_acc[2 * c2 + 1], ph0, pl0, ph1, pl1, v10, v11);
             }
@@ -606,7 +604,7 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     CUtensorMap k_map, v_map;
     if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
     const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
-                        (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 1024;
+                        (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 16 + 1024;
     auto kern = tok_keys ? decode_kernel<D, true> : decode_kernel<D, false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
