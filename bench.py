@@ -18,6 +18,7 @@ scaling is weak.  Rank 0 prints ONE JSON line.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -361,22 +362,66 @@ def main():
     sel_gbs = b0["select_call"] / (call_us["se_page_select"] * 1e-6) / 1e9
     step_gbs = total_bytes / (ms_per_step * 1e-3) / 1e9
 
-    # ---- end to end through the public API with host buffers
-    pinned_in = [(w.q.cpu().pin_memory(), w.seq_lens.cpu().pin_memory(), w.page_table.cpu().pin_memory())
-                 for w in layers]
-    pinned_out = [(torch.empty(st.out.shape, dtype=torch.float32).pin_memory(),
-                   torch.empty(st.lse.shape, dtype=torch.float32).pin_memory()) for st in states]
-    h2d = sum(sum(t.numel() * t.element_size() for t in tri) for tri in pinned_in)
-    d2h = sum(sum(t.numel() * t.element_size() for t in pair) for pair in pinned_out)
+    # ---- end to end through the public API with host buffers: the step's inputs (q, lengths, page
+    # table) sit in one pinned block and go up in one copy, out + lse come back in one copy
+    import copy
+
+    def packed(tensors, device, pin):
+        """One byte block holding the tensors back to back (16-byte aligned); returns (block, views)."""
+        offs, total = [], 0
+        for t in tensors:
+            offs.append(total)
+            total += (t.numel() * t.element_size() + 15) // 16 * 16
+        block = torch.empty(total, dtype=torch.uint8, device=device)
+        if pin:
+            block = block.pin_memory()
+        views = [block[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for o, t in zip(offs, tensors)]
+        return block, views
+
+    e2e_states, host_in, dev_in, host_out, dev_out = [], [], [], [], []
+    for w, st in zip(layers, states):
+        ins = [w.q, w.seq_lens, w.page_table]
+        hb, hv = packed(ins, "cpu", True)
+        db, dv = packed(ins, dev, False)
+        for src, h, d in zip(ins, hv, dv):
+            h.copy_(src)
+            d.copy_(src)
+        outs = [st.out, st.lse]
+        ob, ov = packed(outs, dev, False)
+        hob, _ = packed(outs, "cpu", True)
+        st2 = copy.copy(st)                       # same params, workspace, summaries and selection buffers
+        st2.w = dataclasses.replace(w, q=dv[0], seq_lens=dv[1], page_table=dv[2])
+        st2.out, st2.lse = ov
+        e2e_states.append(st2)
+        host_in.append(hb); dev_in.append(db); host_out.append(hob); dev_out.append(ob)
+    h2d = sum(b.numel() for b in host_in)
+    d2h = sum(b.numel() for b in host_out)
+
+    def e2e_body():
+        for st2, u, hb, db, ob, hob in zip(e2e_states, accums, host_in, dev_in, dev_out, host_out):
+            db.copy_(hb, non_blocking=True)
+            st2.step(score_accum=u)
+            hob.copy_(ob, non_blocking=True)
+
+    # the way a serving loop drives the library: the host fills fixed pinned buffers, one graph launch
+    # does upload + step + download, and the host waits for the result before the next step
+    e2e_graph = None
+    if not args.no_graph:
+        s2 = torch.cuda.Stream()
+        s2.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s2):
+            e2e_body()
+        torch.cuda.current_stream().wait_stream(s2)
+        torch.cuda.synchronize()
+        e2e_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(e2e_graph):
+            e2e_body()
 
     def e2e_step():
-        for w, st, u, pin, pout in zip(layers, states, accums, pinned_in, pinned_out):
-            w.q.copy_(pin[0], non_blocking=True)
-            w.seq_lens.copy_(pin[1], non_blocking=True)
-            w.page_table.copy_(pin[2], non_blocking=True)
-            st.step(score_accum=u)
-            pout[0].copy_(st.out, non_blocking=True)
-            pout[1].copy_(st.lse, non_blocking=True)
+        if e2e_graph is not None:
+            e2e_graph.replay()
+        else:
+            e2e_body()
         torch.cuda.synchronize()
 
     for _ in range(3):
