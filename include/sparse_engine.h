@@ -230,6 +230,22 @@ int se_page_select_static(const se_params *p, const void *q, const void *meta,
                           int32_t *dev_status, void *stream);
 
 /*
+ * The two halves of se_page_select as separate calls (same arguments, same workspace): first
+ * se_page_select_scores - the scoring kernel; the fp32 page scores stay in the workspace - then
+ * se_page_select_topk - the top-k kernel, which reads them.  One after the other on the same stream
+ * they are exactly se_page_select (except in dense-layer mode, which only the single call takes);
+ * they exist so that a profiler or a benchmark can time the two kernels apart.
+ */
+int se_page_select_scores(const se_params *p, const void *q, const void *meta,
+                          const int32_t *page_table, const int32_t *seq_lens,
+                          int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
+                          void *workspace, void *stream);
+int se_page_select_topk(const se_params *p, const void *q, const void *meta,
+                        const int32_t *page_table, const int32_t *seq_lens,
+                        int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
+                        void *workspace, void *stream);
+
+/*
  * The two halves of se_sparse_decode as separate calls (same arguments, same workspace): first
  * se_sparse_decode_splits - the split-K attention kernel; pairs held by a single worker get their
  * final out/lse, the others leave partial results in the workspace - then se_combine - the

@@ -22,7 +22,7 @@ SE_DEV_WAIT_TIMEOUT = 4
 
 EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_decode_num_splits", "se_workspace_init",
            "se_meta_update",
-           "se_page_select", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
+           "se_page_select", "se_page_select_scores", "se_page_select_topk", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
            "se_last_device_status", "se_h2o_retain", "se_h2o_compact", "se_observe_decode", "se_token_select",
            "se_token_decode",
            "se_page_select_static")
@@ -69,6 +69,8 @@ def load(build_if_missing: bool = True):
     lib.se_workspace_init.argtypes = [pp, vp, vp]
     lib.se_meta_update.argtypes = [pp, vp, i32p, i32p, i32p, vp, vp]
     lib.se_page_select.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
+    lib.se_page_select_scores.argtypes = lib.se_page_select.argtypes
+    lib.se_page_select_topk.argtypes = lib.se_page_select.argtypes
     lib.se_page_select_fused.argtypes = [pp, vp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_sparse_decode.argtypes = [pp, vp, vp, vp, i32p, i32p, i32p, i32p, fp, fp, fp, vp, vp]
     lib.se_sparse_decode_splits.argtypes = lib.se_sparse_decode.argtypes
@@ -83,7 +85,8 @@ def load(build_if_missing: bool = True):
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
                  "se_sparse_decode", "se_sparse_decode_splits", "se_combine", "se_last_device_status",
                  "se_h2o_retain", "se_h2o_compact", "se_decode_num_splits", "se_page_select_static",
-                 "se_observe_decode", "se_token_select", "se_token_decode"):
+                 "se_observe_decode", "se_token_select", "se_token_decode", "se_page_select_scores",
+                 "se_page_select_topk"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -155,13 +158,22 @@ def se_meta_update(p, k_cache, page_table, seq_lens, meta, first_tok=None) -> No
                                  _ptr(meta, torch.bfloat16, "meta"), _stream()), "se_meta_update")
 
 
-def se_page_select(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, workspace) -> None:
-    _check(load().se_page_select(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+def se_page_select(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, workspace,
+                   entry="se_page_select") -> None:
+    _check(getattr(load(), entry)(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
                                  _ptr(meta, torch.bfloat16, "meta"),
                                  _ptr(page_table, torch.int32, "page_table"),
                                  _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens),
                                  _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
-                                 _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_page_select")
+                                 _ptr(workspace, torch.uint8, "workspace"), _stream()), entry)
+
+
+def se_page_select_scores(*args, **kw) -> None:
+    se_page_select(*args, entry="se_page_select_scores", **kw)
+
+
+def se_page_select_topk(*args, **kw) -> None:
+    se_page_select(*args, entry="se_page_select_topk", **kw)
 
 
 def se_page_select_fused(p, q, k_cache, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,
@@ -303,9 +315,10 @@ class DecodeState:
     def update_meta(self):
         se_meta_update(self.p, self.w.k_cache, self.w.page_table, self.w.seq_lens, self.meta)
 
-    def select(self, budget: Optional[int] = None):
+    def select(self, budget: Optional[int] = None, entry="se_page_select"):
         se_page_select(self.p, self.w.q, self.meta, self.w.page_table, self.w.seq_lens,
-                       self.w.budget if budget is None else budget, self.sel_idx, self.sel_cnt, self.workspace)
+                       self.w.budget if budget is None else budget, self.sel_idx, self.sel_cnt, self.workspace,
+                       entry=entry)
 
     def decode(self, score_accum=None, entry="se_sparse_decode"):
         se_sparse_decode(self.p, self.w.q, self.w.k_cache, self.w.v_cache, self.w.page_table,

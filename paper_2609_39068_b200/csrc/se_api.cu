@@ -138,9 +138,9 @@ int se_meta_update(const se_params *p, const void *k_cache, const int32_t *page_
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
 }
 
-int se_page_select(const se_params *p, const void *q, const void *meta, const int32_t *page_table,
+static int page_select_stages(const se_params *p, const void *q, const void *meta, const int32_t *page_table,
                    const int32_t *seq_lens, int32_t budget_tokens, int32_t *sel_idx,
-                   int32_t *sel_cnt, void *workspace, void *stream) {
+                   int32_t *sel_cnt, void *workspace, void *stream, int stages) {
     int rc = validate(p);
     if (rc != SE_OK) return rc;
     if (!q || !meta || !page_table || !seq_lens || !sel_idx || !sel_cnt || !workspace)
@@ -153,8 +153,26 @@ int se_page_select(const se_params *p, const void *q, const void *meta, const in
     if (k_pages + p->sink_pages + p->recent_pages > p->k_max) return SE_ERR_INVALID_ARG;
     const WorkspaceLayout L = make_layout(*p);
     cudaError_t e = launch_page_select(*p, q, meta, nullptr, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
-                                       workspace, L, static_cast<cudaStream_t>(stream));
+                                       workspace, L, static_cast<cudaStream_t>(stream), stages);
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_page_select(const se_params *p, const void *q, const void *meta, const int32_t *page_table,
+                   const int32_t *seq_lens, int32_t budget_tokens, int32_t *sel_idx,
+                   int32_t *sel_cnt, void *workspace, void *stream) {
+    return page_select_stages(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, workspace, stream, 3);
+}
+
+int se_page_select_scores(const se_params *p, const void *q, const void *meta, const int32_t *page_table,
+                          const int32_t *seq_lens, int32_t budget_tokens, int32_t *sel_idx,
+                          int32_t *sel_cnt, void *workspace, void *stream) {
+    return page_select_stages(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, workspace, stream, 1);
+}
+
+int se_page_select_topk(const se_params *p, const void *q, const void *meta, const int32_t *page_table,
+                        const int32_t *seq_lens, int32_t budget_tokens, int32_t *sel_idx,
+                        int32_t *sel_cnt, void *workspace, void *stream) {
+    return page_select_stages(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, workspace, stream, 2);
 }
 
 int se_page_select_fused(const se_params *p, const void *q, const void *k_cache, void *meta,

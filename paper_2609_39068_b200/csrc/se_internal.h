@@ -34,7 +34,8 @@ cudaError_t launch_meta_update(const se_params &p, const void *k_cache, const in
 cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta, const void *k_cache,
                                const int32_t *page_table, const int32_t *seq_lens, int k_pages,
                                int32_t *sel_idx, int32_t *sel_cnt, void *workspace,
-                               const WorkspaceLayout &L, cudaStream_t stream);
+                               const WorkspaceLayout &L, cudaStream_t stream, int stages = 3);
+// stages: 1 = scoring kernel only (scores stay in the workspace), 2 = top-k kernel only, 3 = both
 
 cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *k_cache,
                                  const void *v_cache, const int32_t *page_table,

@@ -734,11 +734,11 @@ cudaError_t launch_score(const se_params &p, const void *q, const void *meta, co
 cudaError_t launch_page_select(const se_params &p, const void *q, const void *meta, const void *k_cache,
                                const int32_t *page_table, const int32_t *seq_lens, int k_pages,
                                int32_t *sel_idx, int32_t *sel_cnt, void *workspace,
-                               const WorkspaceLayout &L, cudaStream_t stream) {
+                               const WorkspaceLayout &L, cudaStream_t stream, int stages) {
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     float *scores = reinterpret_cast<float *>(ws + L.scores);
     uint32_t *status = reinterpret_cast<uint32_t *>(ws + L.status);
-    if (k_pages >= p.max_pages && p.k_max >= p.max_pages) {
+    if (stages == 3 && k_pages >= p.max_pages && p.k_max >= p.max_pages) {
         // dense layer: the budget covers any context this shape can hold
         if (k_cache != nullptr) {           // the fused call still owes the newest page's summary
             cudaError_t em = launch_meta_update(p, k_cache, page_table, seq_lens, nullptr, const_cast<void *>(meta), stream);
@@ -749,10 +749,13 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
                                                                     p.max_pages, p.k_max, sel_idx, sel_cnt);
         return cudaGetLastError();
     }
-    cudaError_t e = (p.D == 128)
-                        ? launch_score<128>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream)
-                        : launch_score<64>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream);
-    if (e != cudaSuccess) return e;
+    if (stages & 1) {
+        cudaError_t e = (p.D == 128)
+                            ? launch_score<128>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream)
+                            : launch_score<64>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream);
+        if (e != cudaSuccess) return e;
+    }
+    if (!(stages & 2)) return cudaSuccess;
     const int pairs = p.B * p.H_kv;
 #define SE_TOPK(THREADS, KPT)                                                                         \
     do {                                                                                              \

@@ -336,6 +336,20 @@ def test_nan_in_slots_past_the_length_does_not_leak():
     compare(finite, st, u_before=w_cpu.score_accum.numpy(), u_after=u.cpu().numpy())
 
 
+def test_score_and_topk_calls_equal_the_single_call():
+    w_cpu = wl.build("two", 879, 0, [5000, 300, 9000], 8, 2, 128, 1024, "cpu", permute_pool=True)
+    w, st, _ = run_gpu(w_cpu)
+    s1, c1 = st.sel_idx.clone(), st.sel_cnt.clone()
+    st.sel_idx.fill_(-5)
+    st.sel_cnt.fill_(-5)
+    st.select(entry="se_page_select_scores")
+    torch.cuda.synchronize()
+    assert int(st.sel_cnt[0, 0]) == -5            # the scoring half writes no selection
+    st.select(entry="se_page_select_topk")
+    torch.cuda.synchronize()
+    assert torch.equal(s1, st.sel_idx) and torch.equal(c1, st.sel_cnt) and st.status() == 0
+
+
 def test_h2o_accumulation_small():
     w_cpu = wl.build("h2o", 880, 0, [700, 1300, 90], 8, 2, 128, 256, "cpu", permute_pool=True,
                      with_score_accum=True, poison_tail=True)
