@@ -486,6 +486,7 @@ def main():
                 "l2": ("flushed with a %d MiB write before every step" % (2 * L2_BYTES >> 20)) if flush
                       else "inputs larger than L2 (%.0f MB touched per step)" % (working_set / 1e6),
                 "parallelism": "1 GPU" if world == 1 else "%d replicas, no collective" % world,
+                "global_batch": layers[0].B * world,
             },
             "algorithmic_bytes_per_step": total_bytes,
             "achieved_gbs": step_gbs * world,
