@@ -191,7 +191,7 @@ def oracle_time(w, target_s=(10.0, 30.0)):
     u = None if sub.score_accum is None else sub.score_accum.numpy().astype(np.float64)
     times = []
     t_begin = time.perf_counter()
-    while len(times) < 3 or (time.perf_counter() - t_begin < target_s[0] and len(times) < 50):
+    while len(times) < 3 or time.perf_counter() - t_begin < target_s[0]:
         t0 = time.perf_counter()
         oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
         times.append(time.perf_counter() - t0)
@@ -203,8 +203,8 @@ def oracle_time(w, target_s=(10.0, 30.0)):
     best = min(times)
     return dict(value=best * scale * 1e6, unit="us", cores=oracle.num_threads(), kind="oracle",
                 sample="%d of %d requests (every %d-th), fp64 C oracle with OpenMP over (request, kv-head), "
-                       "best of %d runs = %.1f ms, scaled x%.2f by page count to the full batch"
-                       % (sub.B, w.B, max(1, w.B // 16), len(times), best * 1e3, scale),
+                       "best of %d runs (%.0f s of wall time) = %.1f ms, scaled x%.2f by page count to the full batch"
+                       % (sub.B, w.B, max(1, w.B // 16), len(times), time.perf_counter() - t_begin, best * 1e3, scale),
                 sample_seconds=best)
 
 
