@@ -104,7 +104,7 @@ def test_observe_select_reuse_small(D, H_q, H_kv, prune):
     torch.cuda.synchronize()
     assert torch.equal(st.out, st2.out) and torch.equal(st.lse, st2.lse)
     s_ref, present, s_gpu = check_scores(w_cpu, keys)
-    for budget, recent in [(64, 8), (200, 0), (16, 40), (2000, 4)]:
+    for budget, recent in [(64, 8), (200, 0), (16, 40), (2000, 4), (0, 8)]:
         tok_idx, tok_cnt = select(st, keys, w, budget, recent)
         check_select(w_cpu, s_ref, present, s_gpu, tok_idx, tok_cnt, budget, recent)
         # two sparse layers reuse the set on their own caches
