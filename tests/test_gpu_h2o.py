@@ -145,3 +145,57 @@ def test_eviction_workload_full_size_sampled():
     assert np.array_equal(wl.bf16_bits(got.k_cache), k_ref)
     assert np.array_equal(wl.bf16_bits(got.v_cache), v_ref)
     assert np.array_equal(got.score_accum.numpy().astype(np.float64), u_ref)
+
+
+def test_h2o_lifecycle_decode_evict_decode():
+    """Scores accumulate during a dense decode step, the eviction keeps the heavy hitters and the recent
+    window, and the next decode step runs on the compacted cache with the scores still aligned: every
+    stage against the oracle doing the same."""
+    w_cpu = wl.build("life", 966, 0, [400, 150, 64], 8, 2, 128, 64, "cpu", permute_pool=True, with_score_accum=True)
+    w_cpu.score_accum.zero_()                       # scores start at zero
+    w = w_cpu.to("cuda")
+    a = host_arrays(w_cpu)
+    n_pages = (a["seq_lens"] + 15) // 16
+    sel = np.full((w.B, w.H_kv, w.max_pages), -1, np.int32)
+    scnt = np.zeros((w.B, w.H_kv), np.int32)
+    for r in range(w.B):
+        sel[r, :, :n_pages[r]] = np.arange(n_pages[r])
+        scnt[r, :] = n_pages[r]
+    # step 1: full attention, scores accumulate
+    st = binding.DecodeState(w, k_max=w.max_pages)
+    st.sel_idx.copy_(torch.from_numpy(sel))
+    st.sel_cnt.copy_(torch.from_numpy(scnt))
+    st.decode(score_accum=w.score_accum)
+    torch.cuda.synchronize()
+    u_ref = np.zeros_like(w_cpu.score_accum.numpy(), dtype=np.float64)
+    oracle.attend(a["q"], a["k"], a["v"], a["page_table"], a["seq_lens"], sel, scnt, u_accum=u_ref)
+    u_gpu = w.score_accum.cpu().numpy().astype(np.float64)
+    assert np.abs(u_gpu - u_ref).max() <= 1e-4 + 1e-3 * np.abs(u_ref).max()
+    # eviction on the GPU's own fp32 scores: bit-exact against the oracle fed with them
+    budget, recent = 96, 16
+    p, ws, keep_idx, keep_cnt = gpu_retain(w, budget, recent)
+    ref_idx, ref_cnt = oracle.h2o_retain(u_gpu, a["page_table"], a["seq_lens"], budget, recent)
+    assert np.array_equal(keep_idx.cpu().numpy(), ref_idx) and np.array_equal(keep_cnt.cpu().numpy(), ref_cnt)
+    k2, v2, u2, len2 = oracle.h2o_compact(a["k"], a["v"], u_gpu, a["page_table"], ref_idx, ref_cnt)
+    new_lens = torch.zeros((w.B,), dtype=torch.int32, device="cuda")
+    binding.se_h2o_compact(p, w.k_cache, w.v_cache, w.score_accum, w.page_table, keep_idx, keep_cnt, new_lens, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(new_lens.cpu().numpy(), len2) and np.array_equal(wl.bf16_bits(w.k_cache), k2)
+    # step 2: the next decode step on the compacted cache keeps accumulating on the moved scores
+    n2 = (len2 + 15) // 16
+    sel2 = np.full_like(sel, -1)
+    scnt2 = np.zeros_like(scnt)
+    for r in range(w.B):
+        sel2[r, :, :n2[r]] = np.arange(n2[r])
+        scnt2[r, :] = n2[r]
+    w2 = wl.Workload(**{**w.__dict__, "seq_lens": new_lens})
+    st2 = binding.DecodeState(w2, k_max=w.max_pages)
+    st2.sel_idx.copy_(torch.from_numpy(sel2))
+    st2.sel_cnt.copy_(torch.from_numpy(scnt2))
+    st2.decode(score_accum=w.score_accum)
+    torch.cuda.synchronize()
+    assert st2.status() == 0
+    out_ref, lse_ref = oracle.attend(a["q"], k2, v2, a["page_table"], len2, sel2, scnt2, u_accum=u2)
+    assert np.abs(st2.out.cpu().numpy() - out_ref).max() <= 1e-2
+    assert np.abs(st2.lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    assert np.abs(w.score_accum.cpu().numpy().astype(np.float64) - u2).max() <= 1e-4 + 1e-3 * np.abs(u2).max()
