@@ -51,3 +51,63 @@ def test_random_shapes(seed):
                 recent_pages=c["recent"])
     else:
         compare(w_cpu, st, sink_pages=c["sink"], recent_pages=c["recent"])
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_random_h2o_evictions(seed):
+    from test_gpu_h2o import check_retain
+    import oracle
+    from helpers import host_arrays
+    rng = np.random.default_rng(2000 + seed)
+    D = int(rng.choice([64, 128]))
+    H_kv = int(rng.choice([1, 2, 4]))
+    B = int(rng.integers(1, 5))
+    seq = [int(x) for x in rng.integers(1, 3000, size=B)]
+    budget = int(rng.integers(1, 1500))
+    recent = int(rng.integers(0, 1.2 * budget + 2))
+    w_cpu = wl.build("fz", 750 + seed, 0, seq, H_kv * int(rng.integers(1, 5)), H_kv, D, 64, "cpu",
+                     permute_pool=True, with_score_accum=True)
+    levels = int(rng.choice([0, 2, 16]))
+    if levels:
+        w_cpu.score_accum = torch.round(w_cpu.score_accum * levels) / levels
+    w, p, ws, keep_idx, keep_cnt = check_retain(w_cpu, budget, recent)
+    a = host_arrays(w_cpu)
+    k_ref, v_ref, u_ref, len_ref = oracle.h2o_compact(a["k"], a["v"], w_cpu.score_accum.numpy().astype(np.float64),
+                                                      a["page_table"], keep_idx.cpu().numpy(), keep_cnt.cpu().numpy())
+    new_lens = torch.zeros((w.B,), dtype=torch.int32, device="cuda")
+    binding.se_h2o_compact(p, w.k_cache, w.v_cache, w.score_accum, w.page_table, keep_idx, keep_cnt, new_lens, ws)
+    torch.cuda.synchronize()
+    assert binding.se_last_device_status(ws) == 0
+    assert np.array_equal(new_lens.cpu().numpy(), len_ref)
+    assert np.array_equal(wl.bf16_bits(w.k_cache), k_ref) and np.array_equal(wl.bf16_bits(w.v_cache), v_ref)
+    assert np.array_equal(w.score_accum.cpu().numpy().astype(np.float64), u_ref)
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_random_selection_reuse(seed):
+    from test_gpu_token import observe, check_scores, select, check_select, token_decode, check_attend
+    rng = np.random.default_rng(3000 + seed)
+    D = int(rng.choice([64, 128]))
+    H_kv = int(rng.choice([1, 2, 4]))
+    G = int(rng.integers(1, 9))
+    B = int(rng.integers(1, 5))
+    seq = [int(x) for x in rng.integers(1, 2500, size=B)]
+    prune = float(rng.choice([0.0, 0.2]))
+    budget, recent = int(rng.integers(0, 600)), int(rng.integers(0, 40))
+    if budget + recent == 0:
+        budget = 1
+    w_cpu = wl.build("fz", 760 + seed, 0, seq, H_kv * G, H_kv, D, 64, "cpu", permute_pool=True, prune_fraction=prune,
+                     poison_tail=True)
+    w = w_cpu.to("cuda")
+    st, keys = observe(w)
+    s_ref, present, s_gpu = check_scores(w_cpu, keys)
+    tok_idx, tok_cnt = select(st, keys, w, budget, recent)
+    check_select(w_cpu, s_ref, present, s_gpu, tok_idx, tok_cnt, budget, recent)
+    w1_cpu = wl.build("fz", 760 + seed, 1, seq, H_kv * G, H_kv, D, 64, "cpu", permute_pool=True, prune_fraction=prune,
+                      poison_tail=True)
+    w1 = w1_cpu.to("cuda")
+    p = binding.make_params(w.B, H_kv * G, H_kv, D, w.max_pages, w.num_phys_pages, (budget + recent + 15) // 16)
+    ws = binding.alloc_workspace(p, "cuda")
+    out, lse = token_decode(w1, p, ws, tok_idx, tok_cnt)
+    assert binding.se_last_device_status(ws) == 0
+    check_attend(w1_cpu, tok_idx, tok_cnt, out, lse)
