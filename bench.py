@@ -161,6 +161,15 @@ def algorithmic_bytes(w, sel_cnt, h2o: bool):
                 total=meta + kv + q + outlse + accum, present_pages=present, selected_pages=k_eff)
 
 
+def checksums(w):
+    """64-bit sums of the raw bits of the seeded inputs (reproducibility record, not arithmetic of the method)."""
+    def s64(t):
+        v = t.contiguous().view(torch.int32) if t.element_size() * t.numel() % 4 == 0 else t.contiguous().view(torch.int16)
+        return "%016x" % (int(v.sum(dtype=torch.int64).item()) & 0xFFFFFFFFFFFFFFFF)
+    return {"q": s64(w.q), "k_cache": s64(w.k_cache), "v_cache": s64(w.v_cache),
+            "page_table": s64(w.page_table), "seq_lens": s64(w.seq_lens)}
+
+
 def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0):
     fn = wl.CONFIGS[config]
     if batch:
@@ -487,6 +496,7 @@ def main():
                       else "inputs larger than L2 (%.0f MB touched per step)" % (working_set / 1e6),
                 "parallelism": "1 GPU" if world == 1 else "%d replicas, no collective" % world,
                 "global_batch": layers[0].B * world,
+                "checksums_layer0": checksums(layers[0]),
             },
             "algorithmic_bytes_per_step": total_bytes,
             "achieved_gbs": step_gbs * world,
