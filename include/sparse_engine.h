@@ -44,7 +44,8 @@
  *  - Inputs must be finite; behaviour with NaN/Inf in q, K, V is unspecified.
  *  - Physical page ids outside [0, num_phys_pages) and selected pages outside the
  *    request are never dereferenced: the access is skipped and a bit is set in the
- *    device status word (see se_last_device_status).
+ *    device status word (see se_last_device_status).  se_meta_update is the one exception:
+ *    it takes no workspace, hence has no status word, and skips such a page id silently.
  */
 #ifndef SPARSE_ENGINE_H_
 #define SPARSE_ENGINE_H_
@@ -120,12 +121,13 @@ int se_workspace_init(const se_params *p, void *workspace, void *stream);
  * equation): for every kv-head h and channel c of a page,
  *     meta[pid,h,0,c] = min_t K[pid,h,t,c],   meta[pid,h,1,c] = max_t K[pid,h,t,c]
  * over the tokens t of the page that lie below the request's length.
- *   first_tok == NULL : recompute only the page holding each request's newest token
- *                       ("new keys update the extrema of their pages"); run after the
- *                       token's K has been written to k_cache.
+ *   first_tok == NULL : incremental mode - recompute only the summary of the page that
+ *                       holds each request's newest token (same passage, the sentence after
+ *                       the score equation); run after the token's K is in k_cache.
  *   first_tok != NULL : [B] int32; recompute every page of request r from the page
  *                       holding token first_tok[r] on (0 = rebuild all, e.g. after prefill).
- * Pages with page_table == -1 and pages no request refers to are left untouched.  The
+ * Pages with page_table == -1, pages whose id is outside [0, num_phys_pages) (skipped without a
+ * report: this call has no status word) and pages no request refers to are left untouched.  The
  * result is exact (a min/max of bf16 values); -0 orders below +0.  Requests that alias
  * the same physical page write identical values.  A request's partially filled last
  * page must not be aliased by another request of a different length.
@@ -167,8 +169,8 @@ int se_page_select(const se_params *p, const void *q, const void *meta,
  * kv-head, over the tokens below the length, exactly as se_meta_update does - uses it for the
  * score and writes it to `meta`; every other page's summary is read from `meta` as usual.  Saves
  * the separate kernel of se_meta_update.  Results (meta, sel_idx, sel_cnt) are identical to the
- * two calls made one after the other.  (Quest summary and score equations, TopK; "new keys update
- * the extrema of their pages".)
+ * two calls made one after the other.  (Appendix A, Quest summary and score equations and the
+ * incremental-update sentence after them; TopK entry of the notation table.)
  */
 int se_page_select_fused(const se_params *p, const void *q, const void *k_cache, void *meta,
                          const int32_t *page_table, const int32_t *seq_lens,
@@ -234,7 +236,11 @@ int se_page_select_static(const se_params *p, const void *q, const void *meta,
  * se_page_select_scores - the scoring kernel; the fp32 page scores stay in the workspace - then
  * se_page_select_topk - the top-k kernel, which reads them.  One after the other on the same stream
  * they are exactly se_page_select (except in dense-layer mode, which only the single call takes);
- * they exist so that a profiler or a benchmark can time the two kernels apart.
+ * they exist so that a profiler or a benchmark can time the two kernels apart, and so that a test can
+ * read the scores: after se_page_select_scores the workspace holds, from byte offset 256 on,
+ * B*H_kv rows of P floats, P = max_pages rounded up to a multiple of 4; element b of row r*H_kv + h is
+ * the fp32 score of logical page b of request r for kv-head h, -inf where the page is absent;
+ * elements from ceil(len_r/16) on are not written.
  */
 int se_page_select_scores(const se_params *p, const void *q, const void *meta,
                           const int32_t *page_table, const int32_t *seq_lens,
@@ -317,8 +323,9 @@ int se_h2o_retain(const se_params *p, const float *score_accum, const int32_t *p
                   int32_t *keep_idx, int32_t *keep_cnt, void *workspace, void *stream);
 
 /*
- * H2O eviction as slot compaction ("KV outside R is evicted, while the scores of retained entries
- * persist"): for every (request, kv-head) the retained tokens keep_idx[r,h,0..keep_cnt) move, in
+ * H2O eviction as slot compaction of the retained set (Appendix A, H2O retention equation and the
+ * sentence after it: what is not retained leaves the cache, retained tokens keep their accumulated
+ * scores): for every (request, kv-head) the retained tokens keep_idx[r,h,0..keep_cnt) move, in
  * order, to token positions 0..keep_cnt-1 of the request - K row, V row and accumulated score of
  * position i become those of position keep_idx[r,h,i] - and new_seq_lens[r] = keep_cnt[r,0].
  * In place: k_cache, v_cache and score_accum are read and written; slots past the new length keep

@@ -172,6 +172,16 @@ def se_page_select_scores(*args, **kw) -> None:
     se_page_select(*args, entry="se_page_select_scores", **kw)
 
 
+def page_scores_view(p: SeParams, workspace: torch.Tensor) -> torch.Tensor:
+    """The fp32 page scores the scoring kernel left in ``workspace`` as a [B, H_kv, max_pages] view
+    (byte offset 256, rows of max_pages rounded up to a multiple of 4 floats; entries past a
+    request's last page are not written)."""
+    pitch = (p.max_pages + 3) // 4 * 4
+    n = p.B * p.H_kv * pitch
+    flat = workspace[256:256 + 4 * n].view(torch.float32)
+    return flat.view(p.B, p.H_kv, pitch)[:, :, :p.max_pages]
+
+
 def se_page_select_topk(*args, **kw) -> None:
     se_page_select(*args, entry="se_page_select_topk", **kw)
 
@@ -295,13 +305,16 @@ class DecodeState:
     selection and outputs.  Convenience for tests, the smoke check and the benchmark."""
 
     def __init__(self, w, k_max: Optional[int] = None, sm_scale: float = 0.0, sink_pages: int = 0,
-                 recent_pages: int = 0):
+                 recent_pages: int = 0, workspace: Optional[torch.Tensor] = None):
         dev = w.q.device
         self.w = w
         self.k_max = int(k_max if k_max is not None else max(w.budget // 16 + sink_pages + recent_pages, 1))
         self.p = make_params(w.B, w.H_q, w.H_kv, w.D, w.max_pages, w.num_phys_pages, self.k_max, sm_scale,
                              sink_pages=sink_pages, recent_pages=recent_pages)
-        self.workspace = alloc_workspace(self.p, dev)
+        # layers of one model step may share a workspace (their calls are ordered on one stream)
+        if workspace is not None and workspace.numel() < se_workspace_bytes(self.p):
+            raise SparseEngineError("shared workspace is smaller than se_workspace_bytes")
+        self.workspace = alloc_workspace(self.p, dev) if workspace is None else workspace
         self.meta = torch.zeros((w.num_phys_pages, w.H_kv, 2, w.D), dtype=torch.bfloat16, device=dev)
         self.sel_idx = torch.full((w.B, w.H_kv, self.k_max), -7, dtype=torch.int32, device=dev)
         self.sel_cnt = torch.full((w.B, w.H_kv), -7, dtype=torch.int32, device=dev)

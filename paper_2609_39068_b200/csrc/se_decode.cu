@@ -25,21 +25,6 @@
 
 #include "se_internal.h"
 
-// Optional per-warp phase timing for development builds (-DSE_DECODE_PROFILE); compiled out of
-// the library otherwise.
-#ifdef SE_DECODE_PROFILE
-__device__ long long g_dec_prof[8 * 4096];
-#define SE_PROF_DECL long long prof_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long prof_t_ = clock64(); const long long prof_t0_ = prof_t_;
-#define SE_PROF_LAP(i) { const long long t_ = clock64(); prof_[i] += t_ - prof_t_; prof_t_ = t_; }
-#define SE_PROF_ADD(i, v) { prof_[i] += (v); }
-#define SE_PROF_STORE(w) { if ((threadIdx.x & 31) == 0 && (w) < 4096) { prof_[7] = clock64() - prof_t0_; for (int i_ = 0; i_ < 8; ++i_) g_dec_prof[(w) * 8 + i_] = prof_[i_]; } }
-#else
-#define SE_PROF_DECL
-#define SE_PROF_LAP(i)
-#define SE_PROF_ADD(i, v)
-#define SE_PROF_STORE(w)
-#endif
-
 namespace se {
 
 namespace {
@@ -127,8 +112,6 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     // V (B operand, transposed): matrices {tok 0-7 | 8-15} fastest, then {chunk c | c+1}
     const int v_row = (lane & 7) + 8 * ((lane >> 3) & 1);
     const int v_chunk_add = lane >> 4;
-
-    SE_PROF_DECL
     uint32_t phases = 0;          // parity bit per stage
     int stage_c = 0, stage_i = 0; // next stage to consume / to fill
     bool failed = false;
@@ -282,8 +265,6 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             o_acc[nt][0] = 0.f; o_acc[nt][1] = 0.f; o_acc[nt][2] = 0.f; o_acc[nt][3] = 0.f;
         }
         float m_run = -INFINITY, l_run = 0.f;       // of head gid; l is this lane's share (its 4 token columns)
-        SE_PROF_LAP(0)
-
         while (!failed) {
             if (ce == n_ent) {                       // list exhausted: more slots of this segment left?
                 if (chunk_end >= seg_end) break;
@@ -300,8 +281,6 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
                 break;
             }
             phases ^= (1u << stage_c);
-            SE_PROF_LAP(1)
-            SE_PROF_ADD(5, 1)
             const uint32_t Ks = ring0 + stage_c * C::STAGEB;
             const uint32_t Vs = Ks + C::PAGEB;
             stage_c = (stage_c + 1 == nstage) ? 0 : stage_c + 1;
@@ -402,13 +381,9 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             }
             __syncwarp();     // all lanes are done with this stage before it is refilled
             ++ce;
-            SE_PROF_LAP(2)
             top_up();
-            SE_PROF_LAP(4)
         }
         if (failed) break;
-
-        SE_PROF_LAP(6)
         // ---- the four lanes of a head hold disjoint token columns: fold their l
         l_run += __shfl_xor_sync(kFull, l_run, 1);
         l_run += __shfl_xor_sync(kFull, l_run, 2);
@@ -443,8 +418,6 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
             }
         }
     }
-    SE_PROF_LAP(3)
-    SE_PROF_STORE(gw)
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // bounded wait for whatever this warp still has in flight before the CTA can retire
@@ -935,12 +908,6 @@ cudaError_t launch_token_decode(const se_params &p, const void *q, const void *k
 
 
 int decode_warps_per_cta() { return kDecWarps; }
-
-#ifdef SE_DECODE_PROFILE
-extern "C" int se_debug_decode_profile(long long *host_out, int n_warps) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_dec_prof, sizeof(long long) * 8 * n_warps);
-}
-#endif
 
 cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *k_cache,
                                  const void *v_cache, const int32_t *page_table,

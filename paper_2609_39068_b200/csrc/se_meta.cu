@@ -1,5 +1,6 @@
 // Quest page summaries: channel-wise min / max of K over the valid tokens of a page
-// (Appendix A, Quest summary equation; "new keys update the extrema of their pages").
+// (Appendix A, Quest summary equation; the incremental mode follows the sentence after the score
+// equation: a newly written key only changes the extrema of the page it lands in).
 //
 // One warp per (request, logical page, kv-head).  A K page of one head is a contiguous
 // [16, D] bf16 tile; a row is read with 16-byte loads by D/8 lanes, several rows per warp

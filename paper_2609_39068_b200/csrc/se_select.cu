@@ -21,25 +21,6 @@
 //                page and the list is ascending.
 #include "se_internal.h"
 
-// Optional per-warp phase timing for development builds (-DSE_SCORE_PROFILE); compiled out of the
-// library otherwise.
-#ifdef SE_SCORE_PROFILE
-__device__ long long g_score_prof[8 * 4096];
-__device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define SP_DECL long long prof_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long prof_t_ = clock64(); const long long prof_t0_ = prof_t_; prof_[5] = gtimer();
-#define SP_LAP(i) { const long long t_ = clock64(); prof_[i] += t_ - prof_t_; prof_t_ = t_; }
-#define SP_ADD(i, v) { prof_[i] += (v); }
-#define SP_STORE(w) { if ((threadIdx.x & 31) == 0 && (w) < 4096) { prof_[7] = clock64() - prof_t0_; prof_[6] = gtimer(); for (int i_ = 0; i_ < 8; ++i_) g_score_prof[(w) * 8 + i_] = prof_[i_]; } }
-extern "C" int se_debug_score_profile(long long *host_out, int n_warps) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_score_prof, sizeof(long long) * 8 * n_warps);
-}
-#else
-#define SP_DECL
-#define SP_LAP(i)
-#define SP_ADD(i, v)
-#define SP_STORE(w)
-#endif
-
 namespace se {
 
 namespace {
@@ -104,7 +85,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
              float *__restrict__ scores, int pitch, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
              uint32_t *status) {
     using C = ScoreCfg<D>;
-    SP_DECL
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // layout: [buffers: warps*2*BUF] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints] [lens: B ints]
     uint8_t *bufs = smem_raw;
@@ -330,8 +310,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     // ldmatrix row address of this lane inside a buffer: matrix (lane>>3) = {pages 0-7 | 8-15} x
     // {first | second 16-byte piece of the k16 step}
     const uint32_t lm_off = (uint32_t)(((lane & 7) + 8 * ((lane >> 3) & 1)) * C::PITCH + (lane >> 4) * 16);
-
-    SP_LAP(0)
     while (cur.unit >= 0) {
         // wait for the current buffer
         if (!mbar_wait(bar0 + slot * 8, (phases >> slot) & 1u)) {
@@ -339,8 +317,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             break;
         }
         phases ^= (1u << slot);
-        SP_LAP(1)
-        SP_ADD(4, 1)
         if (pend_slot == slot) {
             reduce_page(kpend, pend_pid, pend_h, buf0 + slot * C::BUF + pend_lane * C::PITCH);
             pend_slot = -1;
@@ -371,8 +347,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             if (cur.b0 + gid + 8 < cur.n_r) dst[gid + 8] = (pid_hi >= 0) ? s_hi * scale : ninf;
         }
         __syncwarp();        // every lane is done reading the buffer before it is refilled
-        SP_LAP(2)
-
         // refill the buffer just consumed with `nn` (its page-table entries arrived long ago)
         if (nn.unit >= 0) pid_nn = issue(nn, slot, pid_nn);
         // advance: cur <- nxt <- nn <- the batch after
@@ -386,9 +360,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
         next_batch(nn);
         pid_nn = load_pids(nn);
         slot ^= 1;
-        SP_LAP(3)
     }
-    SP_STORE(gw)
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // give the copy that may still be in flight a bounded chance to land before leaving
@@ -408,9 +380,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
 // over the per-thread counts then gives every thread the position of its pages in the
 // ascending output list.
 // ---------------------------------------------------------------------------------
-#ifndef SE_TOPK_MARK
-#define SE_TOPK_MARK(i)          // hook for an external timing probe; empty in the library
-#endif
 constexpr int kTopkBins = 2048;
 constexpr int kTopkBinBits = 11;
 constexpr int kTopkList = 32;        // bins with up to this many keys are ranked by brute force
@@ -431,7 +400,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
     __shared__ uint32_t s_lkey[kTopkList];
     __shared__ int s_lpage[kTopkList];
     __shared__ int s_ln;
-    SE_TOPK_MARK(9);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair = blockIdx.x;
     const int r = pair / H_kv;
@@ -463,7 +431,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
             keys[4 * j4 + c] = key;
         }
     }
-    SE_TOPK_MARK(0);
 #pragma unroll
     for (int e = 0; e < BPT; ++e) s_hist[tid * BPT + e] = 0;
     if (tid == 0) s_ln = 0;
@@ -503,8 +470,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
     }
     forced = min(forced, k_max);
     const int k_eff = min(min(k_pages, k_max - forced), present);      // candidates to take
-    SE_TOPK_MARK(1);
-
     if (k_eff + forced == 0) {
         for (int i = tid; i < k_max; i += THREADS) out[i] = -1;
         if (tid == 0) sel_cnt[pair] = 0;
@@ -542,7 +507,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
                 }
             }
             __syncthreads();
-            SE_TOPK_MARK(2);
             // the bin b with  #(keys in bins above b) < remaining <= #(keys in bins above or in b)
             int loc[BPT], sum = 0;
 #pragma unroll
@@ -564,7 +528,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
                 }
             }
             __syncthreads();
-            SE_TOPK_MARK(3);
             const int digit = (kTopkBins - 1) - s_res[0];
             const int inbin = s_res[2];
             remaining -= s_res[1];
@@ -596,7 +559,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
                     }
                 }
                 __syncthreads();
-                SE_TOPK_MARK(6);
                 // every warp ranks the (at most 32) collected keys on its own: lane i holds entry i,
                 // the entry that `remaining - 1` others precede is the threshold
                 {
@@ -613,7 +575,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
                     T_key = __shfl_sync(kFull, mk, owner);
                     T_page = __shfl_sync(kFull, mp, owner);
                 }
-                SE_TOPK_MARK(7);
                 break;
             }
         }
@@ -637,8 +598,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
         __syncthreads();
         T_page = s_res[5];
     }
-
-    SE_TOPK_MARK(4);
     // ---- ordered compaction
     uint32_t takemask = forcedmask;
     const int jT = T_page - base;            // page <= T_page  <=>  j <= jT
@@ -648,7 +607,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
         takemask |= (uint32_t)take << j;
     }
     int pos = cta_excl_scan<NW>(__popc(takemask), s_tot[3], lane, warp);
-    SE_TOPK_MARK(8);
     const int total = k_eff + forced;
     if (k_max <= kTopkBins) {
         // the list is put together in shared memory (the histogram is no longer needed) and
@@ -673,7 +631,6 @@ topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restri
         for (int i = total + tid; i < k_max; i += THREADS) out[i] = -1;
     }
     if (tid == 0) sel_cnt[pair] = k_eff + forced;
-    SE_TOPK_MARK(5);
 }
 
 // Dense-layer mode (budget >= context): every present page is selected, so there is nothing to

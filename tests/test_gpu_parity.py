@@ -49,7 +49,12 @@ def compare(w_cpu, st, rows=None, u_before=None, u_after=None, check_meta=True, 
     cnt = st.sel_cnt.cpu().numpy()[rows]
     differing = check_selection(sel, cnt, P, present, w_cpu.budget, sink_pages=sink_pages,
                                 recent_pages=recent_pages, seq_lens=sl)
-    assert differing <= max(1, (len(rows) * w_cpu.H_kv) // 4), "too many rows differ inside the tie band"
+    # A row may differ from the strict fp64 top-k only where the k-th and (k+1)-th scores are closer than
+    # the fp32 scoring error (~3e-7 relative) - far rarer than a gap inside the 1e-5 band (a few percent
+    # of the rows): more than 3 % of the rows differing means the scores are off, not tied.
+    n_rows = len(rows) * w_cpu.H_kv
+    assert differing <= max(1, (3 * n_rows + 99) // 100), \
+        "%d of %d rows (%.1f %%) differ from the strict top-k inside the tie band" % (differing, n_rows, 100.0 * differing / n_rows)
     for r in range(len(rows)):
         for h in range(w_cpu.H_kv):
             row = sel[r, h, :cnt[r, h]]
@@ -378,6 +383,109 @@ def test_bad_selection_sets_status_and_is_skipped():
     assert st.status() == 0                            # reading the status clears it
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G", [1, 4, 7, 8])
+def _score_magnitude(a, meta_bits, r, h, G, n_r):
+    """sm_scale * max over the group's heads of sum_c |q_c| * max(|min_c|, |max_c|) per page of (r, h):
+    the size of the terms the score sums, which is what its fp32 rounding error scales with."""
+    from helpers import bits_to_f64
+    pt = a["page_table"][r, :n_r]
+    pid = np.where(pt >= 0, pt, 0)
+    m = bits_to_f64(meta_bits[pid, h])                        # [n_r, 2, D]
+    big = np.maximum(np.abs(m[:, 0]), np.abs(m[:, 1]))         # [n_r, D]
+    qa = np.abs(bits_to_f64(a["q"][r, h * G:(h + 1) * G]))     # [G, D]
+    return (qa @ big.T).max(axis=0) / np.sqrt(qa.shape[1])
+
+
+def _check_scores(w_cpu, st, a):
+    got = binding.page_scores_view(st.p, st.workspace).cpu().numpy().astype(np.float64)
+    meta_bits = wl.bf16_bits(st.meta)
+    S, P, present = oracle.quest_scores(a["q"], meta_bits, a["page_table"], a["seq_lens"])
+    G = w_cpu.H_q // w_cpu.H_kv
+    n_checked, worst = 0, 0.0
+    for r in range(w_cpu.B):
+        n_r = (int(a["seq_lens"][r]) + 15) // 16
+        for h in range(w_cpu.H_kv):
+            row, ref, pres = got[r, h, :n_r], P[r, h, :n_r], present[r, :n_r]
+            assert np.all(np.isneginf(row[~pres])), "absent pages must score -inf"
+            mag = _score_magnitude(a, meta_bits, r, h, G, n_r)
+            assert np.all(mag[pres] >= np.abs(ref[pres]) * (1 - 1e-12))
+            rel = np.abs(row[pres] - ref[pres]) / mag[pres]
+            worst = max(worst, float(rel.max(initial=0.0)))
+            n_checked += int(pres.sum())
+    assert worst <= 2e-6, worst
+    return n_checked
+
+
+def test_page_scores_element_by_element(D, G):
+    """The fp32 page scores themselves (not only which pages win) against the oracle's fp64 scores:
+    every present page of every (request, kv-head) within 2e-6 of the size of the summed terms (<= 256 exact
+    bf16 products accumulated in fp32 by the tensor cores), -inf on absent pages.  Pruned pages, partial last pages, an empty
+    slot and outlier channels are in the mix."""
+    w_cpu = wl.build("scores", 815 + G, 0, [1234, 77, 600, 0, 16, 4000], 2 * G, 2, D, 160, "cpu", permute_pool=True,
+                     prune_fraction=0.2, poison_tail=True, outliers=True)
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    st.select(entry="se_page_select_scores")
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    n_checked = _check_scores(w_cpu, st, host_arrays(w_cpu))
+    assert n_checked > 300
+
+
+def test_page_scores_of_config2_element_by_element():
+    w_cpu = wl.config2("cpu")
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    st.select(entry="se_page_select_scores")
+    torch.cuda.synchronize()
+    assert _check_scores(w_cpu, st, host_arrays(w_cpu)) == 8 * 8 * 2048
+
+
+def _run_shard(w, accum):
+    st = binding.DecodeState(w)
+    short = (w.seq_lens - 1).clamp(min=0).contiguous()
+    ft = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    binding.se_meta_update(st.p, w.k_cache, w.page_table, short, st.meta, first_tok=ft)
+    u = w.score_accum.clone() if accum else None
+    st.step(score_accum=u)
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    return st, u
+
+
+@pytest.mark.parametrize("many_pairs", [True, False])
+def test_kv_head_shards_reproduce_the_unsharded_step(many_pairs):
+    """Tensor-parallel sharding by kv-head needs no exchange: the CUDA step run on the two shards of
+    wl.shard_kv_heads, concatenated, is the unsharded CUDA step.  With enough pairs that neither run splits
+    a pair (many_pairs) every output is bit-identical; with few pairs the split-K geometry differs
+    between the shapes, so out/lse/score_accum agree to fp32 rounding and the rest bit for bit."""
+    if many_pairs:
+        seq = [300 + 37 * i for i in range(100)]            # 100 requests x 8 kv-heads: 400 pairs per shard
+    else:
+        seq = [5000, 3000, 9000, 17]
+    w = wl.build("tp", 895, 0, seq, 16, 8, 128, 256, "cpu", permute_pool=True, prune_fraction=0.1,
+                 with_score_accum=True, poison_tail=True).to("cuda")
+    full, u_full = _run_shard(w, True)
+    if many_pairs:
+        assert binding.se_decode_num_splits(full.p) == 1
+    parts = [_run_shard(wl.shard_kv_heads(w, r, 2), True) for r in range(2)]
+    if many_pairs:
+        assert all(binding.se_decode_num_splits(st.p) == 1 for st, _ in parts)
+    cat = lambda f, dim: torch.cat([f(st, u) for st, u in parts], dim=dim)
+    assert torch.equal(cat(lambda st, u: st.meta.view(torch.int16), 1), full.meta.view(torch.int16))
+    assert torch.equal(cat(lambda st, u: st.sel_idx, 1), full.sel_idx)
+    assert torch.equal(cat(lambda st, u: st.sel_cnt, 1), full.sel_cnt)
+    out, lse, acc = cat(lambda st, u: st.out, 1), cat(lambda st, u: st.lse, 1), cat(lambda st, u: u, 1)
+    if many_pairs:
+        assert torch.equal(out, full.out) and torch.equal(lse, full.lse) and torch.equal(acc, u_full)
+    else:
+        assert (out - full.out).abs().max().item() <= 1e-5 and (lse - full.lse).abs().max().item() <= 1e-5
+        assert (acc - u_full).abs().max().item() <= 1e-5
+
+
 # ---------------------------------------------------------------- the named configurations
 
 def test_maximum_sizes_one_request():
@@ -411,16 +519,15 @@ def _gpu_built(cfg_fn, **kw):
     return w, w.to("cpu")
 
 
-def test_config3_full_size_sampled_requests():
+def test_config3_full_size_all_requests():
     w, w_cpu = _gpu_built(wl.config3)
     st = binding.DecodeState(w)
     st.rebuild_meta()
     st.step()
     torch.cuda.synchronize()
     assert st.status() == 0
-    lens = w_cpu.seq_lens.numpy()
-    rows = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 0, 17, 42, 63})
-    compare(w_cpu, st, rows=rows)
+    compare(w_cpu, st)                       # every one of the 64 requests
+    _check_scores(w_cpu, st, host_arrays(w_cpu))
 
 
 def test_config4_long_context_with_h2o():
@@ -436,14 +543,111 @@ def test_config4_long_context_with_h2o():
     assert abs(du.sum().item() - w.B * w.H_q) <= 1e-3 * w.B * w.H_q
 
 
-@pytest.mark.parametrize("layer", [0, 27])
-def test_config5_one_layer_sampled_requests(layer):
+@pytest.mark.parametrize("layer", [0, 13, 27])
+def test_config5_one_layer_all_requests(layer):
+    torch.cuda.empty_cache()
     w, w_cpu = _gpu_built(wl.config5, layer=layer)
     st = binding.DecodeState(w)
     st.rebuild_meta()
     st.step()
     torch.cuda.synchronize()
     assert st.status() == 0
-    lens = w_cpu.seq_lens.numpy()
-    rows = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 1, 64, 127})
-    compare(w_cpu, st, rows=rows)
+    compare(w_cpu, st)                       # every one of the 128 requests
+    _check_scores(w_cpu, st, host_arrays(w_cpu))
+
+
+def test_config5_28_layer_graph_replay_matches_oracle():
+    """The step the benchmark times - 28 layers captured in one CUDA graph, all layers sharing one
+    workspace - is the checked computation: after two replays the summaries, selections and outputs of
+    layers 0, 13 and 27 are compared with the oracle for every request, and the second replay must
+    reproduce the first bit for bit."""
+    torch.cuda.empty_cache()
+    n_layers, check = 28, (0, 13, 27)
+    layers = [wl.config5("cuda", layer=l) for l in range(n_layers)]
+    for w in layers[1:]:                     # the block table is per request, shared by all layers
+        w.page_table, w.seq_lens = layers[0].page_table, layers[0].seq_lens
+    states = [binding.DecodeState(layers[0])]
+    for w in layers[1:]:
+        states.append(binding.DecodeState(w, workspace=states[0].workspace))
+    # stale summaries for each request's newest page: the fused step has to refresh them
+    short = (layers[0].seq_lens - 1).contiguous()
+    ft = torch.zeros(layers[0].B, dtype=torch.int32, device="cuda")
+    for st in states:
+        binding.se_meta_update(st.p, st.w.k_cache, st.w.page_table, short, st.meta, first_tok=ft)
+
+    def step():
+        for st in states:
+            st.step()
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for st in states:
+        st.out.fill_(float("nan")); st.lse.fill_(float("nan")); st.sel_idx.fill_(-7); st.sel_cnt.fill_(-7)
+    graph.replay()
+    torch.cuda.synchronize()
+    first = {l: (states[l].out.clone(), states[l].lse.clone(), states[l].sel_idx.clone()) for l in check}
+    for st in states:
+        st.out.fill_(float("nan")); st.lse.fill_(float("nan")); st.sel_idx.fill_(-7); st.sel_cnt.fill_(-7)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert states[0].status() == 0
+    for st in states:
+        assert torch.isfinite(st.out).all() and int(st.sel_cnt.min()) >= 0
+    for l in check:
+        o, ls, si = first[l]
+        assert torch.equal(o, states[l].out) and torch.equal(ls, states[l].lse) and torch.equal(si, states[l].sel_idx)
+        compare(layers[l].to("cpu"), states[l])
+    del graph
+
+
+def test_config5_dense_first_layers_in_one_graph():
+    """Per-layer policy of the paper's Quest settings: the first two layers attend everything (dense-layer
+    mode: budget >= context), the others select under the budget - all captured in ONE graph with a
+    shared workspace.  Small version of the config-5 recipe (16 requests, 6 layers)."""
+    torch.cuda.empty_cache()
+    n_layers, n_dense = 6, 2
+    layers = [wl.config5("cuda", layer=l, B=16) for l in range(n_layers)]
+    for w in layers[1:]:
+        w.page_table, w.seq_lens = layers[0].page_table, layers[0].seq_lens
+    mp = layers[0].max_pages
+    big = binding.DecodeState(layers[0], k_max=mp)            # sized for the dense layers
+    states = [big] + [binding.DecodeState(w, k_max=mp if l + 1 < n_dense else None, workspace=big.workspace)
+                      for l, w in enumerate(layers[1:])]
+    for st in states:
+        st.rebuild_meta()
+
+    def step():
+        for l, st in enumerate(states):
+            if l < n_dense:
+                st.select_fused(budget=16 * mp)
+                st.decode()
+            else:
+                st.step()
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for st in states:
+        st.out.fill_(float("nan")); st.lse.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert big.status() == 0
+    for l, st in enumerate(states):
+        w_cpu = layers[l].to("cpu")
+        if l < n_dense:
+            w_cpu.budget = 16 * mp
+        compare(w_cpu, st)
+    del graph

@@ -71,7 +71,7 @@ def test_meta_min_below_max_and_idempotent():
 
 def test_meta_incremental_equals_rebuild():
     """Appending one token and updating only its page gives the same summaries as a
-    rebuild from scratch (new keys update the extrema of their page)."""
+    rebuild from scratch (Appendix A, Quest: a new key changes only its own page's summary)."""
     w, a = small_case(3, seq=(33, 48, 16, 5))
     ft = np.zeros(w.B, np.int32)
     grown = a["seq_lens"].copy()
