@@ -70,6 +70,11 @@ extern "C" {
 #define SE_DEV_BAD_SELECTION        2u  /* sel_idx entry outside the request / sel_cnt > k_max */
 #define SE_DEV_WAIT_TIMEOUT         4u  /* a bounded wait on an asynchronous copy gave up   */
 
+/* se_params.flags: by default the library picks the launch plan from the shape alone; these bits
+ * force one of the two plans of se_page_select (results are identical either way). */
+#define SE_FLAG_SELECT_TWO_KERNELS  1u  /* scoring kernel, then a top-k kernel (one CTA per pair)   */
+#define SE_FLAG_SELECT_ONE_KERNEL   2u  /* the scoring grid runs each pair's top-k itself           */
+
 typedef struct se_params {
     int32_t B;               /* requests in the batch (>= 1)                                */
     int32_t H_q;             /* query heads                                                 */
@@ -81,7 +86,7 @@ typedef struct se_params {
     int32_t num_phys_pages;  /* P_phys, pages in k_cache / v_cache / meta / score_accum     */
     int32_t k_max;           /* row stride of sel_idx, >= floor(budget / 16), 1..4096       */
     float   sm_scale;        /* logit scale; 0 selects 1/sqrt(D)                            */
-    uint32_t flags;          /* reserved, must be 0                                         */
+    uint32_t flags;          /* 0 or SE_FLAG_* bits                                         */
     int32_t sink_pages;      /* se_page_select: the first this many logical pages of every  */
     int32_t recent_pages;    /* request and the last this many are always selected, outside
                                 the budget (0 = pure top-k); see se_page_select             */
@@ -98,6 +103,10 @@ const char *se_strerror(int code);
  * The caller allocates that many bytes (256-byte aligned), runs se_workspace_init once,
  * and may then reuse the buffer for any number of calls with the same `p`.  Calls that
  * share a workspace must be ordered on the device (same stream or explicit dependencies).
+ * Calls whose `p` differ only in k_max, sm_scale, flags, sink_pages or recent_pages (the layers
+ * of one model step, some dense and some sparse) may share one workspace sized and
+ * initialised for the `p` with the largest se_workspace_bytes: the control block at its head
+ * depends on B and H_kv only.
  */
 size_t se_workspace_bytes(const se_params *p);
 
@@ -110,9 +119,10 @@ size_t se_workspace_bytes(const se_params *p);
 int se_decode_num_splits(const se_params *p);
 
 /*
- * Zeroes the control block (status word, work-queue counters) at the head of the
- * workspace.  Required once after allocation; the kernels leave the counters at zero
- * when they finish, so it need not be repeated.
+ * Zeroes the control block (status word, work-queue and per-pair arrival counters) at the
+ * head of the workspace.  Required once after allocation; the kernels leave the counters at
+ * zero when they finish, so it need not be repeated - except after a call that reported
+ * SE_DEV_WAIT_TIMEOUT, which may have left counters behind: run it again then.
  */
 int se_workspace_init(const se_params *p, void *workspace, void *stream);
 
@@ -237,8 +247,8 @@ int se_page_select_static(const se_params *p, const void *q, const void *meta,
  * se_page_select_topk - the top-k kernel, which reads them.  One after the other on the same stream
  * they are exactly se_page_select (except in dense-layer mode, which only the single call takes);
  * they exist so that a profiler or a benchmark can time the two kernels apart, and so that a test can
- * read the scores: after se_page_select_scores the workspace holds, from byte offset 256 on,
- * B*H_kv rows of P floats, P = max_pages rounded up to a multiple of 4; element b of row r*H_kv + h is
+ * read the scores: after se_page_select_scores the workspace holds, from byte offset
+ * 256 + (8*B*H_kv rounded up to a multiple of 256) on, B*H_kv rows of P floats, P = max_pages rounded up to a multiple of 4; element b of row r*H_kv + h is
  * the fp32 score of logical page b of request r for kv-head h, -inf where the page is absent;
  * elements from ceil(len_r/16) on are not written.
  */

@@ -113,9 +113,13 @@ def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
+SE_FLAG_SELECT_TWO_KERNELS = 1
+SE_FLAG_SELECT_ONE_KERNEL = 2
+
+
 def make_params(B, H_q, H_kv, D, max_pages, num_phys_pages, k_max, sm_scale=0.0, page_size=16,
-                sink_pages=0, recent_pages=0) -> SeParams:
-    return SeParams(B, H_q, H_kv, D, page_size, max_pages, num_phys_pages, k_max, float(sm_scale), 0,
+                sink_pages=0, recent_pages=0, flags=0) -> SeParams:
+    return SeParams(B, H_q, H_kv, D, page_size, max_pages, num_phys_pages, k_max, float(sm_scale), int(flags),
                     int(sink_pages), int(recent_pages))
 
 
@@ -174,16 +178,13 @@ def se_page_select_scores(*args, **kw) -> None:
 
 def page_scores_view(p: SeParams, workspace: torch.Tensor) -> torch.Tensor:
     """The fp32 page scores the scoring kernel left in ``workspace`` as a [B, H_kv, max_pages] view
-    (byte offset 256, rows of max_pages rounded up to a multiple of 4 floats; entries past a
-    request's last page are not written)."""
+    (they follow the control block: byte offset 256 + 8*B*H_kv rounded up to 256; rows of max_pages
+    rounded up to a multiple of 4 floats; entries past a request's last page are not written)."""
     pitch = (p.max_pages + 3) // 4 * 4
     n = p.B * p.H_kv * pitch
-    flat = workspace[256:256 + 4 * n].view(torch.float32)
+    off = 256 + (8 * p.B * p.H_kv + 255) // 256 * 256
+    flat = workspace[off:off + 4 * n].view(torch.float32)
     return flat.view(p.B, p.H_kv, pitch)[:, :, :p.max_pages]
-
-
-def se_page_select_topk(*args, **kw) -> None:
-    se_page_select(*args, entry="se_page_select_topk", **kw)
 
 
 def se_page_select_fused(p, q, k_cache, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,
@@ -305,12 +306,12 @@ class DecodeState:
     selection and outputs.  Convenience for tests, the smoke check and the benchmark."""
 
     def __init__(self, w, k_max: Optional[int] = None, sm_scale: float = 0.0, sink_pages: int = 0,
-                 recent_pages: int = 0, workspace: Optional[torch.Tensor] = None):
+                 recent_pages: int = 0, workspace: Optional[torch.Tensor] = None, flags: int = 0):
         dev = w.q.device
         self.w = w
         self.k_max = int(k_max if k_max is not None else max(w.budget // 16 + sink_pages + recent_pages, 1))
         self.p = make_params(w.B, w.H_q, w.H_kv, w.D, w.max_pages, w.num_phys_pages, self.k_max, sm_scale,
-                             sink_pages=sink_pages, recent_pages=recent_pages)
+                             sink_pages=sink_pages, recent_pages=recent_pages, flags=flags)
         # layers of one model step may share a workspace (their calls are ordered on one stream)
         if workspace is not None and workspace.numel() < se_workspace_bytes(self.p):
             raise SparseEngineError("shared workspace is smaller than se_workspace_bytes")

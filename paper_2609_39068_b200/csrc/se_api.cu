@@ -22,7 +22,8 @@ int validate(const se_params *p) {
     if (G < 1 || G > 8) return SE_ERR_UNSUPPORTED_SHAPE;
     if (p->max_pages < 1 || p->max_pages > 8192 || p->num_phys_pages < 1) return SE_ERR_INVALID_ARG;
     if (p->k_max < 1 || p->k_max > 4096) return SE_ERR_INVALID_ARG;
-    if (p->flags != 0) return SE_ERR_INVALID_ARG;
+    if ((p->flags & ~(SE_FLAG_SELECT_ONE_KERNEL | SE_FLAG_SELECT_TWO_KERNELS)) != 0) return SE_ERR_INVALID_ARG;
+    if ((p->flags & SE_FLAG_SELECT_ONE_KERNEL) && (p->flags & SE_FLAG_SELECT_TWO_KERNELS)) return SE_ERR_INVALID_ARG;
     if (p->sink_pages < 0 || p->recent_pages < 0 || p->sink_pages > 4096 || p->recent_pages > 4096)
         return SE_ERR_INVALID_ARG;
     if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return SE_ERR_INVALID_ARG;
@@ -76,6 +77,8 @@ WorkspaceLayout make_layout(const se_params &p) {
     const int GP = next_pow2(G);
     size_t off = 0;
     L.status = off;      off += 256;
+    L.pairctl = off;     off += align256(pairs * 2 * sizeof(uint32_t));
+    L.has_pairctl = true;
     L.scores = off;      off += align256(pairs * (size_t)score_pitch(p) * 4);
     L.partials = off;    off += align256((size_t)p.B * p.H_q * plan.max_splits * (p.D + 4) * 4);
     L.zbuf = off;        off += align256(pairs * (size_t)p.k_max * kPage * GP * 4);

@@ -19,6 +19,8 @@ constexpr unsigned kFull = 0xffffffffu;
 // ---------------------------------------------------------------------------------
 struct WorkspaceLayout {
     size_t status;          // 256 bytes: uint32 status word, work-queue counters of the score kernel
+    size_t pairctl;         // uint32 [B*H_kv] arrival counters (fused top-k, in-kernel merge); zero between calls
+    bool   has_pairctl;
     size_t scores;          // float  [B*H_kv][score_pitch]
     size_t partials;        // float  [B*H_q*max_splits*(D+2)]
     size_t zbuf;            // float  [B*H_kv*k_max*16*G]  logits kept for the H2O epilogue

@@ -383,8 +383,6 @@ def test_bad_selection_sets_status_and_is_skipped():
     assert st.status() == 0                            # reading the status clears it
 
 
-@pytest.mark.parametrize("D", [64, 128])
-@pytest.mark.parametrize("G", [1, 4, 7, 8])
 def _score_magnitude(a, meta_bits, r, h, G, n_r):
     """sm_scale * max over the group's heads of sum_c |q_c| * max(|min_c|, |max_c|) per page of (r, h):
     the size of the terms the score sums, which is what its fp32 rounding error scales with."""
@@ -417,6 +415,8 @@ def _check_scores(w_cpu, st, a):
     return n_checked
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G", [1, 4, 7, 8])
 def test_page_scores_element_by_element(D, G):
     """The fp32 page scores themselves (not only which pages win) against the oracle's fp64 scores:
     every present page of every (request, kv-head) within 2e-6 of the size of the summed terms (<= 256 exact
@@ -442,6 +442,52 @@ def test_page_scores_of_config2_element_by_element():
     st.select(entry="se_page_select_scores")
     torch.cuda.synchronize()
     assert _check_scores(w_cpu, st, host_arrays(w_cpu)) == 8 * 8 * 2048
+
+
+PLAN_CASES = dict(EDGE_CASES)
+PLAN_CASES.update({
+    "forced":       dict(seq=[2000, 50, 333, 64, 1, 0], H_q=8, H_kv=2, D=128, budget=256, permute_pool=True,
+                         prune_fraction=0.15, sink=4, recent=16),
+    "forced_only":  dict(seq=[40, 100], H_q=4, H_kv=2, D=64, budget=16, sink=3, recent=5),
+    "long_d64":     dict(seq=[131072, 5], H_q=8, H_kv=1, D=64, budget=16 * 300, permute_pool=True),
+    "all_selected": dict(seq=[3000, 200], H_q=8, H_kv=2, D=128, budget=16 * 188),
+    "max_sizes":    dict(seq=[131072], H_q=8, H_kv=1, D=128, budget=65536, permute_pool=True),
+})
+
+
+@pytest.mark.parametrize("name", sorted(PLAN_CASES))
+def test_both_selection_plans_give_the_same_selection(name):
+    """se_page_select has two launch plans (scoring grid that runs each pair's top-k itself / scoring
+    kernel + top-k kernel); whichever the shape picks, both must return the same pages, twice in a row."""
+    kw = dict(PLAN_CASES[name])
+    seq, sink, recent = kw.pop("seq"), kw.pop("sink", 0), kw.pop("recent", 0)
+    w = wl.build(name, 800, 0, seq, kw.pop("H_q"), kw.pop("H_kv"), kw.pop("D"), kw.pop("budget"), "cuda", **kw)
+    res = []
+    for flags in (binding.SE_FLAG_SELECT_TWO_KERNELS, binding.SE_FLAG_SELECT_ONE_KERNEL, 0):
+        st = binding.DecodeState(w, sink_pages=sink, recent_pages=recent, flags=flags)
+        st.rebuild_meta()
+        for rep in range(2):
+            st.sel_idx.fill_(-7)
+            st.sel_cnt.fill_(-7)
+            st.select() if rep == 0 else st.select_fused()
+            torch.cuda.synchronize()
+            assert st.status() == 0
+            res.append((st.sel_idx.clone(), st.sel_cnt.clone()))
+    for idx, cnt in res[1:]:
+        assert torch.equal(idx, res[0][0]) and torch.equal(cnt, res[0][1])
+
+
+def test_ties_with_the_one_kernel_plan():
+    w_cpu = wl.build("ties", 860, 0, [16 * 40, 16 * 700], 4, 1, 128, 16 * 8, "cpu")
+    w_cpu.k_cache[1:] = w_cpu.k_cache[0]
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w, flags=binding.SE_FLAG_SELECT_ONE_KERNEL)
+    st.rebuild_meta()
+    st.select()
+    st.decode()
+    torch.cuda.synchronize()
+    assert st.sel_idx.cpu()[0, 0].tolist() == list(range(8)) and st.sel_idx.cpu()[1, 0].tolist() == list(range(8))
+    compare(w_cpu, st)
 
 
 def _run_shard(w, accum):
