@@ -285,6 +285,15 @@ def main():
     working_set = total_bytes
     flush = working_set < 2 * L2_BYTES
     flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
+    flush_src = torch.zeros(2 * L2_BYTES // 4, dtype=torch.int32, device=dev) if flush else None
+    flush_sink = torch.zeros(1, dtype=torch.int32, device=dev) if flush else None
+
+    def flush_l2(i):
+        """Evicts the step's data from L2: a 252 MiB write, then a 252 MiB read of another buffer, so that
+        the lines the timed step displaces are clean (displacing the write's dirty lines would charge
+        the step one write-back per byte it reads)."""
+        flush_buf.fill_(i & 0xFF)
+        flush_sink.copy_(flush_src.max().reshape(1))
 
     graph = None
     if not args.no_graph:
@@ -315,7 +324,7 @@ def main():
         starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
         ends = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
         for i in range(K):
-            flush_buf.fill_(i & 0xFF)
+            flush_l2(i)
             starts[i].record()
             run_step()
             ends[i].record()
@@ -344,7 +353,7 @@ def main():
         if flush:
             tot = 0.0
             for i in range(iters):
-                flush_buf.fill_(i & 0xFF)
+                flush_l2(i)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(); fn(); b.record()
                 torch.cuda.synchronize()
@@ -366,6 +375,7 @@ def main():
         "se_page_select_scores": time_call(lambda: st0.select(entry="se_page_select_scores"), iters),
         "se_page_select_topk": time_call(lambda: st0.select(entry="se_page_select_topk"), iters),
         "se_page_select_fused": time_call(st0.select_fused, iters),
+        "se_decode_step": time_call(lambda: st0.step(u0), iters),
         "se_sparse_decode": time_call(lambda: st0.decode(u0), iters),
         "se_sparse_decode_splits": time_call(lambda: st0.decode(u0, entry="se_sparse_decode_splits"), iters),
         "se_combine": time_call(lambda: st0.decode(u0, entry="se_combine"), iters),
@@ -458,7 +468,7 @@ def main():
     a.record()
     for i in range(e2e_iters):
         if flush:
-            flush_buf.fill_(i & 0xFF)
+            flush_l2(i)
         e2e_step()
     b.record()
     barrier()
@@ -479,8 +489,7 @@ def main():
     if rank == 0:
         # score, top-k, decode (summary update fused into score); the merge kernel runs only when
         # the pairs are split or the H2O epilogue is on
-        merges = binding.se_decode_num_splits(states[0].p) > 1 or h2o
-        launches_per_step = n_layers * (3 + int(merges))
+        launches_per_step = n_layers * binding.se_decode_step_launches(states[0].p, layers[0].budget, h2o)
         line = {
             "metric": METRIC, "value": ms_per_step * 1e3, "unit": "us", "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -492,7 +501,7 @@ def main():
                 "page_size": 16, "budget_tokens": layers[0].budget, "storage_dtype": "bf16",
                 "present_pages": b0["present_pages"], "selected_pages": b0["selected_pages"],
                 "h2o_epilogue": h2o, "cuda_graph": graph is not None,
-                "l2": ("flushed with a %d MiB write before every step" % (2 * L2_BYTES >> 20)) if flush
+                "l2": ("flushed before every step: a %d MiB write, then a %d MiB read (leaves clean lines)" % (2 * L2_BYTES >> 20, 2 * L2_BYTES >> 20)) if flush
                       else "inputs larger than L2 (%.0f MB touched per step)" % (working_set / 1e6),
                 "parallelism": "1 GPU" if world == 1 else "%d replicas, no collective" % world,
                 "global_batch": layers[0].B * world,

@@ -70,11 +70,6 @@ extern "C" {
 #define SE_DEV_BAD_SELECTION        2u  /* sel_idx entry outside the request / sel_cnt > k_max */
 #define SE_DEV_WAIT_TIMEOUT         4u  /* a bounded wait on an asynchronous copy gave up   */
 
-/* se_params.flags: by default the library picks the launch plan from the shape alone; these bits
- * force one of the two plans of se_page_select (results are identical either way). */
-#define SE_FLAG_SELECT_TWO_KERNELS  1u  /* scoring kernel, then a top-k kernel (one CTA per pair)   */
-#define SE_FLAG_SELECT_ONE_KERNEL   2u  /* the scoring grid runs each pair's top-k itself           */
-
 typedef struct se_params {
     int32_t B;               /* requests in the batch (>= 1)                                */
     int32_t H_q;             /* query heads                                                 */
@@ -86,7 +81,7 @@ typedef struct se_params {
     int32_t num_phys_pages;  /* P_phys, pages in k_cache / v_cache / meta / score_accum     */
     int32_t k_max;           /* row stride of sel_idx, >= floor(budget / 16), 1..4096       */
     float   sm_scale;        /* logit scale; 0 selects 1/sqrt(D)                            */
-    uint32_t flags;          /* 0 or SE_FLAG_* bits                                         */
+    uint32_t flags;          /* reserved, must be 0                                         */
     int32_t sink_pages;      /* se_page_select: the first this many logical pages of every  */
     int32_t recent_pages;    /* request and the last this many are always selected, outside
                                 the budget (0 = pure top-k); see se_page_select             */
@@ -112,9 +107,9 @@ size_t se_workspace_bytes(const se_params *p);
 
 /*
  * Split-K geometry se_sparse_decode uses for `p` (host, pure): the number of splits every
- * (request, kv-head) pair is cut into, or 0 if `p` is invalid.  1 means every pair is attended by
- * one worker, which writes out/lse itself; the merge kernel then only runs for the H2O epilogue.
- * Informational: lets a caller count kernel launches or size its own tooling.
+ * (request, kv-head) pair is cut into (warps, or whole CTAs when there is at most one pair per
+ * SM), or 0 if `p` is invalid.  1 means every pair is attended by one worker, which writes out/lse
+ * itself.  Informational: lets a caller size its own tooling.
  */
 int se_decode_num_splits(const se_params *p);
 
@@ -208,6 +203,31 @@ int se_sparse_decode(const se_params *p, const void *q, const void *k_cache,
                      const int32_t *seq_lens, const int32_t *sel_idx,
                      const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
                      void *workspace, void *stream);
+
+/*
+ * One decode step of a layer in one call: se_meta_update(first_tok = NULL), se_page_select and
+ * se_sparse_decode, with the same results (meta, sel_idx, sel_cnt, out, lse, score_accum; Appendix A,
+ * Quest summary and score equations, TopK, selected-attention and H2O equations).  The call picks
+ * the launch plan from the shape alone:
+ *   - budget_tokens/16 < max_pages (a sparse layer): the scoring kernel (which also refreshes the
+ *     summary of each request's newest page) leaves the fp32 page scores in the workspace, and the
+ *     attention kernel selects each pair's pages from them in its prologue - no top-k kernel, no
+ *     round trip of the selection through memory before the first page is fetched.  With at most one
+ *     (request, kv-head) pair per SM the attention kernel also merges its split partials itself, so
+ *     the step is two launches (three with score_accum, whose epilogue needs the final lse).
+ *     Shapes the in-kernel top-k does not cover (more than 4096 pages per request together with
+ *     more than one pair per SM) run the top-k kernel in between.
+ *   - budget_tokens/16 >= max_pages and k_max >= max_pages (a dense layer, e.g. the first layers of
+ *     a model whose remaining layers are sparse): summary update, list of all present pages,
+ *     attention.
+ * sel_idx / sel_cnt are outputs here.  se_decode_step_launches tells how many kernels a step
+ * launches for `p` (host, pure; 0 if the arguments are invalid).
+ */
+int se_decode_step(const se_params *p, const void *q, const void *k_cache, const void *v_cache, void *meta,
+                   const int32_t *page_table, const int32_t *seq_lens, int32_t budget_tokens,
+                   int32_t *sel_idx, int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                   void *workspace, void *stream);
+int se_decode_step_launches(const se_params *p, int32_t budget_tokens, int with_score_accum);
 
 /*
  * se_page_select without any caller-provided scratch.  (The paper has no counterpart: this entry

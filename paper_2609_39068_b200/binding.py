@@ -25,7 +25,7 @@ EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_decode_num_spl
            "se_page_select", "se_page_select_scores", "se_page_select_topk", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
            "se_last_device_status", "se_h2o_retain", "se_h2o_compact", "se_observe_decode", "se_token_select",
            "se_token_decode",
-           "se_page_select_static")
+           "se_page_select_static", "se_decode_step", "se_decode_step_launches")
 SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -82,11 +82,13 @@ def load(build_if_missing: bool = True):
     lib.se_h2o_retain.argtypes = [pp, fp, i32p, i32p, ctypes.c_int32, ctypes.c_int32, i32p, i32p, vp, vp]
     lib.se_h2o_compact.argtypes = [pp, vp, vp, fp, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp]
     lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
+    lib.se_decode_step.argtypes = [pp, vp, vp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, fp, fp, fp, vp, vp]
+    lib.se_decode_step_launches.argtypes = [pp, ctypes.c_int32, ctypes.c_int]
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
                  "se_sparse_decode", "se_sparse_decode_splits", "se_combine", "se_last_device_status",
                  "se_h2o_retain", "se_h2o_compact", "se_decode_num_splits", "se_page_select_static",
                  "se_observe_decode", "se_token_select", "se_token_decode", "se_page_select_scores",
-                 "se_page_select_topk"):
+                 "se_page_select_topk", "se_decode_step", "se_decode_step_launches"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -111,10 +113,6 @@ def _ptr(t: Optional[torch.Tensor], dtype, name: str):
 
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
-
-
-SE_FLAG_SELECT_TWO_KERNELS = 1
-SE_FLAG_SELECT_ONE_KERNEL = 2
 
 
 def make_params(B, H_q, H_kv, D, max_pages, num_phys_pages, k_max, sm_scale=0.0, page_size=16,
@@ -219,6 +217,22 @@ def se_sparse_decode_splits(*args, **kw) -> None:
 
 def se_combine(*args, **kw) -> None:
     se_sparse_decode(*args, entry="se_combine", **kw)
+
+
+def se_decode_step(p, q, k_cache, v_cache, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt, out, lse,
+                   workspace, score_accum=None) -> None:
+    _check(load().se_decode_step(ctypes.byref(p), _ptr(q, torch.bfloat16, "q"),
+                                 _ptr(k_cache, torch.bfloat16, "k_cache"), _ptr(v_cache, torch.bfloat16, "v_cache"),
+                                 _ptr(meta, torch.bfloat16, "meta"), _ptr(page_table, torch.int32, "page_table"),
+                                 _ptr(seq_lens, torch.int32, "seq_lens"), int(budget_tokens),
+                                 _ptr(sel_idx, torch.int32, "sel_idx"), _ptr(sel_cnt, torch.int32, "sel_cnt"),
+                                 _ptr(out, torch.float32, "out"), _ptr(lse, torch.float32, "lse"),
+                                 _ptr(score_accum, torch.float32, "score_accum"),
+                                 _ptr(workspace, torch.uint8, "workspace"), _stream()), "se_decode_step")
+
+
+def se_decode_step_launches(p: SeParams, budget_tokens: int, with_score_accum: bool) -> int:
+    return int(load().se_decode_step_launches(ctypes.byref(p), int(budget_tokens), int(bool(with_score_accum))))
 
 
 def se_page_select_static(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,
@@ -344,15 +358,18 @@ class DecodeState:
                              self.w.budget if budget is None else budget, self.sel_idx, self.sel_cnt,
                              self.workspace)
 
-    def step(self, score_accum=None, fused: bool = True):
-        """One decode step of the layer: newest-page summary, selection, attention.  ``fused``
-        folds the summary update into the scoring kernel (se_page_select_fused)."""
+    def step(self, score_accum=None, fused: bool = True, budget: Optional[int] = None):
+        """One decode step of the layer: newest-page summary, selection, attention.  ``fused`` =
+        se_decode_step (one call, launch plan picked by the library); otherwise the three separate
+        calls se_meta_update, se_page_select, se_sparse_decode."""
         if fused:
-            self.select_fused()
+            se_decode_step(self.p, self.w.q, self.w.k_cache, self.w.v_cache, self.meta, self.w.page_table,
+                           self.w.seq_lens, self.w.budget if budget is None else budget, self.sel_idx,
+                           self.sel_cnt, self.out, self.lse, self.workspace, score_accum=score_accum)
         else:
             self.update_meta()
-            self.select()
-        self.decode(score_accum)
+            self.select(budget)
+            self.decode(score_accum)
 
     def status(self) -> int:
         return se_last_device_status(self.workspace)

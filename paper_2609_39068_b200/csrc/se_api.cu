@@ -22,8 +22,7 @@ int validate(const se_params *p) {
     if (G < 1 || G > 8) return SE_ERR_UNSUPPORTED_SHAPE;
     if (p->max_pages < 1 || p->max_pages > 8192 || p->num_phys_pages < 1) return SE_ERR_INVALID_ARG;
     if (p->k_max < 1 || p->k_max > 4096) return SE_ERR_INVALID_ARG;
-    if ((p->flags & ~(SE_FLAG_SELECT_ONE_KERNEL | SE_FLAG_SELECT_TWO_KERNELS)) != 0) return SE_ERR_INVALID_ARG;
-    if ((p->flags & SE_FLAG_SELECT_ONE_KERNEL) && (p->flags & SE_FLAG_SELECT_TWO_KERNELS)) return SE_ERR_INVALID_ARG;
+    if (p->flags != 0) return SE_ERR_INVALID_ARG;
     if (p->sink_pages < 0 || p->recent_pages < 0 || p->sink_pages > 4096 || p->recent_pages > 4096)
         return SE_ERR_INVALID_ARG;
     if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return SE_ERR_INVALID_ARG;
@@ -48,14 +47,31 @@ float effective_scale(const se_params &p) {
 
 int decode_warps_per_cta();
 
-// Split-K geometry: every (request, kv-head) pair is cut into the same number of splits.  With two
-// or more pairs per SM the pairs themselves fill the machine (a few warps per SM, each with a deep
-// copy pipeline, already saturate HBM) and splitting would only add the merge; below that, as many
-// splits as the persistent warps of the grid can take in one round (one unit per warp).
-DecodePlan make_decode_plan(const se_params &p) {
+// Launch geometry of the attention step, from the shape alone.
+//  - at most one pair per SM: CTA units.  A pair gets cpp = min(SMs / pairs, ceil(k_max / 8)) CTAs (a
+//    warp should hold at least one page); up to kMergeInKernelMax of them are merged by the
+//    last-arriving CTA, more by the merge kernel.
+//  - fewer than two pairs per SM: warp units, every pair cut into as many splits as the persistent
+//    warps of the grid can take in one round; the merge kernel combines them.
+//  - two or more pairs per SM: warp units, one per pair (a few warps per SM, each with a deep copy
+//    pipeline, already saturate HBM; splitting would only add the merge).
+DecodePlan make_decode_plan(const se_params &p, bool warp_units_only) {
     DecodePlan plan;
     const int warps_per_cta = decode_warps_per_cta();
     const long long pairs = (long long)p.B * p.H_kv;
+    plan.cta_units = !warp_units_only && pairs <= kAssumedSMs;
+    plan.merge_in_kernel = false;
+    if (plan.cta_units) {
+        long long cpp = kAssumedSMs / pairs;
+        const long long useful = (p.k_max + warps_per_cta - 1) / warps_per_cta;
+        if (cpp > useful) cpp = useful;
+        if (cpp < 1) cpp = 1;
+        plan.max_splits = (int)cpp;
+        plan.pages_per_split = (int)((p.k_max + cpp - 1) / cpp);
+        plan.merge_in_kernel = cpp <= 8;
+        plan.grid = (int)(pairs * cpp);
+        return plan;
+    }
     const long long warps = (long long)kAssumedSMs * warps_per_cta;
     long long splits = warps / pairs;
     if (splits < 1 || pairs >= 2LL * kAssumedSMs) splits = 1;
@@ -69,9 +85,17 @@ DecodePlan make_decode_plan(const se_params &p) {
     return plan;
 }
 
+// The attention kernel selects the pages itself where a whole CTA works on one pair (cta_topk in the
+// prologue: 2-5 us).  With warp units a warp would have to run the top-k alone: measured 10 us (256
+// pages) to 45 us (4096 pages) per pair against 7.5 us for the top-k kernel over all 512 pairs of
+// config 3, so those shapes keep the top-k kernel.
+bool select_in_decode_ok(const se_params &p) { return make_decode_plan(p).cta_units; }
+
 WorkspaceLayout make_layout(const se_params &p) {
     WorkspaceLayout L;
     const DecodePlan plan = make_decode_plan(p);
+    const DecodePlan plan_w = make_decode_plan(p, true);       // observation / token layers use warp units
+    const int max_splits = plan.max_splits > plan_w.max_splits ? plan.max_splits : plan_w.max_splits;
     const size_t pairs = (size_t)p.B * p.H_kv;
     const int G = p.H_q / p.H_kv;
     const int GP = next_pow2(G);
@@ -80,10 +104,10 @@ WorkspaceLayout make_layout(const se_params &p) {
     L.pairctl = off;     off += align256(pairs * 2 * sizeof(uint32_t));
     L.has_pairctl = true;
     L.scores = off;      off += align256(pairs * (size_t)score_pitch(p) * 4);
-    L.partials = off;    off += align256((size_t)p.B * p.H_q * plan.max_splits * (p.D + 4) * 4);
+    L.partials = off;    off += align256((size_t)p.B * p.H_q * max_splits * (p.D + 4) * 4);
     L.zbuf = off;        off += align256(pairs * (size_t)p.k_max * kPage * GP * 4);
     L.total = off;
-    L.max_splits = plan.max_splits;
+    L.max_splits = max_splits;
     return L;
 }
 
@@ -217,10 +241,56 @@ static int sparse_decode_stages(const se_params *p, const void *q, const void *k
                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
             return SE_ERR_CUDA;
     }
-    cudaError_t e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens, sel_idx,
-                                         sel_cnt, out, lse, score_accum, tok_keys, workspace, L, stages,
+    // the kernels only read the caller's selection here (from_scores == nullptr)
+    cudaError_t e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens,
+                                         const_cast<int32_t *>(sel_idx), const_cast<int32_t *>(sel_cnt), nullptr, out,
+                                         lse, score_accum, tok_keys, workspace, L, stages,
                                          static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+// What se_decode_step launches for `p`: 0 = dense layer (summary update, list of all pages, attention),
+// 1 = scoring kernel + attention kernel that selects in its prologue, 2 = scoring, top-k kernel, attention.
+static int step_plan(const se_params &p, int k_pages) {
+    if (k_pages >= p.max_pages && p.k_max >= p.max_pages) return 0;
+    return select_in_decode_ok(p) ? 1 : 2;
+}
+
+int se_decode_step(const se_params *p, const void *q, const void *k_cache, const void *v_cache, void *meta,
+                   const int32_t *page_table, const int32_t *seq_lens, int32_t budget_tokens, int32_t *sel_idx,
+                   int32_t *sel_cnt, float *out, float *lse, float *score_accum, void *workspace, void *stream) {
+    int rc = validate(p);
+    if (rc != SE_OK) return rc;
+    if (!q || !k_cache || !v_cache || !meta || !page_table || !seq_lens || !sel_idx || !sel_cnt || !out || !lse ||
+        !workspace)
+        return SE_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(meta) || !aligned16(page_table) ||
+        !aligned16(seq_lens) || !aligned16(sel_idx) || !aligned16(sel_cnt) || !aligned16(out) || !aligned16(lse) ||
+        !aligned16(score_accum) || !aligned16(workspace))
+        return SE_ERR_MISALIGNED;
+    if (budget_tokens < kPage) return SE_ERR_INVALID_ARG;
+    const int k_pages = budget_tokens / kPage;
+    if (k_pages + p->sink_pages + p->recent_pages > p->k_max) return SE_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(*p);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int plan = step_plan(*p, k_pages);
+    // plan 1: only the scoring kernel of the selection runs (stages = 1); the scores stay in the workspace
+    cudaError_t e = launch_page_select(*p, q, meta, k_cache, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
+                                       workspace, L, s, plan == 1 ? 1 : 3);
+    if (e != cudaSuccess) return SE_ERR_CUDA;
+    const SelectFromScores from_scores = {k_pages};
+    e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
+                             plan == 1 ? &from_scores : nullptr, out, lse, score_accum, nullptr, workspace, L, 3, s);
+    return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
+}
+
+int se_decode_step_launches(const se_params *p, int32_t budget_tokens, int with_score_accum) {
+    if (validate(p) != SE_OK || budget_tokens < kPage) return 0;
+    const int plan = step_plan(*p, budget_tokens / kPage);
+    const DecodePlan dp = make_decode_plan(*p);
+    const bool merged = dp.max_splits == 1 || (dp.cta_units && dp.merge_in_kernel);
+    const int attention = 1 + ((!merged || with_score_accum) ? 1 : 0);
+    return (plan == 1 ? 1 : 2) + attention;
 }
 
 int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,

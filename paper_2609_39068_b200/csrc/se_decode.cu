@@ -1,49 +1,63 @@
-// Split-K paged attention over the selected pages, log-sum-exp merge and the H2O epilogue
+// Paged attention over the selected pages, log-sum-exp merge and the H2O epilogue
 // (Appendix A, selected-attention equation and H2O accumulated-score equation).
 //
-// decode_kernel  Every warp is an autonomous pipeline.  The selected pages of all
-//                (request, kv-head) pairs form one flat list of pairs*k_max slots; each warp
-//                owns an equal contiguous slice of it, so a pair is split over as many
-//                warps as its slots span (split-K) and all warps carry the same load.
-//                K and V pages ([16 tokens, D] bf16, contiguous per head) are fetched by TMA
-//                tensor copies (2-D tiles of 16 rows x 64 channels, 128-byte swizzle, one
-//                mbarrier per ring stage) so that ldmatrix reads them without bank conflicts.
-//                Per page and for the G query heads of the kv-head at once:
-//                    S^T[head, token] = Q[head, :] . K[token, :]^T      (m16n8k16, fp32 accumulate)
-//                    online softmax in base 2 on the accumulator fragments
-//                    O[head, :]      += P[head, token] . V[token, :]    (P split into two bf16 terms)
-//                The accumulator layout of S^T is the A-operand layout of P, so the
-//                probabilities never leave registers.  A warp that holds all pages of a pair
-//                writes out/lse itself; otherwise it stores a partial (acc, m, l).
-//                An earlier plain-FMA version of this kernel needed ~1050 warp instructions per
-//                page (8 KB) and was issue-bound at 65 % of the copy bandwidth.
-// combine_kernel merges the split partials of every pair (one warp per query head, so the
-//                merge of many splits is spread wide instead of falling on one warp) and adds
-//                exp(z - lse), summed over the query heads of the kv-head, to the accumulated
-//                score of every attended token slot (the H2O epilogue).
+// Two attention kernels share the per-page arithmetic (WarpAttn) and the per-warp copy pipeline
+// (attend_range); which one runs follows from the shape alone (make_decode_plan):
+//
+// decode_kernel      many (request, kv-head) pairs.  Persistent grid, every warp an autonomous
+//                    pipeline working through (pair, split) units; with two or more pairs per SM
+//                    a pair is one unit and its warp writes out/lse itself, otherwise the pair is cut
+//                    into splits whose partials (acc, m, l) combine_kernel merges.
+// decode_cta_kernel  at most one pair per SM.  A CTA is one (pair, CTA-split); its eight warps share
+//                    the CTA's pages, their partials are merged through shared memory, and when a
+//                    pair has several CTAs the last one to arrive (an atomic ticket: nobody waits)
+//                    merges the CTAs' partials - no merge kernel, no partials of single warps.
+//
+// decode_cta_kernel can take the selection from the page scores themselves (kSelect): the CTA runs
+// the top-k in its prologue (se_topk.cuh: cta_topk), while the shared-memory ring is still empty and
+// serves as its scratch; the list is also written to sel_idx / sel_cnt.  That removes the top-k
+// kernel and the selection's round trip from the step.  (With warp units a warp would have to run the
+// top-k alone, which is slower than the top-k kernel: those shapes keep it.)
+//
+// Per page, for the G query heads of the kv-head at once:
+//     S^T[head, token] = Q[head, :] . K[token, :]^T      (m16n8k16, fp32 accumulate)
+//     online softmax in base 2 on the accumulator fragments
+//     O[head, :]      += P[head, token] . V[token, :]    (P split into two bf16 terms)
+// K and V pages ([16 tokens, D] bf16, contiguous per head) arrive by one 3-D TMA tensor copy each
+// (64 channels x 16 rows x D/64 halves, 128-byte swizzle, one mbarrier per ring stage), so ldmatrix
+// reads them without bank conflicts.  The accumulator layout of S^T is the A-operand layout of P, so
+// the probabilities never leave registers.
+//
+// combine_kernel     merges split partials where the attention kernel did not (one warp per query
+//                    head) and adds exp(z - lse), summed over the query heads of the kv-head, to the
+//                    accumulated score of every attended token slot (the H2O epilogue).
 #include <cuda.h>
 
 #include "se_internal.h"
+#include "se_topk.cuh"
 
 namespace se {
 
 namespace {
 
 constexpr int kDecWarps = 8;
-constexpr int kChunk = 128;              // selected-page slots looked up at once
+constexpr int kChunk = 128;              // selected pages looked up at once
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileBytes = kPage * 128;  // one TMA box: 16 rows x 64 bf16
+constexpr int kMergeInKernelMax = 8;     // CTA-splits per pair the last-arriving CTA merges itself
 
 template <int D>
 struct DecCfg {
-    static constexpr int HALVES = D / 64;                      // 64-channel tiles per page
     static constexpr int PAGEB = kPage * D * 2;                // bytes of one K (or V) page
     static constexpr int STAGEB = 2 * PAGEB;                   // K tiles then V tiles
     static constexpr int MAXST = 8;                            // most stages one warp can hold
-    // Stages a CTA shares out among its busy warps.  More copies in flight than this made the
-    // kernel slower, not faster (measured: 24 pages in flight per SM lose 3 % against 16 to 20).
+    // Stages a CTA of decode_kernel shares out among its busy warps.  More copies in flight than
+    // this made that kernel slower, not faster (measured: 24 pages in flight per SM lose 3 %
+    // against 16 to 20).
     static constexpr int CTA_STAGES = 20 * (128 / D);
+    // decode_cta_kernel: three stages for each of the eight warps
+    static constexpr int CTA_STAGES_SPLIT = 24 * (128 / D);
     static constexpr int KSTEPS = D / 16;
     static constexpr int NTILES = D / 8;                       // n8 tiles of the output
     static constexpr int PSTRIDE = D + 4;                      // floats per partial row
@@ -64,106 +78,197 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
-template <int D, bool kObserve>
-__global__ void __launch_bounds__(kDecWarps * 32, 1)
-decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
-              const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
-              const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ sel_idx,
-              const int32_t *__restrict__ sel_cnt, float *__restrict__ out, float *__restrict__ lse,
-              float *__restrict__ partials, float *__restrict__ zbuf, uint32_t *__restrict__ tok_keys,
-              int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
-              int max_splits, float scale_log2, uint32_t *status) {
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------
+// Per-warp attention state: Q fragments, output accumulators and the running softmax statistics
+// of the G query heads of one kv-head.  Lane (gid = lane >> 2, tid4 = lane & 3) holds head row gid.
+// ---------------------------------------------------------------------------------
+template <int D>
+struct WarpAttn {
     using C = DecCfg<D>;
-    extern __shared__ uint8_t smem_dyn[];
-    // tiles must sit on 1024-byte boundaries for the 128-byte swizzle pattern
-    uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // The CTA's stages are shared out among the warps that have work: warp w of this CTA is busy iff
-    // its first unit w*gridDim.x + blockIdx.x exists, so the busy warps are the lowest ones.  Every
-    // busy warp gets the same number of stages (warps with unequal pipelines finish apart).
-    int busy = (B * H_kv * max_splits - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    busy = busy < 1 ? 1 : (busy > kDecWarps ? kDecWarps : busy);
-    const int nstage = warp < busy ? min(C::MAXST, C::CTA_STAGES / busy) : 0;
-    uint8_t *ring = smem_al + (size_t)(warp * nstage) * C::STAGEB;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB) + warp * C::MAXST;
-    if (lane == 0) {
-        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 2);
-        mbar_fence_init();
+    uint32_t qa[C::KSTEPS][2];       // Q as the A operand: row gid = query head gid (rows >= G and 8..15 zero)
+    float o_acc[C::NTILES][4];       // elements 0,1: p_hi products, 2,3: p_lo products (added in finish())
+    float m_run, l_run;              // of head gid; l is this lane's share (its 4 token columns) until finish()
+    // ldmatrix lane offsets inside a 16x128-byte swizzled tile (byte offset of the lane's row, its row & 7,
+    // and which of the two 16-byte chunks of a pair it addresses)
+    int k_rowoff, k_swz, k_chunk_add;    // K (B operand, not transposed): matrices {tok 0-7 | 8-15} x {chunk c | c+1}
+    int v_rowoff, v_swz, v_chunk_add, v_row;   // V (transposed): matrices {tok 0-7 | 8-15} fastest, then {chunk c | c+1}
+    int t0;                              // first token column of this lane
+
+    __device__ __forceinline__ void init_lane(int lane) {
+        const int k_row = (lane & 7) + 8 * (lane >> 4);
+        k_rowoff = k_row * 128;
+        k_swz = k_row & 7;
+        k_chunk_add = (lane >> 3) & 1;
+        v_row = (lane & 7) + 8 * ((lane >> 3) & 1);
+        v_rowoff = v_row * 128;
+        v_swz = v_row & 7;
+        v_chunk_add = lane >> 4;
+        t0 = 2 * (lane & 3);
     }
-    __syncwarp();
-    const uint32_t bar0 = smem_u32(&bars[0]);
-    const uint32_t ring0 = smem_u32(ring);
 
-    const int H_q = H_kv * G;
-    const int gid = lane >> 2, tid4 = lane & 3;          // fragment coordinates: head row / column pair
-    const bool head_ok = gid < G;
-    // Work unit = (pair, split): slots [pair*k_max + split*pages_per_split, +pages_per_split) of the
-    // flat slot space slot = pair*k_max + i (the host guarantees it fits 31 bits).  Units are dealt
-    // to warps so that warp w of every CTA is busy before warp w+1 of any CTA.
-    const int n_units = B * H_kv * max_splits;
-    const int gw = warp * gridDim.x + blockIdx.x;
-    const int warps_total = kDecWarps * gridDim.x;
-    int x_end = 0;                                   // end of the current unit's slot range
+    __device__ __forceinline__ void load_q(const uint16_t *__restrict__ q, size_t head0, int lane, int G) {
+        const int gid = lane >> 2, tid4 = lane & 3;
+        const bool head_ok = gid < G;
+        const uint16_t *src = q + (head0 + (head_ok ? gid : 0)) * D + 2 * tid4;
+#pragma unroll
+        for (int s = 0; s < C::KSTEPS; ++s) {
+            const uint32_t w0 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16));
+            const uint32_t w1 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16 + 8));
+            qa[s][0] = head_ok ? w0 : 0u;
+            qa[s][1] = head_ok ? w1 : 0u;
+        }
+    }
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int nt = 0; nt < C::NTILES; ++nt) {
+            o_acc[nt][0] = 0.f; o_acc[nt][1] = 0.f; o_acc[nt][2] = 0.f; o_acc[nt][3] = 0.f;
+        }
+        m_run = -INFINITY;
+        l_run = 0.f;
+    }
+    // Logits (base 2, scaled) of head gid for tokens 2*tid4, 2*tid4+1, 8+2*tid4, 9+2*tid4 of the page
+    // whose K tiles sit at Ks; tokens >= nv are masked to -inf.
+    __device__ __forceinline__ void logits(uint32_t Ks, int nv, float scale_log2, float (&z)[4]) const {
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        float s0b[4] = {0.f, 0.f, 0.f, 0.f}, s1b[4] = {0.f, 0.f, 0.f, 0.f};   // odd k-steps: shorter chains
+#pragma unroll
+        for (int s = 0; s < C::KSTEPS; ++s) {
+            const int hf = s >> 2;
+            const int chunk = 2 * (s & 3) + k_chunk_add;
+            uint32_t b00, b01, b10, b11;     // {tok 0-7: k lo, k hi}, {tok 8-15: k lo, k hi}
+            ldmatrix_x4(Ks + hf * kTileBytes + k_rowoff + ((chunk ^ k_swz) << 4), b00, b01, b10, b11);
+            if (s & 1) {
+                mma_bf16_16816(s0b, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                mma_bf16_16816(s1b, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+            } else {
+                mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
+                mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
+            }
+        }
+        s0[0] += s0b[0]; s0[1] += s0b[1]; s1[0] += s1b[0]; s1[1] += s1b[1];
+        z[0] = (t0 < nv) ? s0[0] * scale_log2 : -INFINITY;
+        z[1] = (t0 + 1 < nv) ? s0[1] * scale_log2 : -INFINITY;
+        z[2] = (t0 + 8 < nv) ? s1[0] * scale_log2 : -INFINITY;
+        z[3] = (t0 + 9 < nv) ? s1[1] * scale_log2 : -INFINITY;
+    }
+    // Online-softmax update with the page's logits and O += P . V for the V tiles at Vs.
+    __device__ __forceinline__ void accumulate(uint32_t Vs, int nv, const float (&z)[4], uint32_t zero_chunk) {
+        float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+        pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
+        pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
+        const float m_new = fmaxf(m_run, pmax);           // finite: token 0 of a page is always valid
+        const float corr = exp2f(m_run - m_new);          // 0 on the first page (m_run = -inf)
+        if (__any_sync(kFull, m_new != m_run)) {
+            l_run *= corr;
+#pragma unroll
+            for (int nt = 0; nt < C::NTILES; ++nt) {
+                o_acc[nt][0] *= corr;
+                o_acc[nt][1] *= corr;
+                o_acc[nt][2] *= corr;
+                o_acc[nt][3] *= corr;
+            }
+            m_run = m_new;
+        }
+        float p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = exp2f(z[e] - m_run);    // exp2(-inf) = 0 for masked tokens
+        l_run += (p[0] + p[1]) + (p[2] + p[3]);
+        // P as the A operand, split into two bf16 terms so that p_hi + p_lo carries 16 bits.  The
+        // group has at most 8 heads, so rows 8-15 of the m16 tile are free: p_hi goes into rows
+        // 0-7 and p_lo into rows 8-15, and one MMA yields both products (accumulator elements
+        // 0,1 and 2,3 of this lane); they are added in finish().
+        const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
+        const float2 f0 = bf16x2_to_f2(ph0), f1 = bf16x2_to_f2(ph1);
+        const uint32_t pl0 = pack_bf16(p[0] - f0.x, p[1] - f0.y), pl1 = pack_bf16(p[2] - f1.x, p[3] - f1.y);
+#pragma unroll
+        for (int c2 = 0; c2 < C::NTILES / 2; ++c2) {
+            const int hf = c2 >> 2;
+            const int chunk = 2 * (c2 & 3) + v_chunk_add;
+            uint32_t v00, v01, v10, v11;     // {chunk c: tok 0-7, tok 8-15}, {chunk c+1: ...}
+            // token rows past the request's length may hold anything (NaN included) and their
+            // weights are zero: their lanes read a zeroed chunk instead
+            const uint32_t va = Vs + hf * kTileBytes + v_rowoff + ((chunk ^ v_swz) << 4);
+            ldmatrix_x4_trans(v_row < nv ? va : zero_chunk, v00, v01, v10, v11);
+            mma_bf16_16816(o_acc[2 * c2], ph0, pl0, ph1, pl1, v00, v01);
+            mma_bf16_16816(o_acc[2 * c2 + 1], ph0, pl0, ph1, pl1, v10, v11);
+        }
+    }
+    // The four lanes of a head hold disjoint token columns: fold their l; add the p_hi and p_lo products.
+    __device__ __forceinline__ void finish() {
+        l_run += __shfl_xor_sync(kFull, l_run, 1);
+        l_run += __shfl_xor_sync(kFull, l_run, 2);
+#pragma unroll
+        for (int nt = 0; nt < C::NTILES; ++nt) {
+            o_acc[nt][0] += o_acc[nt][2];
+            o_acc[nt][1] += o_acc[nt][3];
+        }
+    }
+};
 
-    // ldmatrix lane offsets inside a 16x128-byte swizzled tile.
-    // K (B operand, not transposed): matrices {tok 0-7 | 8-15} x {chunk c | c+1}
-    const int k_row = (lane & 7) + 8 * (lane >> 4);
-    const int k_chunk_add = (lane >> 3) & 1;
-    // V (B operand, transposed): matrices {tok 0-7 | 8-15} fastest, then {chunk c | c+1}
-    const int v_row = (lane & 7) + 8 * ((lane >> 3) & 1);
-    const int v_chunk_add = lane >> 4;
-    uint32_t phases = 0;          // parity bit per stage
-    int stage_c = 0, stage_i = 0; // next stage to consume / to fill
-    bool failed = false;
+// ---------------------------------------------------------------------------------
+// Per-warp copy pipeline: a ring of `nstage` stages (one stage = K page + V page of one head), one
+// mbarrier per stage, and the list of the pages of the current chunk of selection entries.
+// ---------------------------------------------------------------------------------
+struct WarpPipe {
+    uint32_t ring0, bar0;    // shared-memory addresses of the warp's first stage / first barrier
+    int nstage;
+    uint32_t phases;         // parity bit per stage
+    int stage_c, stage_i;    // next stage to consume / to fill
+    int *ent_y;              // row of the page's first token in the [pages*heads*16, D] view of the cache
+    int *ent_info;           // valid tokens (bits 0-4) | selection index i (bits 5..)
+    int *ent_b;              // logical page (only read by an observation layer)
+};
 
-    // ---- page list.  The valid selected pages of a chunk of up to kChunk slots are looked up
-    // at once (selection -> page table, two dependent loads for the whole chunk) and kept in
-    // shared memory; the copy pipeline then runs over that list without any further global
-    // look-ups, across pair boundaries.
-    //   ent_y    row of the page's first token in the [pages*heads*16, D] view of the cache
-    //   ent_info valid tokens (bits 0-4) | selection index i (bits 5-16) | slot - chunk_base (bits 17-23)
-    //   ent_b    logical page (only read by an observation layer)
-    int *ent_y = reinterpret_cast<int *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8) +
-                 warp * 3 * kChunk;
-    int *ent_info = ent_y + kChunk;
-    int *ent_b = ent_info + kChunk;
-    // 16 zero bytes per CTA (behind the page lists)
-    const uint32_t zero_chunk = smem_u32(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8 +
-                                         (size_t)kDecWarps * 3 * kChunk * sizeof(int));
-    if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8 +
-                                                     (size_t)kDecWarps * 3 * kChunk * sizeof(int))[threadIdx.x] = 0u;
-    __syncthreads();
-    int chunk_base = 0, chunk_end = 0;           // slots [chunk_base, chunk_end) are in the list
+struct AttendArgs {
+    const CUtensorMap *k_map, *v_map;
+    const int32_t *page_table;
+    int max_pages, H_kv, P_phys, G, GP;
+    float *zrow;             // H2O: logits of this pair, [k_max][16][GP] (nullptr = off)
+    uint32_t *keys_row;      // observation layer: token keys of this request (nullptr = off)
+    float scale_log2;
+    uint32_t zero_chunk;
+    uint32_t *status;
+};
+
+// Attends the selection entries [i_lo, i_hi) of one (request r, kv-head hh) pair; sel_at(i) is the
+// logical page of entry i.  The valid pages of up to kChunk entries are looked up at once (selection
+// -> page table, two dependent loads for the whole chunk) and kept in shared memory; the copy
+// pipeline then runs over that list without further global look-ups.  Returns false when a bounded
+// wait gave up.  `first` (when kFirst) holds the entries i_lo + rep*32 + lane of the first chunk, loaded by
+// the caller ahead of time so that they travel together with the lengths instead of after them.
+template <int D, bool kObserve, bool kFirst, typename SelAt>
+__device__ __forceinline__ bool attend_range(WarpPipe &P, WarpAttn<D> &A, const AttendArgs &a, SelAt sel_at,
+                                             const int (&first)[kChunk / 32], int i_lo, int i_hi, int r, int hh, int len,
+                                             int n_r, int lane) {
+    using C = DecCfg<D>;
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const float scale_log2 = a.scale_log2;
+    const uint32_t zero_chunk = a.zero_chunk;
+    float *const zrow = a.zrow;
+    const int GP = a.GP;
+    const bool head_ok = gid < a.G;
+    int chunk_end = i_lo;
     int n_ent = 0, ce = 0, pe = 0;               // entries, next to consume, next to issue
 
     auto fill_chunk = [&](int base) {
-        chunk_base = base;
-        chunk_end = min(x_end, base + kChunk);
-        const int pair0 = base / k_max;
-        const int i0 = base - pair0 * k_max;
+        const int end = min(i_hi, base + kChunk);
         int sl_pid[kChunk / 32], sl_meta[kChunk / 32], sl_b[kObserve ? kChunk / 32 : 1];
 #pragma unroll
         for (int rep = 0; rep < kChunk / 32; ++rep) {
-            const int off = rep * 32 + lane;
+            const int i = base + rep * 32 + lane;
             int pid = -1, meta = 0, lb = 0;
-            if (base + off < chunk_end) {
-                const int dp = (i0 + off) / k_max;
-                const int pair = pair0 + dp;
-                const int i = i0 + off - dp * k_max;
-                const int r = pair / H_kv;
-                const int hh = pair - r * H_kv;
-                const int b = __ldg(sel_idx + base + off);      // speculative: checked against cnt below
-                const int cnt = min(__ldg(sel_cnt + pair), k_max);
-                const int len = __ldg(seq_lens + r);
-                const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
-                if (i < cnt && n_r > 0) {
-                    if (b < 0 || b >= n_r) {
-                        atomicOr(status, SE_DEV_BAD_SELECTION);
-                    } else {
-                        pid = __ldg(page_table + (size_t)r * max_pages + b);
-                        lb = b;
-                        meta = min(kPage, len - b * kPage) | (i << 5) | (off << 17) | (hh << 24);
-                    }
+            if (i < end) {
+                const int b = (kFirst && base == i_lo) ? first[rep] : sel_at(i);
+                if (b < 0 || b >= n_r) {
+                    atomicOr(a.status, SE_DEV_BAD_SELECTION);
+                } else {
+                    pid = __ldg(a.page_table + (size_t)r * a.max_pages + b);
+                    lb = b;
+                    meta = min(kPage, len - b * kPage) | (i << 5);
                 }
             }
             sl_pid[rep] = pid;
@@ -175,22 +280,23 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
         for (int rep = 0; rep < kChunk / 32; ++rep) {
             int pid = sl_pid[rep];
             const bool looked_up = sl_meta[rep] != 0;
-            if (looked_up && pid >= P_phys) {
-                atomicOr(status, SE_DEV_BAD_PAGE_ID);
+            if (looked_up && pid >= a.P_phys) {
+                atomicOr(a.status, SE_DEV_BAD_PAGE_ID);
                 pid = -1;
             } else if (looked_up && pid < 0) {
-                atomicOr(status, SE_DEV_BAD_SELECTION);
+                atomicOr(a.status, SE_DEV_BAD_SELECTION);
             }
             const unsigned vm = __ballot_sync(kFull, pid >= 0);
             if (pid >= 0) {
                 const int pos = count + __popc(vm & ((1u << lane) - 1u));
-                ent_y[pos] = (pid * H_kv + (sl_meta[rep] >> 24)) * kPage;
-                ent_info[pos] = sl_meta[rep] & 0x00ffffff;
-                if (kObserve) ent_b[pos] = sl_b[rep];
+                P.ent_y[pos] = (pid * a.H_kv + hh) * kPage;
+                P.ent_info[pos] = sl_meta[rep];
+                if (kObserve) P.ent_b[pos] = sl_b[rep];
             }
             count += __popc(vm);
         }
         __syncwarp();
+        chunk_end = end;
         n_ent = count;
         ce = 0;
         pe = 0;
@@ -199,229 +305,464 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     // K page, lane 1 the V page; each arms the stage's barrier with its own byte count (the barrier
     // expects two arrivals, so the lanes need no ordering between themselves).
     auto top_up = [&]() {
-        while (pe < n_ent && pe < ce + nstage) {
+        while (pe < n_ent && pe < ce + P.nstage) {
             if (lane < 2) {
-                const uint32_t bar = bar0 + stage_i * 8;
-                const uint32_t dst = ring0 + stage_i * C::STAGEB + lane * C::PAGEB;
+                const uint32_t bar = P.bar0 + P.stage_i * 8;
+                const uint32_t dst = P.ring0 + P.stage_i * C::STAGEB + lane * C::PAGEB;
                 mbar_expect_tx(bar, C::PAGEB);
-                tma_load_page(dst, lane ? &v_map : &k_map, ent_y[pe], bar);
+                tma_load_page(dst, lane ? a.v_map : a.k_map, P.ent_y[pe], bar);
             }
-            stage_i = (stage_i + 1 == nstage) ? 0 : stage_i + 1;
+            P.stage_i = (P.stage_i + 1 == P.nstage) ? 0 : P.stage_i + 1;
             ++pe;
         }
     };
 
-    for (int unit = gw; unit < n_units && !failed; unit += warps_total) {
+    fill_chunk(i_lo);
+    top_up();
+    for (;;) {
+        if (ce == n_ent) {                       // list exhausted: more entries left?
+            if (chunk_end >= i_hi) break;
+            fill_chunk(chunk_end);
+            top_up();
+            continue;
+        }
+        const int info = P.ent_info[ce];
+        const int nv_j = info & 31;
+        const int i_j = info >> 5;
+        if (!mbar_wait(P.bar0 + P.stage_c * 8, (P.phases >> P.stage_c) & 1u)) return false;
+        P.phases ^= (1u << P.stage_c);
+        const uint32_t Ks = P.ring0 + P.stage_c * C::STAGEB;
+        const uint32_t Vs = Ks + C::PAGEB;
+        P.stage_c = (P.stage_c + 1 == P.nstage) ? 0 : P.stage_c + 1;
+
+        float z[4];
+        A.logits(Ks, nv_j, scale_log2, z);
+        const int t0 = 2 * tid4;
+        if (zrow != nullptr && head_ok) {
+            float *zp = zrow + ((size_t)i_j * kPage) * GP + gid;
+            zp[(t0) * GP] = z[0];
+            zp[(t0 + 1) * GP] = z[1];
+            zp[(t0 + 8) * GP] = z[2];
+            zp[(t0 + 9) * GP] = z[3];
+        }
+        if (kObserve) {
+            // observation layer: s(j) = max over every query head of the logit (Appendix A, OmniKV
+            // selection equation).  Here: max over the group's heads (rows gid; rows past the group
+            // hold zero queries and are left out), then an atomic max over the kv-heads on the
+            // order-preserving integer image of the score.
+            float m4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float v = head_ok ? z[e] : -INFINITY;
+                v = fmaxf(v, __shfl_xor_sync(kFull, v, 4));
+                v = fmaxf(v, __shfl_xor_sync(kFull, v, 8));
+                v = fmaxf(v, __shfl_xor_sync(kFull, v, 16));
+                m4[e] = v;
+            }
+            if (gid == 0) {
+                uint32_t *kp = a.keys_row + P.ent_b[ce] * kPage;
+                if (m4[0] > -INFINITY) atomicMax(kp + t0, f32_key(m4[0] * kLn2));
+                if (m4[1] > -INFINITY) atomicMax(kp + t0 + 1, f32_key(m4[1] * kLn2));
+                if (m4[2] > -INFINITY) atomicMax(kp + t0 + 8, f32_key(m4[2] * kLn2));
+                if (m4[3] > -INFINITY) atomicMax(kp + t0 + 9, f32_key(m4[3] * kLn2));
+            }
+        }
+        A.accumulate(Vs, nv_j, z, zero_chunk);
+        __syncwarp();     // all lanes are done with this stage before it is refilled
+        ++ce;
+        top_up();
+    }
+    return true;
+}
+
+// Where a unit's selection comes from: the list the caller passes (sel_idx / sel_cnt are read) or,
+// with kSelect, the page scores in the workspace (the top-k runs here and sel_idx / sel_cnt are written).
+struct SelectArgs {
+    int32_t *sel_idx;        // [pairs][k_max]
+    int32_t *sel_cnt;        // [pairs]
+    const float *scores;     // [pairs][pitch]
+    int pitch, k_pages, sink, recent;
+};
+
+// ---------------------------------------------------------------------------------
+// decode_kernel: persistent warps over (pair, split) units.
+// ---------------------------------------------------------------------------------
+template <int D, bool kObserve>
+__global__ void __launch_bounds__(kDecWarps * 32, 1)
+decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+              const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
+              const int32_t *__restrict__ seq_lens, const SelectArgs sa, float *__restrict__ out,
+              float *__restrict__ lse, float *__restrict__ partials, float *__restrict__ zbuf,
+              uint32_t *__restrict__ tok_keys, int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max,
+              int pages_per_split, int max_splits, float scale_log2, uint32_t *status) {
+    using C = DecCfg<D>;
+    extern __shared__ uint8_t smem_dyn[];
+    // tiles must sit on 1024-byte boundaries for the 128-byte swizzle pattern
+    uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // The CTA's stages are shared out among the warps that have work: warp w of this CTA is busy iff
+    // its first unit w*gridDim.x + blockIdx.x exists, so the busy warps are the lowest ones.  Every
+    // busy warp of the GRID gets the same number of stages - that of the fullest CTAs - so that the
+    // bytes a CTA keeps in flight, and with them its share of the memory bandwidth, follow its
+    // number of units: a CTA with three units and deeper pipelines would finish well before the CTAs
+    // with four, which then decide the kernel's time at less than full bandwidth.
+    int busy = (B * H_kv * max_splits - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    busy = busy < 1 ? 1 : (busy > kDecWarps ? kDecWarps : busy);
+    int busy_max = (B * H_kv * max_splits + (int)gridDim.x - 1) / (int)gridDim.x;
+    busy_max = busy_max > kDecWarps ? kDecWarps : busy_max;
+    WarpPipe P;
+    P.nstage = warp < busy ? min(C::MAXST, C::CTA_STAGES / busy_max) : 0;
+    uint8_t *ring = smem_al + (size_t)(warp * P.nstage) * C::STAGEB;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)C::CTA_STAGES * C::STAGEB) + warp * C::MAXST;
+    if (lane == 0) {
+        for (int s = 0; s < P.nstage; ++s) mbar_init(smem_u32(&bars[s]), 2);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    P.bar0 = smem_u32(&bars[0]);
+    P.ring0 = smem_u32(ring);
+    P.phases = 0;
+    P.stage_c = 0;
+    P.stage_i = 0;
+    uint8_t *lists = smem_al + (size_t)C::CTA_STAGES * C::STAGEB + kDecWarps * C::MAXST * 8;
+    P.ent_y = reinterpret_cast<int *>(lists) + warp * 3 * kChunk;
+    P.ent_info = P.ent_y + kChunk;
+    P.ent_b = P.ent_info + kChunk;
+    // 16 zero bytes per CTA (behind the page lists)
+    uint8_t *zero_bytes = lists + (size_t)kDecWarps * 3 * kChunk * sizeof(int);
+    if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(zero_bytes)[threadIdx.x] = 0u;
+    __syncthreads();
+
+    AttendArgs a;
+    a.k_map = &k_map;
+    a.v_map = &v_map;
+    a.page_table = page_table;
+    a.max_pages = max_pages;
+    a.H_kv = H_kv;
+    a.P_phys = P_phys;
+    a.G = G;
+    a.GP = GP;
+    a.scale_log2 = scale_log2;
+    a.zero_chunk = smem_u32(zero_bytes);
+    a.status = status;
+
+    const int H_q = H_kv * G;
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const bool head_ok = gid < G;
+    // Work unit = (pair, split): selection entries [split*pages_per_split, +pages_per_split) of the pair.
+    // Units are dealt to warps so that warp w of every CTA is busy before warp w+1 of any CTA.
+    const int n_units = B * H_kv * max_splits;
+    const int warps_total = kDecWarps * gridDim.x;
+    bool failed = false;
+    WarpAttn<D> A;
+    A.init_lane(lane);
+
+    for (int unit = warp * gridDim.x + blockIdx.x; unit < n_units && !failed; unit += warps_total) {
         const int pair = unit / max_splits;
         const int my_split = unit - pair * max_splits;
         const int i_lo = my_split * pages_per_split;
         if (i_lo >= k_max) continue;
         const int r = pair / H_kv, h = pair % H_kv;
-        const int seg_begin = pair * k_max + i_lo;
-
-        // ---- Q as the A operand: row gid = query head gid of the group (rows >= G and 8..15 are
-        // zero).  Issued first: these loads depend on nothing and overlap the look-ups below.
-        uint32_t qa[C::KSTEPS][2];
-        {
-            const uint16_t *src = q + ((size_t)r * H_q + h * G + (head_ok ? gid : 0)) * D + 2 * tid4;
+        const size_t head0 = (size_t)r * H_q + h * G;
+        int32_t *sel_row = sa.sel_idx + (size_t)pair * k_max;
+        // Loads that depend on nothing go out first and travel together: the lengths, the selection
+        // count, Q, and (when the caller supplies the list) the first chunk of selection entries.
+        int first[kChunk / 32];
+        A.load_q(q, head0, lane, G);
 #pragma unroll
-            for (int s = 0; s < C::KSTEPS; ++s) {
-                const uint32_t w0 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16));
-                const uint32_t w1 = __ldg(reinterpret_cast<const uint32_t *>(src + s * 16 + 8));
-                qa[s][0] = head_ok ? w0 : 0u;
-                qa[s][1] = head_ok ? w1 : 0u;
-            }
+        for (int rep = 0; rep < kChunk / 32; ++rep) {
+            const int i = i_lo + rep * 32 + lane;
+            first[rep] = i < min(i_lo + pages_per_split, k_max) ? __ldg(sel_row + i) : -1;
         }
-        // ---- page list of the unit's slot range: selection entries, selection count and length
-        // travel together (one round trip), the page-table entries follow (a second one)
-        x_end = pair * k_max + min(i_lo + pages_per_split, k_max);
-        fill_chunk(seg_begin);
-        int cnt = __ldg(sel_cnt + pair);          // same words the look-up just fetched: cache hits
+        const int len = __ldg(seq_lens + r);
+        const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
+        int cnt = __ldg(sa.sel_cnt + pair);
         if (cnt > k_max) {
             if (lane == 0) atomicOr(status, SE_DEV_BAD_SELECTION);
             cnt = k_max;
         }
-        const int len = __ldg(seq_lens + r);
-        const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
         if (cnt <= 0 || n_r == 0) {
             if (my_split == 0) {      // the first split of the pair reports "nothing attended"
                 for (int g = 0; g < G; ++g) {
-                    float *o = out + ((size_t)r * H_q + h * G + g) * D;
+                    float *o = out + (head0 + g) * D;
                     for (int c = lane; c < D; c += 32) o[c] = 0.f;
-                    if (lane == 0) lse[(size_t)r * H_q + h * G + g] = -INFINITY;
+                    if (lane == 0) lse[head0 + g] = -INFINITY;
                 }
             }
             continue;
         }
         if (i_lo >= cnt) continue;
         const int i_hi = min(min(i_lo + pages_per_split, k_max), cnt);
-        const int seg_end = pair * k_max + i_hi;                      // first slot past this unit
         const int n_split = (cnt + pages_per_split - 1) / pages_per_split;   // splits of this pair that hold pages
-        top_up();
 
-        float o_acc[C::NTILES][4];
-#pragma unroll
-        for (int nt = 0; nt < C::NTILES; ++nt) {
-            o_acc[nt][0] = 0.f; o_acc[nt][1] = 0.f; o_acc[nt][2] = 0.f; o_acc[nt][3] = 0.f;
+        A.reset();
+        a.zrow = zbuf != nullptr ? zbuf + (size_t)pair * k_max * kPage * GP : nullptr;
+        a.keys_row = kObserve ? tok_keys + (size_t)r * max_pages * kPage : nullptr;
+        auto sel_at = [&](int i) { return __ldg(sel_row + i); };
+        if (!attend_range<D, kObserve, true>(P, A, a, sel_at, first, i_lo, i_hi, r, h, len, n_r, lane)) {
+            failed = true;
+            break;
         }
-        float m_run = -INFINITY, l_run = 0.f;       // of head gid; l is this lane's share (its 4 token columns)
-        while (!failed) {
-            if (ce == n_ent) {                       // list exhausted: more slots of this segment left?
-                if (chunk_end >= seg_end) break;
-                fill_chunk(chunk_end);
-                top_up();
-                continue;
-            }
-            const int info = ent_info[ce];
-            if (chunk_base + (info >> 17) >= seg_end) break;    // next entry belongs to the next pair
-            const int nv_j = info & 31;
-            const int i_j = (info >> 5) & 4095;
-            if (!mbar_wait(bar0 + stage_c * 8, (phases >> stage_c) & 1u)) {
-                failed = true;
-                break;
-            }
-            phases ^= (1u << stage_c);
-            const uint32_t Ks = ring0 + stage_c * C::STAGEB;
-            const uint32_t Vs = Ks + C::PAGEB;
-            stage_c = (stage_c + 1 == nstage) ? 0 : stage_c + 1;
-
-            // ---- S^T[head, token] = Q . K^T : two n8 tiles (tokens 0-7, 8-15)
-            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-            float s0b[4] = {0.f, 0.f, 0.f, 0.f}, s1b[4] = {0.f, 0.f, 0.f, 0.f};   // odd k-steps: shorter chains
-#pragma unroll
-            for (int s = 0; s < C::KSTEPS; ++s) {
-                const int hf = s >> 2;
-                const int chunk = 2 * (s & 3) + k_chunk_add;
-                uint32_t b00, b01, b10, b11;     // {tok 0-7: k lo, k hi}, {tok 8-15: k lo, k hi}
-                ldmatrix_x4(Ks + hf * kTileBytes + k_row * 128 + ((chunk ^ (k_row & 7)) << 4), b00, b01, b10, b11);
-                if (s & 1) {
-                    mma_bf16_16816(s0b, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
-                    mma_bf16_16816(s1b, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
-                } else {
-                    mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, b00, b01);
-                    mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, b10, b11);
-                }
-            }
-            s0[0] += s0b[0]; s0[1] += s0b[1]; s1[0] += s1b[0]; s1[1] += s1b[1];
-            // this lane: head gid, tokens 2*tid4, 2*tid4+1 (s0) and 8+2*tid4, 9+2*tid4 (s1)
-            const int t0 = 2 * tid4;
-            float z[4];
-            z[0] = (t0 < nv_j) ? s0[0] * scale_log2 : -INFINITY;
-            z[1] = (t0 + 1 < nv_j) ? s0[1] * scale_log2 : -INFINITY;
-            z[2] = (t0 + 8 < nv_j) ? s1[0] * scale_log2 : -INFINITY;
-            z[3] = (t0 + 9 < nv_j) ? s1[1] * scale_log2 : -INFINITY;
-            if (zbuf != nullptr && head_ok) {
-                float *zp = zbuf + (((size_t)pair * k_max + i_j) * kPage) * GP + gid;
-                zp[(t0) * GP] = z[0];
-                zp[(t0 + 1) * GP] = z[1];
-                zp[(t0 + 8) * GP] = z[2];
-                zp[(t0 + 9) * GP] = z[3];
-            }
-            if (kObserve) {
-                // observation layer: s(j) = max over every query head of the logit (Appendix A, OmniKV
-                // selection equation).  Here: max over the group's heads (rows gid), then an atomic
-                // max over the kv-heads on the order-preserving integer image of the score.
-                float m4[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = head_ok ? z[e] : -INFINITY;
-                    v = fmaxf(v, __shfl_xor_sync(kFull, v, 4));
-                    v = fmaxf(v, __shfl_xor_sync(kFull, v, 8));
-                    v = fmaxf(v, __shfl_xor_sync(kFull, v, 16));
-                    m4[e] = v;
-                }
-                if (gid == 0) {
-                    uint32_t *kp = tok_keys + (size_t)r * max_pages * kPage + ent_b[ce] * kPage;
-                    if (m4[0] > -INFINITY) atomicMax(kp + t0, f32_key(m4[0] * kLn2));
-                    if (m4[1] > -INFINITY) atomicMax(kp + t0 + 1, f32_key(m4[1] * kLn2));
-                    if (m4[2] > -INFINITY) atomicMax(kp + t0 + 8, f32_key(m4[2] * kLn2));
-                    if (m4[3] > -INFINITY) atomicMax(kp + t0 + 9, f32_key(m4[3] * kLn2));
-                }
-            }
-            float pmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
-            pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 1));
-            pmax = fmaxf(pmax, __shfl_xor_sync(kFull, pmax, 2));
-            const float m_new = fmaxf(m_run, pmax);           // finite: token 0 of a page is always valid
-            const float corr = exp2f(m_run - m_new);          // 0 on the first page (m_run = -inf)
-            if (__any_sync(kFull, m_new != m_run)) {
-                l_run *= corr;
-#pragma unroll
-                for (int nt = 0; nt < C::NTILES; ++nt) {
-                    o_acc[nt][0] *= corr;
-                    o_acc[nt][1] *= corr;
-                    o_acc[nt][2] *= corr;
-                    o_acc[nt][3] *= corr;
-                }
-                m_run = m_new;
-            }
-            float p[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) p[e] = exp2f(z[e] - m_run);    // exp2(-inf) = 0 for masked tokens
-            l_run += (p[0] + p[1]) + (p[2] + p[3]);
-            // P as the A operand, split into two bf16 terms so that p_hi + p_lo carries 16 bits.  The
-            // group has at most 8 heads, so rows 8-15 of the m16 tile are free: p_hi goes into rows
-            // 0-7 and p_lo into rows 8-15, and one MMA yields both products (accumulator elements
-            // 0,1 and 2,3 of this lane); they are added when the unit ends.
-            const uint32_t ph0 = pack_bf16(p[0], p[1]), ph1 = pack_bf16(p[2], p[3]);
-            const float2 f0 = bf16x2_to_f2(ph0), f1 = bf16x2_to_f2(ph1);
-            const uint32_t pl0 = pack_bf16(p[0] - f0.x, p[1] - f0.y), pl1 = pack_bf16(p[2] - f1.x, p[3] - f1.y);
-
-            // ---- O[head, :] += P . V : n8 tiles over the channels, k16 = the 16 tokens
-#pragma unroll
-            for (int c2 = 0; c2 < C::NTILES / 2; ++c2) {
-                const int hf = c2 >> 2;
-                const int chunk = 2 * (c2 & 3) + v_chunk_add;
-                uint32_t v00, v01, v10, v11;     // {chunk c: tok 0-7, tok 8-15}, {chunk c+1: ...}
-                // token rows past the request's length may hold anything (NaN included) and their
-                // weights are zero: their lanes read a zeroed chunk instead
-                const uint32_t va = Vs + hf * kTileBytes + v_row * 128 + ((chunk ^ (v_row & 7)) << 4);
-                ldmatrix_x4_trans(v_row < nv_j ? va : zero_chunk, v00, v01, v10, v11);
-                mma_bf16_16816(o_acc[2 * c2], ph0, pl0, ph1, pl1, v00, v01);
-                mma_bf16_16816(o_acc[2 * c2 + 1], ph0, pl0, ph1, pl1, v10, v11);
-            }
-            __syncwarp();     // all lanes are done with this stage before it is refilled
-            ++ce;
-            top_up();
-        }
-        if (failed) break;
-        // ---- the four lanes of a head hold disjoint token columns: fold their l
-        l_run += __shfl_xor_sync(kFull, l_run, 1);
-        l_run += __shfl_xor_sync(kFull, l_run, 2);
-#pragma unroll
-        for (int nt = 0; nt < C::NTILES; ++nt) {        // p_hi and p_lo products
-            o_acc[nt][0] += o_acc[nt][2];
-            o_acc[nt][1] += o_acc[nt][3];
-        }
+        A.finish();
 
         if (n_split == 1) {
             if (head_ok) {
-                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                float *o = out + ((size_t)r * H_q + h * G + gid) * D + 2 * tid4;
+                const float inv = A.l_run > 0.f ? 1.f / A.l_run : 0.f;
+                float *o = out + (head0 + gid) * D + 2 * tid4;
 #pragma unroll
                 for (int nt = 0; nt < C::NTILES; ++nt)
-                    *reinterpret_cast<float2 *>(o + nt * 8) = make_float2(o_acc[nt][0] * inv, o_acc[nt][1] * inv);
-                if (tid4 == 0)
-                    lse[(size_t)r * H_q + h * G + gid] = l_run > 0.f ? (m_run + log2f(l_run)) * kLn2 : -INFINITY;
+                    *reinterpret_cast<float2 *>(o + nt * 8) = make_float2(A.o_acc[nt][0] * inv, A.o_acc[nt][1] * inv);
+                if (tid4 == 0) lse[head0 + gid] = A.l_run > 0.f ? (A.m_run + log2f(A.l_run)) * kLn2 : -INFINITY;
             }
             continue;
         }
-
         // ---- store the partial; combine_kernel merges the splits of a pair afterwards
         if (head_ok) {
-            float *pr = partials + (((size_t)r * H_q + h * G + gid) * max_splits + my_split) * C::PSTRIDE;
+            float *pr = partials + ((head0 + gid) * max_splits + my_split) * C::PSTRIDE;
 #pragma unroll
             for (int nt = 0; nt < C::NTILES; ++nt)
-                *reinterpret_cast<float2 *>(pr + nt * 8 + 2 * tid4) = make_float2(o_acc[nt][0], o_acc[nt][1]);
+                *reinterpret_cast<float2 *>(pr + nt * 8 + 2 * tid4) = make_float2(A.o_acc[nt][0], A.o_acc[nt][1]);
             if (tid4 == 0) {
-                pr[D] = m_run;
-                pr[D + 1] = l_run;
+                pr[D] = A.m_run;
+                pr[D + 1] = A.l_run;
             }
         }
     }
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // bounded wait for whatever this warp still has in flight before the CTA can retire
-        for (int s = 0; s < nstage; ++s) mbar_wait(bar0 + s * 8, (phases >> s) & 1u);
+        for (int s = 0; s < P.nstage; ++s) mbar_wait(P.bar0 + s * 8, (P.phases >> s) & 1u);
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// decode_cta_kernel: one CTA per (pair, CTA-split); gridDim.x = pairs * cpp.
+//   1. selection list of the pair in shared memory: the caller's, or (kSelect) the CTA's own top-k of
+//      the score row (every CTA of a pair computes the same list; CTA-split 0 writes it out);
+//   2. the cnt selected pages are cut into n_active = ceil(cnt / ceil(cnt / cpp)) equal CTA slices, a
+//      slice into eight warp ranges; each warp attends its range (attend_range);
+//   3. the warps' partials are merged through shared memory (weights 2^(m_w - m*));
+//   4. one active CTA: out / lse are final.  Several: the CTA stores its partial and takes a ticket
+//      (atomic counter per pair, zero between launches); with merge_here the CTA holding the last
+//      ticket merges all of them, otherwise combine_kernel does.
+// ---------------------------------------------------------------------------------
+template <int D>
+struct CtaCfg {
+    using C = DecCfg<D>;
+    static constexpr int STAGES_PER_WARP = C::CTA_STAGES_SPLIT / kDecWarps;
+    static constexpr int RED_PITCH = D + 8;                    // floats per (warp, head) row of the merge buffer
+    static constexpr size_t kStages = (size_t)C::CTA_STAGES_SPLIT * C::STAGEB;
+    static constexpr size_t kBars = kStages;
+    static constexpr size_t kLists = kBars + (size_t)kDecWarps * C::MAXST * 8;
+    static constexpr size_t kZero = kLists + (size_t)kDecWarps * 3 * kChunk * sizeof(int);
+    static constexpr size_t kSmall = kZero + 16;               // merge statistics: 4 * 64 floats + flags
+    static constexpr size_t kSel = kSmall + 4 * 64 * sizeof(float) + 64;
+    static_assert(sizeof(TopkScratch) + cta_topk_key_words(8192, kDecWarps * 32) * 4 <= kStages,
+                  "the top-k keys and scratch live in the empty ring");
+    static_assert((size_t)kDecWarps * 8 * RED_PITCH * sizeof(float) <= kStages, "merge buffer lives in the drained ring");
+    static size_t smem_bytes(int k_max) { return kSel + (size_t)k_max * sizeof(int) + 1024; }
+};
+
+template <int D, bool kSelect>
+__global__ void __launch_bounds__(kDecWarps * 32, 1)
+decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+                  const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
+                  const int32_t *__restrict__ seq_lens, const SelectArgs sa, float *__restrict__ out,
+                  float *__restrict__ lse, float *partials, float *__restrict__ zbuf, int H_kv, int G, int GP,
+                  int max_pages, int P_phys, int k_max, int cpp, int merge_here, float scale_log2, uint32_t *status,
+                  uint32_t *ticket) {
+    using C = DecCfg<D>;
+    using L = CtaCfg<D>;
+    extern __shared__ uint8_t smem_dyn[];
+    uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const int pair = blockIdx.x / cpp, cs = blockIdx.x - pair * cpp;
+    const int r = pair / H_kv, h = pair - r * H_kv;
+    const int H_q = H_kv * G;
+    const size_t head0 = (size_t)r * H_q + h * G;
+
+    WarpPipe P;
+    P.nstage = L::STAGES_PER_WARP;
+    uint8_t *ring = smem_al + (size_t)(warp * L::STAGES_PER_WARP) * C::STAGEB;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + L::kBars) + warp * C::MAXST;
+    if (lane == 0) {
+        for (int s = 0; s < P.nstage; ++s) mbar_init(smem_u32(&bars[s]), 2);
+        mbar_fence_init();
+    }
+    P.bar0 = smem_u32(&bars[0]);
+    P.ring0 = smem_u32(ring);
+    P.phases = 0;
+    P.stage_c = 0;
+    P.stage_i = 0;
+    P.ent_y = reinterpret_cast<int *>(smem_al + L::kLists) + warp * 3 * kChunk;
+    P.ent_info = P.ent_y + kChunk;
+    P.ent_b = P.ent_info + kChunk;
+    if (tid < 4) reinterpret_cast<uint32_t *>(smem_al + L::kZero)[tid] = 0u;
+    float *s_m = reinterpret_cast<float *>(smem_al + L::kSmall);      // [warp][head]
+    float *s_l = s_m + 64;                                            // [warp][head]
+    float *s_M = s_l + 64;                                            // [head] merged maximum
+    float *s_L = s_M + 64;                                            // [head] merged sum
+    int *s_flag = reinterpret_cast<int *>(s_L + 64);
+    int *list = reinterpret_cast<int *>(smem_al + L::kSel);
+
+    const int len = __ldg(seq_lens + r);
+    const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
+    int32_t *sel_row = sa.sel_idx + (size_t)pair * k_max;
+    int cnt;
+    if (kSelect) {
+        TopkScratch &S = *reinterpret_cast<TopkScratch *>(smem_al);
+        uint32_t *keys = reinterpret_cast<uint32_t *>(smem_al + ((sizeof(TopkScratch) + 15) & ~(size_t)15));
+        cnt = cta_topk<kDecWarps * 32>(sa.scores + (size_t)pair * sa.pitch, n_r, sa.k_pages, k_max, sa.sink, sa.recent,
+                                       keys, S, list, cs == 0 ? sel_row : nullptr);
+        if (cs == 0 && tid == 0) sa.sel_cnt[pair] = cnt;
+        fence_proxy_async();          // the scratch was written with ordinary stores; tensor copies refill it
+    } else {
+        cnt = __ldg(sa.sel_cnt + pair);
+        if (cnt > k_max) {
+            if (tid == 0) atomicOr(status, SE_DEV_BAD_SELECTION);
+            cnt = k_max;
+        }
+        for (int i = tid; i < cnt; i += kDecWarps * 32) list[i] = __ldg(sel_row + i);
+    }
+    __syncthreads();
+    if (cnt <= 0 || n_r == 0) {
+        if (cs == 0) {
+            for (int e = tid; e < G * D; e += kDecWarps * 32) out[head0 * D + e] = 0.f;
+            if (tid < G) lse[head0 + tid] = -INFINITY;
+        }
+        return;
+    }
+    const int per_cta = (cnt + cpp - 1) / cpp;
+    const int n_active = (cnt + per_cta - 1) / per_cta;
+    if (cs >= n_active) return;
+    const int c_lo = cs * per_cta, c_hi = min(cnt, c_lo + per_cta);
+    const int per_warp = (c_hi - c_lo + kDecWarps - 1) / kDecWarps;
+    const int i_lo = min(c_hi, c_lo + warp * per_warp), i_hi = min(c_hi, i_lo + per_warp);
+
+    AttendArgs a;
+    a.k_map = &k_map;
+    a.v_map = &v_map;
+    a.page_table = page_table;
+    a.max_pages = max_pages;
+    a.H_kv = H_kv;
+    a.P_phys = P_phys;
+    a.G = G;
+    a.GP = GP;
+    a.scale_log2 = scale_log2;
+    a.zero_chunk = smem_u32(smem_al + L::kZero);
+    a.status = status;
+    a.zrow = zbuf != nullptr ? zbuf + (size_t)pair * k_max * kPage * GP : nullptr;
+    a.keys_row = nullptr;
+
+    WarpAttn<D> A;
+    A.init_lane(lane);
+    A.reset();
+    bool ok = true;
+    if (i_lo < i_hi) {
+        A.load_q(q, head0, lane, G);
+        const int none[kChunk / 32] = {};
+        ok = attend_range<D, false, false>(P, A, a, [&](int i) { return list[i]; }, none, i_lo, i_hi, r, h, len, n_r,
+                                           lane);
+    }
+    if (!ok) {
+        if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
+        for (int s = 0; s < P.nstage; ++s) mbar_wait(P.bar0 + s * 8, (P.phases >> s) & 1u);
+    }
+    A.finish();
+
+    // ---- merge of the eight warps through shared memory.  Rows past the group hold zero queries:
+    // finite values that nobody reads.
+    if (tid4 == 0) {
+        s_m[warp * 8 + gid] = A.m_run;
+        s_l[warp * 8 + gid] = A.l_run;
+    }
+    __syncthreads();                  // every warp has drained its ring: it becomes the merge buffer
+    float mstar = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) mstar = fmaxf(mstar, s_m[w * 8 + gid]);
+    float lsum = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+        const float mw = s_m[w * 8 + gid];
+        lsum += (mw == -INFINITY) ? 0.f : exp2f(mw - mstar) * s_l[w * 8 + gid];
+    }
+    const float wgt = (A.m_run == -INFINITY) ? 0.f : exp2f(A.m_run - mstar);
+    float *red = reinterpret_cast<float *>(smem_al);
+    {
+        float *dst = red + (size_t)(warp * 8 + gid) * L::RED_PITCH + 2 * tid4;
+#pragma unroll
+        for (int nt = 0; nt < C::NTILES; ++nt)
+            *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(A.o_acc[nt][0] * wgt, A.o_acc[nt][1] * wgt);
+    }
+    if (warp == 0 && tid4 == 0) {
+        s_M[gid] = mstar;
+        s_L[gid] = lsum;
+    }
+    __syncthreads();
+    const bool single = n_active == 1;
+    for (int e = tid; e < G * D; e += kDecWarps * 32) {
+        const int g = e / D, c = e - g * D;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecWarps; ++w) acc += red[(size_t)(w * 8 + g) * L::RED_PITCH + c];
+        if (single) {
+            const float lg = s_L[g];
+            out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
+        } else {
+            partials[((head0 + g) * cpp + cs) * C::PSTRIDE + c] = acc;
+        }
+    }
+    if (tid < G) {
+        const float lg = s_L[tid], mg = s_M[tid];
+        if (single) {
+            lse[head0 + tid] = lg > 0.f ? (mg + log2f(lg)) * kLn2 : -INFINITY;
+        } else {
+            float *pr = partials + ((head0 + tid) * cpp + cs) * C::PSTRIDE;
+            pr[D] = mg;
+            pr[D + 1] = lg;
+        }
+    }
+    if (single || !merge_here) return;
+
+    // ---- several CTAs share the pair: the one holding the last ticket merges their partials
+    __threadfence();                  // this CTA's partial, before its ticket
+    __syncthreads();
+    if (tid == 0) {
+        const uint32_t t = atomicAdd(ticket + pair, 1u);
+        const int last = t == (uint32_t)n_active - 1u;
+        if (last) ticket[pair] = 0u;  // every other CTA has drawn already: left at zero for the next launch
+        *s_flag = last;
+    }
+    __syncthreads();
+    if (!*s_flag) return;
+    __threadfence();                  // the other CTAs' partials are visible from here on
+    for (int e = tid; e < G * D; e += kDecWarps * 32) {
+        const int g = e / D, c = e - g * D;
+        const float *pr = partials + ((head0 + g) * cpp) * C::PSTRIDE;
+        float ms[kMergeInKernelMax], accs[kMergeInKernelMax];
+        float mg = -INFINITY;
+#pragma unroll
+        for (int s = 0; s < kMergeInKernelMax; ++s) {
+            ms[s] = -INFINITY;
+            accs[s] = 0.f;
+            if (s < n_active) {
+                ms[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
+                accs[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + c);
+            }
+            mg = fmaxf(mg, ms[s]);
+        }
+        float acc = 0.f, lg = 0.f;
+#pragma unroll
+        for (int s = 0; s < kMergeInKernelMax; ++s) {
+            if (s < n_active && ms[s] != -INFINITY) {
+                const float ws = exp2f(ms[s] - mg);
+                acc += ws * accs[s];
+                lg += ws * __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
+            }
+        }
+        out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
+        if (c == 0) lse[head0 + g] = lg > 0.f ? (mg + log2f(lg)) * kLn2 : -INFINITY;
     }
 }
 
@@ -431,6 +772,8 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
 //      out = sum_s 2^(m_s-m*) acc_s / L, lse = (m* + log2 L) ln 2.  Lane s fetches (m_s, l_s),
 //      the weights follow from warp reductions, then each lane sums four channels with the
 //      loads of eight splits in flight together.
+//      cpp > 0: the partials come from decode_cta_kernel, whose split count follows from the pair's
+//      page count (n_split = ceil(cnt / ceil(cnt / cpp))); merged != 0: out/lse are final already.
 //   2. H2O epilogue (zbuf != NULL): score_accum[pid,h,t] += sum_g 2^(z2[g] - lse_g*log2e) for
 //      every attended token slot of the pair.  The slots of a pair are spread over gridDim.y
 //      CTAs; each of them recomputes the pair's lse (the cheap half of the merge), only
@@ -442,7 +785,7 @@ combine_kernel(const float *__restrict__ partials, const float *__restrict__ zbu
                const int32_t *__restrict__ sel_idx, const int32_t *__restrict__ sel_cnt,
                float *__restrict__ out, float *__restrict__ lse, float *__restrict__ score_accum,
                int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int pages_per_split,
-               int max_splits, const int32_t *__restrict__ tok_cnt) {
+               int max_splits, const int32_t *__restrict__ tok_cnt, int cpp, int merged) {
     constexpr int PSTRIDE = D + 4;
     __shared__ float s_lse2[8];
     const int pair = blockIdx.x;
@@ -454,7 +797,8 @@ combine_kernel(const float *__restrict__ partials, const float *__restrict__ zbu
     const int len = seq_lens[r];
     const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
     const bool nothing = cnt <= 0 || n_r == 0;
-    const int n_split = nothing ? 0 : (cnt + pages_per_split - 1) / pages_per_split;
+    if (cpp > 0 && !nothing) pages_per_split = (cnt + cpp - 1) / cpp;
+    const int n_split = (nothing || merged) ? 0 : (cnt + pages_per_split - 1) / pages_per_split;
     const int g = warp;                               // query head of the group handled by this warp
     const bool writer = blockIdx.y == 0;
     if (g < G) {
@@ -564,40 +908,68 @@ bool make_page_map(CUtensorMap *map, const void *base, const se_params &p) {
 
 template <int D>
 cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache, const void *v_cache,
-                          const int32_t *page_table, const int32_t *seq_lens, const int32_t *sel_idx,
-                          const int32_t *sel_cnt, float *out, float *lse, float *score_accum, uint32_t *tok_keys,
-                          void *workspace, const WorkspaceLayout &L, int stages, cudaStream_t stream) {
+                          const int32_t *page_table, const int32_t *seq_lens, int32_t *sel_idx, int32_t *sel_cnt,
+                          const SelectFromScores *from_scores, float *out, float *lse, float *score_accum,
+                          uint32_t *tok_keys, void *workspace, const WorkspaceLayout &L, int stages,
+                          cudaStream_t stream) {
     using C = DecCfg<D>;
-    const DecodePlan plan = make_decode_plan(p);
+    // an observation layer always runs on the warp-unit kernel (the only one that scores tokens)
+    const DecodePlan plan = make_decode_plan(p, tok_keys != nullptr);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     const int G = p.H_q / p.H_kv, GP = next_pow2(G);
     float *zbuf = score_accum ? reinterpret_cast<float *>(ws + L.zbuf) : nullptr;
+    float *partials = reinterpret_cast<float *>(ws + L.partials);
+    uint32_t *status = reinterpret_cast<uint32_t *>(ws + L.status);
+    const bool select = from_scores != nullptr;
+    SelectArgs sa = {};
+    sa.sel_idx = sel_idx;
+    sa.sel_cnt = sel_cnt;
+    if (select) {
+        sa.scores = reinterpret_cast<const float *>(ws + L.scores);
+        sa.pitch = score_pitch(p);
+        sa.k_pages = from_scores->k_pages;
+        sa.sink = p.sink_pages;
+        sa.recent = p.recent_pages;
+    }
     cudaError_t e = cudaSuccess;
     if (stages & 1) {
-    CUtensorMap k_map, v_map;
-    if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
-    const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
-                        (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 16 + 1024;
-    auto kern = tok_keys ? decode_kernel<D, true> : decode_kernel<D, false>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
-        k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-        reinterpret_cast<float *>(ws + L.partials), zbuf, tok_keys,
-        p.B, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
-        effective_scale(p) * kLog2e, reinterpret_cast<uint32_t *>(ws + L.status));
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+        CUtensorMap k_map, v_map;
+        if (!make_page_map(&k_map, k_cache, p) || !make_page_map(&v_map, v_cache, p)) return cudaErrorInvalidValue;
+        const float scale_log2 = effective_scale(p) * kLog2e;
+        if (plan.cta_units) {
+            const size_t smem = CtaCfg<D>::smem_bytes(p.k_max);
+            auto kern = select ? decode_cta_kernel<D, true> : decode_cta_kernel<D, false>;
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
+                k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sa, out, lse, partials, zbuf, p.H_kv, G, GP,
+                p.max_pages, p.num_phys_pages, p.k_max, plan.max_splits, plan.merge_in_kernel ? 1 : 0, scale_log2,
+                status, reinterpret_cast<uint32_t *>(ws + L.pairctl));
+        } else {
+            const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
+                                (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 16 + 1024;
+            if (select) return cudaErrorInvalidValue;         // only CTA units select in the kernel
+            auto kern = tok_keys ? decode_kernel<D, true> : decode_kernel<D, false>;
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
+                k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sa, out, lse, partials, zbuf, tok_keys,
+                p.B, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
+                scale_log2, status);
+        }
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
     }
     if (!(stages & 2)) return e;
-    if (plan.max_splits == 1 && !score_accum) return e;       // every pair is written by one warp
+    const bool merged = plan.max_splits == 1 || (plan.cta_units && plan.merge_in_kernel);
+    if (merged && !score_accum) return e;                     // out/lse are final and there is no epilogue
     // with the H2O epilogue the token slots of a pair (16 per selected page) are spread over
     // several CTAs, two slots per thread
     const int slot_ctas = score_accum ? (p.k_max * kPage + 511) / 512 : 1;
     combine_kernel<D><<<dim3(p.B * p.H_kv, slot_ctas), 256, 0, stream>>>(
-        reinterpret_cast<const float *>(ws + L.partials), zbuf, page_table, seq_lens, sel_idx, sel_cnt, out, lse,
-        score_accum, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
-        nullptr);
+        partials, zbuf, page_table, seq_lens, sel_idx, sel_cnt, out, lse, score_accum, p.H_kv, G, GP, p.max_pages,
+        p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits, nullptr, plan.cta_units ? plan.max_splits : 0,
+        merged ? 1 : 0);
     return cudaGetLastError();
 }
 
@@ -872,7 +1244,7 @@ cudaError_t launch_token_decode_t(const se_params &p, const void *q, const void 
                                   const int32_t *tok_cnt, int n_out, float *out, float *lse, void *workspace,
                                   const WorkspaceLayout &L, cudaStream_t stream) {
     using C = TokCfg<D>;
-    const DecodePlan plan = make_decode_plan(p);        // a unit of the plan = one 16-token tile
+    const DecodePlan plan = make_decode_plan(p, true);  // warp units; a unit of the plan = one 16-token tile
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     const int G = p.H_q / p.H_kv, GP = next_pow2(G);
     const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
@@ -890,7 +1262,7 @@ cudaError_t launch_token_decode_t(const se_params &p, const void *q, const void 
     combine_kernel<D><<<dim3(p.B * p.H_kv, 1), 256, 0, stream>>>(
         reinterpret_cast<const float *>(ws + L.partials), nullptr, page_table, seq_lens, nullptr, nullptr, out, lse,
         nullptr, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max, plan.pages_per_split, plan.max_splits,
-        tok_cnt);
+        tok_cnt, 0, 0);
     return cudaGetLastError();
 }
 
@@ -911,14 +1283,14 @@ int decode_warps_per_cta() { return kDecWarps; }
 
 cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *k_cache,
                                  const void *v_cache, const int32_t *page_table,
-                                 const int32_t *seq_lens, const int32_t *sel_idx,
-                                 const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                                 const int32_t *seq_lens, int32_t *sel_idx, int32_t *sel_cnt,
+                                 const SelectFromScores *from_scores, float *out, float *lse, float *score_accum,
                                  uint32_t *tok_keys, void *workspace, const WorkspaceLayout &L, int stages,
                                  cudaStream_t stream) {
     return (p.D == 128) ? launch_decode<128>(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                                             out, lse, score_accum, tok_keys, workspace, L, stages, stream)
+                                             from_scores, out, lse, score_accum, tok_keys, workspace, L, stages, stream)
                         : launch_decode<64>(p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                                            out, lse, score_accum, tok_keys, workspace, L, stages, stream);
+                                            from_scores, out, lse, score_accum, tok_keys, workspace, L, stages, stream);
 }
 
 }  // namespace se

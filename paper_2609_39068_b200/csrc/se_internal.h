@@ -13,12 +13,22 @@ namespace se {
 // the problem shape alone (never from device data).
 struct DecodePlan {
     int grid;               // CTAs
-    int pages_per_split;    // selected pages one warp handles for one (request, head) pair
-    int max_splits;         // splits per pair = ceil(k_max / pages_per_split)
+    bool cta_units;         // true: decode_cta_kernel, one CTA per (pair, CTA-split); false: decode_kernel,
+                            // one warp per (pair, split)
+    int pages_per_split;    // warp units: selected pages of one split
+    int max_splits;         // splits per pair (warp units: ceil(k_max / pages_per_split); CTA units: CTAs per pair)
+    bool merge_in_kernel;   // CTA units: the last-arriving CTA of a pair merges the pair's partials itself
+};
+
+// the selection comes from the page scores in the workspace: the attention kernel runs the top-k
+struct SelectFromScores {
+    int k_pages;
 };
 
 int  device_sm_count();
-DecodePlan make_decode_plan(const se_params &p);
+DecodePlan make_decode_plan(const se_params &p, bool warp_units_only = false);
+// whether the attention kernel's own top-k covers the shape (otherwise the top-k kernel runs)
+bool select_in_decode_ok(const se_params &p);
 WorkspaceLayout make_layout(const se_params &p);
 float effective_scale(const se_params &p);
 // floats per (request, kv-head) row of the score scratch: rows start 16-byte aligned
@@ -37,10 +47,12 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
                                const WorkspaceLayout &L, cudaStream_t stream, int stages = 3);
 // stages: 1 = scoring kernel only (scores stay in the workspace), 2 = top-k kernel only, 3 = both
 
+// from_scores != nullptr: sel_idx / sel_cnt are OUTPUTS - the attention kernel selects the pages
+// itself from the scores a scoring kernel left in the workspace
 cudaError_t launch_sparse_decode(const se_params &p, const void *q, const void *k_cache,
                                  const void *v_cache, const int32_t *page_table,
-                                 const int32_t *seq_lens, const int32_t *sel_idx,
-                                 const int32_t *sel_cnt, float *out, float *lse, float *score_accum,
+                                 const int32_t *seq_lens, int32_t *sel_idx, int32_t *sel_cnt,
+                                 const SelectFromScores *from_scores, float *out, float *lse, float *score_accum,
                                  uint32_t *tok_keys, void *workspace, const WorkspaceLayout &L, int stages,
                                  cudaStream_t stream);
 // tok_keys != nullptr: observation layer - [B, 16*max_pages] order-preserving integer images of

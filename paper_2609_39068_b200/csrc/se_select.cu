@@ -20,6 +20,7 @@
 //                crossing bin, then a page-ordered compaction, so equal scores go to the lower
 //                page and the list is ascending.
 #include "se_internal.h"
+#include "se_topk.cuh"
 
 namespace se {
 
@@ -75,264 +76,12 @@ __device__ __forceinline__ bool decode_unit(int t, int total_units, int big, con
     return true;
 }
 
-// ---------------------------------------------------------------------------------
-// Top-k of one (request, kv-head) pair by ONE warp, run inside the scoring grid by the warp whose
-// arrival completed the pair's scores (a finite ticket: nobody waits).  Same result as topk_kernel
-// (the k_eff best candidates by (score descending, page ascending), forced pages on top, ascending
-// output), but the keys are re-read from the score row (it sits in L2: it was written moments
-// ago) in every pass instead of living in registers, and the only scratch is a histogram of BINS
-// ints in shared memory.  Passes: span and counts -> histogram over the span and the bin holding
-// the k_eff-th best key (a crowded bin gets another level over its own span) -> the few keys of
-// that bin, ranked by brute force -> emission in page order.
-// ---------------------------------------------------------------------------------
-constexpr int kWarpTopkUnroll = 4;       // float4 loads in flight per lane
-
-__device__ __forceinline__ int warp_incl_scan(int v, int lane) {
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(kFull, v, o);
-        if (lane >= o) v += t;
-    }
-    return v;
-}
-
-// Calls f(u, page0, keys[4], forcedmask) for this lane's float4 groups, in page order over the
-// warp: group u of an iteration covers pages page0..page0+3 with page0 = 4*(f0 + 32*u + lane).
-// Keys of absent pages, of pages past the request and of forced pages are kKeyAbsent; bit c of
-// forcedmask marks a forced page.  Every lane runs the same number of iterations.
-template <typename F>
-__device__ __forceinline__ void warp_topk_pass(const float4 *row4, int n, int sink, int recent, int lane, F &&f) {
-    const int n4 = (n + 3) >> 2;
-    for (int f0 = 0; f0 < n4; f0 += 32 * kWarpTopkUnroll) {
-        float4 v[kWarpTopkUnroll];
-#pragma unroll
-        for (int u = 0; u < kWarpTopkUnroll; ++u) {
-            const int fi = f0 + 32 * u + lane;
-            v[u] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-            if (fi < n4) v[u] = __ldcg(row4 + fi);
-        }
-#pragma unroll
-        for (int u = 0; u < kWarpTopkUnroll; ++u) {
-            if (f0 + 32 * u >= n4) break;                       // uniform over the warp
-            const int page0 = 4 * (f0 + 32 * u + lane);
-            uint32_t keys[4];
-            uint32_t forcedmask = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float ev = c == 0 ? v[u].x : c == 1 ? v[u].y : c == 2 ? v[u].z : v[u].w;
-                uint32_t key = (page0 + c < n) ? f32_key(ev) : kKeyAbsent;
-                if (key != kKeyAbsent && (page0 + c < sink || page0 + c >= n - recent)) {
-                    forcedmask |= 1u << c;
-                    key = kKeyAbsent;
-                }
-                keys[c] = key;
-            }
-            f(page0, keys, forcedmask);
-        }
-    }
-}
-
-template <int BINS>
-__device__ __forceinline__ void warp_topk(const float *row, int n, int k_pages, int k_max, int sink, int recent,
-                                       int32_t *out, int32_t *cnt_out, int *hist, int lane) {
-    constexpr int BPL = BINS / 32;                   // bins per lane
-    constexpr int BINBITS = BINS == 2048 ? 11 : BINS == 1024 ? 10 : 9;
-    static_assert(BINS == (1 << BINBITS) && BPL >= 16, "bins");
-    const float4 *row4 = reinterpret_cast<const float4 *>(row);
-
-    // ---- pass 1: candidates, forced pages, span of the candidates' keys
-    uint32_t kmin = 0xffffffffu, kmax = 0u;
-    int present = 0, forced = 0;
-    warp_topk_pass(row4, n, sink, recent, lane, [&](int, const uint32_t (&keys)[4], uint32_t fm) {
-        forced += __popc(fm);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const bool ok = keys[c] != kKeyAbsent;
-            present += ok;
-            kmin = ok ? min(kmin, keys[c]) : kmin;
-            kmax = ok ? max(kmax, keys[c]) : kmax;
-        }
-    });
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        present += __shfl_xor_sync(kFull, present, o);
-        forced += __shfl_xor_sync(kFull, forced, o);
-        kmin = min(kmin, __shfl_xor_sync(kFull, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
-    }
-    forced = min(forced, k_max);
-    const int k_eff = min(min(k_pages, k_max - forced), present);
-    const int total = k_eff + forced;
-    if (total == 0) {
-        for (int i = lane; i < k_max; i += 32) out[i] = -1;
-        if (lane == 0) *cnt_out = 0;
-        return;
-    }
-
-    // ---- threshold (T_key, T_page): taken <=> key > T_key || (key == T_key && page <= T_page)
-    uint32_t T_key = 0xffffffffu;
-    int T_page = -1;
-    int remaining = k_eff;
-    bool ties = false;
-    if (k_eff > 0 && k_eff == present) {
-        T_key = kmin;
-        T_page = 0x7fffffff;
-    } else if (k_eff > 0 && kmin == kmax) {
-        T_key = kmin;
-        ties = true;
-    } else if (k_eff > 0) {
-        uint32_t lo = kmin;
-        uint32_t span = kmax - kmin + 1u;
-        int width = 32 - __clz(kmax - kmin);
-        for (;;) {
-            const int sh = width > BINBITS ? width - BINBITS : 0;
-#pragma unroll
-            for (int j = 0; j < BPL; ++j) hist[j * 32 + lane] = 0;
-            __syncwarp();
-            warp_topk_pass(row4, n, sink, recent, lane, [&](int, const uint32_t (&keys)[4], uint32_t) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t d = keys[c] - lo;
-                    if (d < span) atomicAdd(&hist[(BINS - 1) - (int)(d >> sh)], 1);
-                }
-            });
-            __syncwarp();
-            // the bin b with  #(keys in bins before b) < remaining <= #(keys in bins up to b): first
-            // the lane whose block of BPL bins holds it (rotated reads: no bank conflicts), then the
-            // bin inside that block
-            int sum = 0;
-#pragma unroll
-            for (int j = 0; j < BPL; ++j) sum += hist[lane * BPL + ((j + lane) & (BPL - 1))];
-            const int inc = warp_incl_scan(sum, lane);
-            const int owner = __ffs(__ballot_sync(kFull, inc - sum < remaining && remaining <= inc)) - 1;
-            int run = __shfl_sync(kFull, inc - sum, owner);
-            int bin = 0, inbin = 0;
-            for (int c = 0; c < BPL; c += 32) {
-                const int v = hist[owner * BPL + c + lane];
-                const int inc2 = warp_incl_scan(v, lane);
-                const int e2 = run + inc2 - v;
-                const unsigned hit = __ballot_sync(kFull, e2 < remaining && remaining <= e2 + v);
-                if (hit) {
-                    const int src = __ffs(hit) - 1;
-                    bin = owner * BPL + c + src;
-                    run = __shfl_sync(kFull, e2, src);
-                    inbin = __shfl_sync(kFull, v, src);
-                    break;
-                }
-                run += __shfl_sync(kFull, inc2, 31);
-            }
-            __syncwarp();
-            const int digit = (BINS - 1) - bin;
-            remaining -= run;
-            lo += (uint32_t)digit << sh;
-            span = 1u << sh;
-            width = sh;
-            T_key = lo;
-            if (inbin == remaining) {            // the whole bin is taken
-                T_page = 0x7fffffff;
-                break;
-            }
-            if (sh == 0) {                       // the bin is one key value: ties
-                ties = true;
-                break;
-            }
-            if (inbin <= 32) {
-                // few keys left: collect them (hist[0..31] keys, hist[32..63] pages, hist[64] count) and
-                // rank each against the others
-                if (lane == 0) hist[64] = 0;
-                __syncwarp();
-                warp_topk_pass(row4, n, sink, recent, lane, [&](int page0, const uint32_t (&keys)[4], uint32_t) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const uint32_t d = keys[c] - lo;
-                        if (d < span) {
-                            const int pos = atomicAdd(&hist[64], 1);
-                            if (pos < 32) {
-                                hist[pos] = (int)keys[c];
-                                hist[32 + pos] = page0 + c;
-                            }
-                        }
-                    }
-                });
-                __syncwarp();
-                const bool has = lane < inbin;
-                const uint32_t mk = has ? (uint32_t)hist[lane] : 0u;
-                const int mp = has ? hist[32 + lane] : 0x7fffffff;
-                int rank = 0;
-                for (int i = 0; i < inbin; ++i) {
-                    const uint32_t ok = __shfl_sync(kFull, mk, i);
-                    const int op = __shfl_sync(kFull, mp, i);
-                    rank += (ok > mk) || (ok == mk && op < mp);
-                }
-                const int own = __ffs(__ballot_sync(kFull, has && rank == remaining - 1)) - 1;
-                T_key = __shfl_sync(kFull, mk, own);
-                T_page = __shfl_sync(kFull, mp, own);
-                __syncwarp();
-                break;
-            }
-        }
-    }
-    if (ties) {
-        // T_page = the remaining-th page, in page order, among the keys equal to T_key
-        int base = 0, found = -1;
-        warp_topk_pass(row4, n, sink, recent, lane, [&](int page0, const uint32_t (&keys)[4], uint32_t) {
-            if (found >= 0) return;                                // uniform: found is broadcast below
-            int cnt = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) cnt += keys[c] == T_key;
-            const int inc = warp_incl_scan(cnt, lane);
-            const int excl = base + inc - cnt;
-            int mine = -1;
-            if (excl < remaining && remaining <= excl + cnt) {
-                int seen = excl;
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (keys[c] == T_key && ++seen == remaining) mine = page0 + c;
-            }
-            const unsigned hit = __ballot_sync(kFull, mine >= 0);
-            if (hit) found = __shfl_sync(kFull, mine, __ffs(hit) - 1);
-            base += __shfl_sync(kFull, inc, 31);
-        });
-        T_page = found;
-    }
-
-    // ---- emission in page order
-    int base = 0;
-    warp_topk_pass(row4, n, sink, recent, lane, [&](int page0, const uint32_t (&keys)[4], uint32_t fm) {
-        uint32_t take = fm;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            take |= (uint32_t)(keys[c] > T_key || (keys[c] == T_key && page0 + c <= T_page)) << c;
-        const int cnt = __popc(take);
-        const int inc = warp_incl_scan(cnt, lane);
-        int pos = base + inc - cnt;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if ((take >> c) & 1u) {
-                if (pos < k_max) out[pos] = page0 + c;
-                ++pos;
-            }
-        }
-        base += __shfl_sync(kFull, inc, 31);
-    });
-    for (int i = total + lane; i < k_max; i += 32) out[i] = -1;
-    if (lane == 0) *cnt_out = total;
-}
-
-// Arguments of the top-k that the scoring grid runs itself (pair_cnt != nullptr): one arrival counter
-// per (request, kv-head) pair, zero on entry and left at zero.
-struct FusedTopk {
-    uint32_t *pair_cnt;
-    int32_t *sel_idx, *sel_cnt;
-    int k_pages, k_max, sink, recent;
-};
-
 template <int D>
-__global__ void __launch_bounds__(kScoreWarps * 32, 3)
+__global__ void __launch_bounds__(kScoreWarps * 32)
 score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t *__restrict__ k_cache,
              uint8_t *meta_out, const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
-             float *scores, int pitch, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
-             uint32_t *status, const FusedTopk tk) {
+             float *__restrict__ scores, int pitch, int B, int H_kv, int G, int max_pages, int P_phys, float scale,
+             uint32_t *status) {
     using C = ScoreCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // layout: [buffers: warps*2*BUF] [mbarriers: warps*2*8] [prefix: B+1 ints] [npages: B ints] [lens: B ints]
@@ -540,40 +289,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
 
     // Three batches are live: `cur` is computed, `nxt` is in flight, `nn` has only its page-table
     // entries on the way, so that its copies can be issued the moment a buffer frees up.
-    // Fused top-k: a request without pages has no work unit, so nobody would arrive for its pairs;
-    // their (empty) selections are written here.
-    if (tk.pair_cnt != nullptr) {
-        for (int r = gw; r < B; r += tw) {
-            if (npages[r] != 0) continue;
-            for (int i = lane; i < H_kv * tk.k_max; i += 32) tk.sel_idx[(size_t)r * H_kv * tk.k_max + i] = -1;
-            for (int h = lane; h < H_kv; h += 32) tk.sel_cnt[(size_t)r * H_kv + h] = 0;
-        }
-    }
-    // Arrival bookkeeping of the fused top-k.  Pages this warp has scored for the pair it is working
-    // on are reported (one atomic add on the pair's counter) when its stream leaves the pair; the
-    // answer is looked at one batch later, so the round trip is hidden.  The warp whose report
-    // completes a pair (counter == pages of the request) runs that pair's top-k.
-    int arr_pages = 0;                           // scored for the current pair, not yet reported
-    int pend_n = 0, pend_add = 0, pend_pair = 0; // a report whose answer has not been looked at (pend_n > 0)
-    uint32_t pend_old = 0;                       // valid in lane 0
-    auto resolve = [&](uint32_t scratch_smem) -> bool {
-        if (pend_n <= 0) return false;
-        const bool last = (int)__shfl_sync(kFull, pend_old, 0) + pend_add == pend_n;
-        const int n = pend_n, pair = pend_pair;
-        pend_n = 0;
-        if (!last) return false;
-        __threadfence();                         // the other warps' scores of this pair are visible from here on
-        if (lane == 0) tk.pair_cnt[pair] = 0u;   // left at zero for the next launch
-        int *hist = reinterpret_cast<int *>(my_buf + (scratch_smem - buf0));
-        warp_topk<(C::BUF >= 8192 ? 2048 : 1024)>(scores + (size_t)pair * pitch, n, tk.k_pages, tk.k_max, tk.sink,
-                                                 tk.recent, tk.sel_idx + (size_t)pair * tk.k_max, tk.sel_cnt + pair,
-                                                 hist, lane);
-        __syncwarp();
-        // the histogram was written through the generic proxy; the buffer is refilled by bulk copies
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        return true;
-    };
-
     Batch cur, nxt, nn;
     decode_unit(gw, total_units, big_units, prefix, npages, B, H_kv, cur);
     if (cur.unit < 0) {
@@ -638,25 +353,6 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
             if (cur.b0 + gid + 8 < cur.n_r) dst[gid + 8] = (pid_hi >= 0) ? s_hi * scale : ninf;
         }
         __syncwarp();        // every lane is done reading the buffer before it is refilled
-
-        if (tk.pair_cnt != nullptr) {
-            arr_pages += max(0, min(kPB, cur.n_r - cur.b0));
-            // the buffer just consumed is free: a top-k that has fallen to this warp uses it as scratch
-            resolve(buf0 + slot * C::BUF);
-            const bool leave = nxt.unit < 0 || nxt.r != cur.r || nxt.h != cur.h;
-            if (leave) {
-                if (arr_pages > 0) {
-                    __threadfence();             // this warp's scores of the pair, before its report
-                    __syncwarp();
-                    pend_pair = cur.r * H_kv + cur.h;
-                    if (lane == 0) pend_old = atomicAdd(tk.pair_cnt + pend_pair, (uint32_t)arr_pages);
-                    pend_add = arr_pages;
-                    pend_n = cur.n_r;
-                }
-                arr_pages = 0;
-            }
-        }
-
         // refill the buffer just consumed with `nn` (its page-table entries arrived long ago)
         if (nn.unit >= 0) pid_nn = issue(nn, slot, pid_nn);
         // advance: cur <- nxt <- nn <- the batch after
@@ -675,274 +371,29 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // give the copy that may still be in flight a bounded chance to land before leaving
         mbar_wait(bar0 + (slot ^ 1) * 8, (phases >> (slot ^ 1)) & 1u);
-    } else if (tk.pair_cnt != nullptr) {
-        resolve(buf0);                           // the last report of this warp; both buffers are free now
     }
     check_out();
 }
 
 // ---------------------------------------------------------------------------------
-// top-k: one CTA per (request, kv-head).  Thread t holds a run of consecutive pages in registers
-// (as order-preserving integer keys), so thread order is page order.  The k-th largest key is
-// found by one 2048-bin histogram over the span [kmin, kmax] of the request's keys; the bin
-// that holds it usually has a handful of keys, which are ranked by brute force (a further
-// histogram level over the bin's span serves crowded bins).  The result is a threshold
-// (key, page): a page is taken when its key is above the threshold key, or equal to it and
-// the page not above the threshold page - equal scores go to the lower page.  One prefix sum
-// over the per-thread counts then gives every thread the position of its pages in the
-// ascending output list.
+// top-k kernel: one CTA per (request, kv-head) runs cta_topk (se_topk.cuh) on the pair's score row;
+// the keys live in dynamic shared memory (cta_topk_key_words(max_pages) words).
 // ---------------------------------------------------------------------------------
-constexpr int kTopkBins = 2048;
-constexpr int kTopkBinBits = 11;
-constexpr int kTopkList = 32;        // bins with up to this many keys are ranked by brute force
+constexpr int kTopkThreads = 256;
 
-// THREADS threads per CTA, up to KPT (a multiple of 4) keys per thread: n <= THREADS*KPT.
-template <int THREADS, int KPT, bool kForced>
-__global__ void __launch_bounds__(THREADS, 1024 / THREADS)
+__global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float *__restrict__ scores, int pitch, const int32_t *__restrict__ seq_lens, int H_kv,
             int max_pages, int k_pages, int k_max, int sink_pages, int recent_pages,
             int32_t *__restrict__ sel_idx, int32_t *__restrict__ sel_cnt) {
-    constexpr int NW = THREADS / 32;
-    constexpr int BPT = kTopkBins / THREADS;           // histogram bins per thread
-    static_assert(KPT % 4 == 0 && KPT <= 32 && BPT >= 1, "top-k shape");
-    __shared__ __align__(16) int s_hist[kTopkBins];    // indexed by 2047 - digit: prefix = keys above
-    __shared__ int s_tot[4][32];
-    __shared__ int s_red[4][NW];
-    __shared__ int s_res[6];
-    __shared__ uint32_t s_lkey[kTopkList];
-    __shared__ int s_lpage[kTopkList];
-    __shared__ int s_ln;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    extern __shared__ __align__(16) uint32_t topk_keys[];
+    __shared__ TopkScratch S;
     const int pair = blockIdx.x;
-    const int r = pair / H_kv;
-    const int len = seq_lens[r];
+    const int len = seq_lens[pair / H_kv];
     int n = len > 0 ? (len + kPage - 1) / kPage : 0;
     if (n > max_pages) n = max_pages;
-    if (n > KPT * THREADS) n = KPT * THREADS;          // cannot happen: the launcher picks KPT from max_pages
-    int32_t *out = sel_idx + (size_t)pair * k_max;
-
-    // thread t owns pages [t*kpe, (t+1)*kpe): kpe is the smallest multiple of 4 that covers the request
-    const int kpe = min(KPT, (((n + THREADS - 1) / THREADS) + 3) & ~3);
-    const int base = tid * kpe;
-    const float4 *row4 = reinterpret_cast<const float4 *>(scores + (size_t)pair * pitch);
-    uint32_t keys[KPT];
-    uint32_t forcedmask = 0;         // pages taken regardless of their score; they do not compete
-#pragma unroll
-    for (int j4 = 0; j4 < KPT / 4; ++j4) {
-        const int i = base + 4 * j4;
-        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-        if (4 * j4 < kpe && i < n) v = __ldg(row4 + (i >> 2));
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const float ev = c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
-            uint32_t key = (i + c < n) ? f32_key(ev) : kKeyAbsent;         // absent pages score -inf
-            if (kForced && key != kKeyAbsent && (i + c < sink_pages || i + c >= n - recent_pages)) {
-                forcedmask |= 1u << (4 * j4 + c);
-                key = kKeyAbsent;
-            }
-            keys[4 * j4 + c] = key;
-        }
-    }
-#pragma unroll
-    for (int e = 0; e < BPT; ++e) s_hist[tid * BPT + e] = 0;
-    if (tid == 0) s_ln = 0;
-
-    // ---- candidates, forced pages, and the span of the candidates' keys
-    uint32_t kmin = 0xffffffffu, kmax = 0u;
-    int present = 0, forced = kForced ? __popc(forcedmask) : 0;
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const bool ok = keys[j] != kKeyAbsent;
-        present += ok;
-        kmin = ok ? min(kmin, keys[j]) : kmin;
-        kmax = ok ? max(kmax, keys[j]) : kmax;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        present += __shfl_xor_sync(kFull, present, o);
-        if (kForced) forced += __shfl_xor_sync(kFull, forced, o);
-        kmin = min(kmin, __shfl_xor_sync(kFull, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
-    }
-    if (lane == 0) {
-        s_red[0][warp] = present;
-        s_red[1][warp] = (int)kmin;
-        s_red[2][warp] = (int)kmax;
-        s_red[3][warp] = forced;
-    }
-    __syncthreads();
-    present = 0;
-    forced = 0;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) {
-        present += s_red[0][w];
-        forced += s_red[3][w];
-        kmin = min(kmin, (uint32_t)s_red[1][w]);
-        kmax = max(kmax, (uint32_t)s_red[2][w]);
-    }
-    forced = min(forced, k_max);
-    const int k_eff = min(min(k_pages, k_max - forced), present);      // candidates to take
-    if (k_eff + forced == 0) {
-        for (int i = tid; i < k_max; i += THREADS) out[i] = -1;
-        if (tid == 0) sel_cnt[pair] = 0;
-        return;
-    }
-
-    // ---- threshold (T_key, T_page): taken <=> key > T_key || (key == T_key && page <= T_page)
-    uint32_t T_key = 0xffffffffu;
-    int T_page = -1;                         // k_eff == 0: nothing competes
-    int remaining = k_eff;                   // still to take among the keys inside the current span
-    bool ties = false;                       // the keys equal to T_key are taken in page order
-    if (k_eff > 0 && k_eff == present) {     // every candidate is wanted
-        T_key = kmin;
-        T_page = 0x7fffffff;
-    } else if (k_eff > 0 && kmin == kmax) {  // all equal
-        T_key = kmin;
-        ties = true;
-    } else if (k_eff > 0) {
-        uint32_t lo = kmin;                              // the current span is [lo, lo + span)
-        uint32_t span = kmax - kmin + 1u;
-        int width = 32 - __clz(kmax - kmin);             // span <= 2^width
-        for (int level = 0;; ++level) {
-            const int sh = width > kTopkBinBits ? width - kTopkBinBits : 0;
-            if (level > 0) {
-#pragma unroll
-                for (int e = 0; e < BPT; ++e) s_hist[tid * BPT + e] = 0;
-                __syncthreads();
-            }
-            // keys spread over the bins nearly evenly, so plain shared-memory atomics rarely collide
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                if ((j & ~3) < kpe) {
-                    const uint32_t d = keys[j] - lo;
-                    if (d < span) atomicAdd(&s_hist[(kTopkBins - 1) - (int)(d >> sh)], 1);
-                }
-            }
-            __syncthreads();
-            // the bin b with  #(keys in bins above b) < remaining <= #(keys in bins above or in b)
-            int loc[BPT], sum = 0;
-#pragma unroll
-            for (int e = 0; e < BPT; ++e) {
-                loc[e] = s_hist[tid * BPT + e];
-                sum += loc[e];
-            }
-            const int excl = cta_excl_scan<NW>(sum, s_tot[level & 1], lane, warp);
-            if (excl < remaining && remaining <= excl + sum) {
-                int run = excl;
-#pragma unroll
-                for (int e = 0; e < BPT; ++e) {
-                    if (run < remaining && remaining <= run + loc[e]) {
-                        s_res[0] = tid * BPT + e;
-                        s_res[1] = run;
-                        s_res[2] = loc[e];
-                    }
-                    run += loc[e];
-                }
-            }
-            __syncthreads();
-            const int digit = (kTopkBins - 1) - s_res[0];
-            const int inbin = s_res[2];
-            remaining -= s_res[1];
-            lo += (uint32_t)digit << sh;
-            span = 1u << sh;
-            width = sh;
-            T_key = lo;
-            if (inbin == remaining) {            // the whole bin is taken
-                T_page = 0x7fffffff;
-                break;
-            }
-            if (sh == 0) {                       // the bin is one key value: ties
-                ties = true;
-                break;
-            }
-            if (inbin <= kTopkList) {
-                // few keys left: collect them and rank each against the others
-#pragma unroll
-                for (int j = 0; j < KPT; ++j) {
-                    if ((j & ~3) < kpe) {
-                        const uint32_t d = keys[j] - lo;
-                        if (d < span) {
-                            const int pos = atomicAdd(&s_ln, 1);
-                            if (pos < kTopkList) {
-                                s_lkey[pos] = keys[j];
-                                s_lpage[pos] = base + j;
-                            }
-                        }
-                    }
-                }
-                __syncthreads();
-                // every warp ranks the (at most 32) collected keys on its own: lane i holds entry i,
-                // the entry that `remaining - 1` others precede is the threshold
-                {
-                    const bool has = lane < inbin;
-                    const uint32_t mk = has ? s_lkey[lane] : 0u;
-                    const int mp = has ? s_lpage[lane] : 0x7fffffff;
-                    int rank = 0;
-                    for (int i = 0; i < inbin; ++i) {
-                        const uint32_t ok = __shfl_sync(kFull, mk, i);
-                        const int op = __shfl_sync(kFull, mp, i);
-                        rank += (ok > mk) || (ok == mk && op < mp);
-                    }
-                    const int owner = __ffs(__ballot_sync(kFull, has && rank == remaining - 1)) - 1;
-                    T_key = __shfl_sync(kFull, mk, owner);
-                    T_page = __shfl_sync(kFull, mp, owner);
-                }
-                break;
-            }
-        }
-    }
-    if (ties) {
-        // T_page = the remaining-th page, in page order, among the keys equal to T_key
-        int cnt = 0;
-#pragma unroll
-        for (int j = 0; j < KPT; ++j) cnt += keys[j] == T_key;
-        const int excl = cta_excl_scan<NW>(cnt, s_tot[2], lane, warp);
-        if (excl < remaining && remaining <= excl + cnt) {
-            int run = excl;
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                if (keys[j] == T_key) {
-                    ++run;
-                    if (run == remaining) s_res[5] = base + j;
-                }
-            }
-        }
-        __syncthreads();
-        T_page = s_res[5];
-    }
-    // ---- ordered compaction
-    uint32_t takemask = forcedmask;
-    const int jT = T_page - base;            // page <= T_page  <=>  j <= jT
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const bool take = keys[j] > T_key || (keys[j] == T_key && j <= jT);
-        takemask |= (uint32_t)take << j;
-    }
-    int pos = cta_excl_scan<NW>(__popc(takemask), s_tot[3], lane, warp);
-    const int total = k_eff + forced;
-    if (k_max <= kTopkBins) {
-        // the list is put together in shared memory (the histogram is no longer needed) and
-        // written out with coalesced stores, padding included
-#pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            if ((takemask >> j) & 1u) {
-                if (pos < k_max) s_hist[pos] = base + j;
-                ++pos;
-            }
-        }
-        __syncthreads();
-        for (int i = tid; i < k_max; i += THREADS) out[i] = i < total ? s_hist[i] : -1;
-    } else {
-#pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            if ((takemask >> j) & 1u) {
-                if (pos < k_max) out[pos] = base + j;
-                ++pos;
-            }
-        }
-        for (int i = total + tid; i < k_max; i += THREADS) out[i] = -1;
-    }
-    if (tid == 0) sel_cnt[pair] = k_eff + forced;
+    const int total = cta_topk<kTopkThreads>(scores + (size_t)pair * pitch, n, k_pages, k_max, sink_pages,
+                                             recent_pages, topk_keys, S, nullptr, sel_idx + (size_t)pair * k_max);
+    if (threadIdx.x == 0) sel_cnt[pair] = total;
 }
 
 // Dense-layer mode (budget >= context): every present page is selected, so there is nothing to
@@ -976,7 +427,7 @@ select_all_kernel(const int32_t *__restrict__ page_table, const int32_t *__restr
 template <int D>
 cudaError_t launch_score(const se_params &p, const void *q, const void *meta, const void *k_cache,
                          const int32_t *page_table, const int32_t *seq_lens, float *scores, uint32_t *status,
-                         const FusedTopk &tk, cudaStream_t stream) {
+                         cudaStream_t stream) {
     using C = ScoreCfg<D>;
     const size_t smem = (size_t)kScoreWarps * 2 * C::BUF + kScoreWarps * 2 * 8 +
                         (size_t)(3 * p.B + 1) * sizeof(int);
@@ -994,7 +445,7 @@ cudaError_t launch_score(const se_params &p, const void *q, const void *meta, co
     kern<<<(unsigned)grid, kScoreWarps * 32, smem, stream>>>(
         (const uint16_t *)q, (const uint8_t *)meta, (const uint8_t *)k_cache, (uint8_t *)const_cast<void *>(meta),
         page_table, seq_lens, scores, score_pitch(p), p.B, p.H_kv,
-        p.H_q / p.H_kv, p.max_pages, p.num_phys_pages, effective_scale(p), status, tk);
+        p.H_q / p.H_kv, p.max_pages, p.num_phys_pages, effective_scale(p), status);
     return cudaGetLastError();
 }
 
@@ -1007,23 +458,6 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     float *scores = reinterpret_cast<float *>(ws + L.scores);
     uint32_t *status = reinterpret_cast<uint32_t *>(ws + L.status);
-    // One kernel or two.  With many pairs the top-k of a pair runs inside the scoring grid, by the warp
-    // whose arrival completed the pair's scores, while the other warps keep streaming: it costs no
-    // launch and no serial phase.  With few pairs every pair completes at the very end, where a top-k
-    // by a single warp would be exposed; a CTA per pair in a kernel of its own is then faster.
-    bool fuse = L.has_pairctl && stages == 3 && p.B * p.H_kv >= 2 * device_sm_count();
-    if (p.flags & SE_FLAG_SELECT_ONE_KERNEL) fuse = L.has_pairctl && stages == 3;
-    if (p.flags & SE_FLAG_SELECT_TWO_KERNELS) fuse = false;
-    FusedTopk tk = {};
-    if (fuse) {
-        tk.pair_cnt = reinterpret_cast<uint32_t *>(ws + L.pairctl);
-        tk.sel_idx = sel_idx;
-        tk.sel_cnt = sel_cnt;
-        tk.k_pages = k_pages;
-        tk.k_max = p.k_max;
-        tk.sink = p.sink_pages;
-        tk.recent = p.recent_pages;
-    }
     if (stages == 3 && k_pages >= p.max_pages && p.k_max >= p.max_pages) {
         // dense layer: the budget covers any context this shape can hold
         if (k_cache != nullptr) {           // the fused call still owes the newest page's summary
@@ -1037,30 +471,16 @@ cudaError_t launch_page_select(const se_params &p, const void *q, const void *me
     }
     if (stages & 1) {
         cudaError_t e = (p.D == 128)
-                            ? launch_score<128>(p, q, meta, k_cache, page_table, seq_lens, scores, status, tk, stream)
-                            : launch_score<64>(p, q, meta, k_cache, page_table, seq_lens, scores, status, tk, stream);
+                            ? launch_score<128>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream)
+                            : launch_score<64>(p, q, meta, k_cache, page_table, seq_lens, scores, status, stream);
         if (e != cudaSuccess) return e;
     }
-    if (!(stages & 2) || fuse) return cudaSuccess;
+    if (!(stages & 2)) return cudaSuccess;
     const int pairs = p.B * p.H_kv;
-#define SE_TOPK(THREADS, KPT)                                                                         \
-    do {                                                                                              \
-        if (p.sink_pages || p.recent_pages)                                                           \
-            topk_kernel<THREADS, KPT, true><<<pairs, THREADS, 0, stream>>>(                           \
-                scores, score_pitch(p), seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, p.sink_pages,      \
-                p.recent_pages,                                                                       \
-                sel_idx, sel_cnt);                                                                    \
-        else                                                                                          \
-            topk_kernel<THREADS, KPT, false><<<pairs, THREADS, 0, stream>>>(                          \
-                scores, score_pitch(p), seq_lens, p.H_kv, p.max_pages, k_pages, p.k_max, 0, 0, sel_idx,     \
-                sel_cnt);                                                                             \
-    } while (0)
-    // short requests: fewer keys per thread; long ones: more threads, so the per-thread chains stay short
-    if (p.max_pages <= 1024) SE_TOPK(256, 4);
-    else if (p.max_pages <= 2048) SE_TOPK(256, 8);
-    else if (p.max_pages <= 4096) SE_TOPK(256, 16);
-    else SE_TOPK(1024, 8);
-#undef SE_TOPK
+    const size_t key_bytes = (size_t)cta_topk_key_words(p.max_pages, kTopkThreads) * sizeof(uint32_t);
+    topk_kernel<<<pairs, kTopkThreads, key_bytes, stream>>>(scores, score_pitch(p), seq_lens, p.H_kv, p.max_pages,
+                                                            k_pages, p.k_max, p.sink_pages, p.recent_pages, sel_idx,
+                                                            sel_cnt);
     return cudaGetLastError();
 }
 
@@ -1122,7 +542,6 @@ extern "C" int se_page_select_static(const se_params *p, const void *q, const vo
     se::WorkspaceLayout L = {};
     L.status = 0;
     L.scores = 256;
-    L.has_pairctl = false;                    // no arrival counters in the array: always the two-kernel selection
     L.total = need;
     cudaError_t e = se::launch_page_select(*p, q, meta, nullptr, page_table, seq_lens, budget_tokens / se::kPage,
                                            sel_idx, sel_cnt, scratch, L, s);

@@ -40,12 +40,10 @@ def test_random_shapes(seed):
     w_cpu = wl.build("fuzz%d" % seed, 700 + seed % 50, 0, c["seq"], c["H_q"], c["H_kv"], c["D"], c["budget"],
                      "cpu", **c["kw"])
     w = w_cpu.to("cuda")
-    # the launch plan is normally picked from the shape; the sweep forces each of them in turn
-    flags = (0, binding.SE_FLAG_SELECT_ONE_KERNEL, binding.SE_FLAG_SELECT_TWO_KERNELS)[seed % 3]
-    st = binding.DecodeState(w, sink_pages=c["sink"], recent_pages=c["recent"], flags=flags)
+    st = binding.DecodeState(w, sink_pages=c["sink"], recent_pages=c["recent"])
     st.rebuild_meta()
     u = w.score_accum.clone() if w.score_accum is not None else None
-    st.step(score_accum=u, fused=bool(seed % 2))
+    st.step(score_accum=u, fused=bool(seed % 2))       # se_decode_step, or the three separate calls
     torch.cuda.synchronize()
     assert st.status() == 0, c
     if u is not None:

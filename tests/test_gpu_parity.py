@@ -456,38 +456,68 @@ PLAN_CASES.update({
 
 
 @pytest.mark.parametrize("name", sorted(PLAN_CASES))
-def test_both_selection_plans_give_the_same_selection(name):
-    """se_page_select has two launch plans (scoring grid that runs each pair's top-k itself / scoring
-    kernel + top-k kernel); whichever the shape picks, both must return the same pages, twice in a row."""
+def test_decode_step_equals_the_separate_calls(name):
+    """se_decode_step (scores -> top-k inside the attention kernel's prologue, in-kernel merge) must
+    return what se_meta_update + se_page_select + se_sparse_decode return: summaries and selection bit for
+    bit, out / lse bit for bit too (same pages, same split geometry), on a first and a second call."""
     kw = dict(PLAN_CASES[name])
     seq, sink, recent = kw.pop("seq"), kw.pop("sink", 0), kw.pop("recent", 0)
-    w = wl.build(name, 800, 0, seq, kw.pop("H_q"), kw.pop("H_kv"), kw.pop("D"), kw.pop("budget"), "cuda", **kw)
+    accum = "shared_prefix_pages" not in kw           # the H2O epilogue does not allow aliased pages
+    w = wl.build(name, 800, 0, seq, kw.pop("H_q"), kw.pop("H_kv"), kw.pop("D"), kw.pop("budget"), "cuda",
+                 with_score_accum=True, **kw)
+    short = (w.seq_lens - 1).clamp(min=0).contiguous()
+    ft = torch.zeros(w.B, dtype=torch.int32, device="cuda")
     res = []
-    for flags in (binding.SE_FLAG_SELECT_TWO_KERNELS, binding.SE_FLAG_SELECT_ONE_KERNEL, 0):
-        st = binding.DecodeState(w, sink_pages=sink, recent_pages=recent, flags=flags)
-        st.rebuild_meta()
-        for rep in range(2):
-            st.sel_idx.fill_(-7)
-            st.sel_cnt.fill_(-7)
-            st.select() if rep == 0 else st.select_fused()
-            torch.cuda.synchronize()
-            assert st.status() == 0
-            res.append((st.sel_idx.clone(), st.sel_cnt.clone()))
-    for idx, cnt in res[1:]:
-        assert torch.equal(idx, res[0][0]) and torch.equal(cnt, res[0][1])
+    for fused in (False, True, True):
+        st = binding.DecodeState(w, sink_pages=sink, recent_pages=recent)
+        binding.se_meta_update(st.p, w.k_cache, w.page_table, short, st.meta, first_tok=ft)   # stale newest page
+        u = w.score_accum.clone()
+        st.step(score_accum=u if accum else None, fused=fused)
+        torch.cuda.synchronize()
+        assert st.status() == 0
+        res.append((st.meta.view(torch.int16).clone(), st.sel_idx.clone(), st.sel_cnt.clone(), st.out.clone(),
+                    st.lse.clone(), u))
+    for other in res[1:]:
+        for x, y in zip(res[0], other):
+            assert torch.equal(x, y)
 
 
-def test_ties_with_the_one_kernel_plan():
+def test_ties_with_selection_inside_the_attention_kernel():
     w_cpu = wl.build("ties", 860, 0, [16 * 40, 16 * 700], 4, 1, 128, 16 * 8, "cpu")
     w_cpu.k_cache[1:] = w_cpu.k_cache[0]
     w = w_cpu.to("cuda")
-    st = binding.DecodeState(w, flags=binding.SE_FLAG_SELECT_ONE_KERNEL)
+    st = binding.DecodeState(w)
     st.rebuild_meta()
-    st.select()
-    st.decode()
+    st.step()
     torch.cuda.synchronize()
     assert st.sel_idx.cpu()[0, 0].tolist() == list(range(8)) and st.sel_idx.cpu()[1, 0].tolist() == list(range(8))
     compare(w_cpu, st)
+
+
+@pytest.mark.parametrize("pairs", [2, 40, 148, 200, 400])
+def test_every_launch_plan_against_the_oracle(pairs):
+    """The attention step has three geometries, picked from the number of (request, kv-head) pairs: CTA
+    units with an in-kernel merge (<= 148 pairs), warp units with splits and the merge kernel (< 296),
+    one warp per pair (>= 296).  Each one against the oracle, with and without the H2O epilogue."""
+    H_kv = 2 if pairs % 2 == 0 else 1
+    B = pairs // H_kv
+    rng = np.random.default_rng(pairs)
+    seq = [int(x) for x in rng.integers(1, 2500, size=B)]
+    seq[0] = 0
+    for accum in (False, True):
+        w_cpu = wl.build("plan%d" % pairs, 897, 0, seq, 4 * H_kv, H_kv, 128, 320, "cpu", permute_pool=True,
+                         prune_fraction=0.1, with_score_accum=True, poison_tail=True)
+        w = w_cpu.to("cuda")
+        st = binding.DecodeState(w)
+        st.rebuild_meta()
+        u = w.score_accum.clone() if accum else None
+        st.step(score_accum=u)
+        torch.cuda.synchronize()
+        assert st.status() == 0
+        if accum:
+            compare(w_cpu, st, u_before=w_cpu.score_accum.numpy(), u_after=u.cpu().numpy())
+        else:
+            compare(w_cpu, st)
 
 
 def _run_shard(w, accum):

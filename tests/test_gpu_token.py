@@ -102,7 +102,9 @@ def test_observe_select_reuse_small(D, H_q, H_kv, prune):
     st2.w, st2.sel_idx, st2.sel_cnt = st.w, st.sel_idx, st.sel_cnt
     st2.decode()
     torch.cuda.synchronize()
-    assert torch.equal(st.out, st2.out) and torch.equal(st.lse, st2.lse)
+    # (an observation layer runs on warp units, the plain call may run on CTA units: same pages, another
+    # split geometry, hence fp32 rounding)
+    assert (st.out - st2.out).abs().max().item() <= 1e-5 and (st.lse - st2.lse).abs().max().item() <= 1e-5
     s_ref, present, s_gpu = check_scores(w_cpu, keys)
     for budget, recent in [(64, 8), (200, 0), (16, 40), (2000, 4), (0, 8)]:
         tok_idx, tok_cnt = select(st, keys, w, budget, recent)
