@@ -91,6 +91,12 @@ DecodePlan make_decode_plan(const se_params &p, bool warp_units_only) {
 // config 3, so those shapes keep the top-k kernel.
 bool select_in_decode_ok(const se_params &p) { return make_decode_plan(p).cta_units; }
 
+// The fused step needs the CTAs of a pair in one thread-block cluster (portable size: up to 8).
+bool score_in_decode_ok(const se_params &p) {
+    const DecodePlan plan = make_decode_plan(p);
+    return plan.cta_units && plan.max_splits <= 8;
+}
+
 WorkspaceLayout make_layout(const se_params &p) {
     WorkspaceLayout L;
     const DecodePlan plan = make_decode_plan(p);
@@ -250,9 +256,11 @@ static int sparse_decode_stages(const se_params *p, const void *q, const void *k
 }
 
 // What se_decode_step launches for `p`: 0 = dense layer (summary update, list of all pages, attention),
-// 1 = scoring kernel + attention kernel that selects in its prologue, 2 = scoring, top-k kernel, attention.
+// 1 = scoring kernel + attention kernel that selects in its prologue, 2 = scoring, top-k kernel, attention,
+// 3 = one kernel that scores, selects and attends.
 static int step_plan(const se_params &p, int k_pages) {
     if (k_pages >= p.max_pages && p.k_max >= p.max_pages) return 0;
+    if (score_in_decode_ok(p)) return 3;
     return select_in_decode_ok(p) ? 1 : 2;
 }
 
@@ -275,12 +283,16 @@ int se_decode_step(const se_params *p, const void *q, const void *k_cache, const
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int plan = step_plan(*p, k_pages);
     // plan 1: only the scoring kernel of the selection runs (stages = 1); the scores stay in the workspace
-    cudaError_t e = launch_page_select(*p, q, meta, k_cache, page_table, seq_lens, k_pages, sel_idx, sel_cnt,
-                                       workspace, L, s, plan == 1 ? 1 : 3);
-    if (e != cudaSuccess) return SE_ERR_CUDA;
-    const SelectFromScores from_scores = {k_pages};
+    cudaError_t e = cudaSuccess;
+    if (plan != 3) {
+        e = launch_page_select(*p, q, meta, k_cache, page_table, seq_lens, k_pages, sel_idx, sel_cnt, workspace, L, s,
+                               plan == 1 ? 1 : 3);
+        if (e != cudaSuccess) return SE_ERR_CUDA;
+    }
+    const SelectFromScores from_scores = {k_pages, plan == 3 ? meta : nullptr};
     e = launch_sparse_decode(*p, q, k_cache, v_cache, page_table, seq_lens, sel_idx, sel_cnt,
-                             plan == 1 ? &from_scores : nullptr, out, lse, score_accum, nullptr, workspace, L, 3, s);
+                             (plan == 1 || plan == 3) ? &from_scores : nullptr, out, lse, score_accum, nullptr,
+                             workspace, L, 3, s);
     return e == cudaSuccess ? SE_OK : SE_ERR_CUDA;
 }
 
@@ -290,7 +302,7 @@ int se_decode_step_launches(const se_params *p, int32_t budget_tokens, int with_
     const DecodePlan dp = make_decode_plan(*p);
     const bool merged = dp.max_splits == 1 || (dp.cta_units && dp.merge_in_kernel);
     const int attention = 1 + ((!merged || with_score_accum) ? 1 : 0);
-    return (plan == 1 ? 1 : 2) + attention;
+    return (plan == 3 ? 0 : plan == 1 ? 1 : 2) + attention;
 }
 
 int se_sparse_decode(const se_params *p, const void *q, const void *k_cache, const void *v_cache,

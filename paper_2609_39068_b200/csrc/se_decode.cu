@@ -536,6 +536,168 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------
+// Scoring phase of the fused step (Appendix A, Quest summary and score equations): the CTA scores the
+// logical pages [b_lo, b_hi) of its pair and writes the fp32 scores to the pair's score row.  Same
+// arithmetic as score_kernel (se_select.cu): sum_c max(q m, q M) = sum_c (q^- m + q^+ M) as a dense
+// [16 pages x 2D] . [2D x G] contraction per batch of 16 summaries, which arrive by 1-D bulk copies
+// into two padded buffers per warp (the warp's share of the still empty ring).  Warp w takes the
+// batches w, w+8, ... of the CTA's range, eight of them at a time: their page-table entries are
+// fetched together, then the batches run through the double buffer.  The summary of the request's
+// newest page is recomputed from K on the spot and written back, as se_meta_update would.
+// Returns false when a bounded wait gave up.
+// ---------------------------------------------------------------------------------
+struct FusedScoreArgs {
+    const uint8_t *meta;     // [P_phys][H_kv][2][D] bf16 (read; the newest page's entry is written)
+    const uint8_t *k_cache;  // [P_phys][H_kv][16][D] bf16
+    float *scores;           // [pairs][pitch]
+    int pitch;
+    float scale;
+};
+
+template <int D>
+__device__ __forceinline__ bool cta_score_range(uint8_t *wbuf, uint32_t bar0, int *pids, const uint16_t *__restrict__ q,
+                                                size_t head0, int G, const FusedScoreArgs &fs,
+                                                const int32_t *__restrict__ pt_row, int n_r, int len, int b_lo, int b_hi,
+                                                int hh, int H_kv, int P_phys, float *score_row, uint32_t *status,
+                                                int warp, int lane) {
+    constexpr int PHB = 4 * D;                   // bytes of one page summary (min row, max row)
+    constexpr int PITCH = PHB + 16;              // padded: conflict-free ldmatrix
+    constexpr int BUF = kPage * PITCH;
+    constexpr int KSTEPS = 2 * D / 16;
+    constexpr int NBC = 8;                       // batches whose page-table entries are fetched together
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const uint32_t buf0 = smem_u32(wbuf);
+    const int nb = (b_hi - b_lo + kPage - 1) / kPage;            // batches of the CTA
+    const int nbw = nb > warp ? (nb - warp + kDecWarps - 1) / kDecWarps : 0;   // batches of this warp
+    if (nbw == 0) return true;
+
+    // B operand: column n = query head n of the group (zero for n >= G); rows k < D carry q^- (they meet
+    // the min row), rows k >= D carry q^+ (they meet the max row)
+    uint32_t bfrag[KSTEPS][2];
+    {
+        const uint16_t *src = q + (head0 + (gid < G ? gid : 0)) * D + 2 * tid4;
+#pragma unroll
+        for (int sidx = 0; sidx < D / 16; ++sidx) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(src + sidx * 16 + 8 * j));
+                if (gid >= G) w = 0u;
+                const uint32_t negmask = ((w >> 15) & 0x00010001u) * 0xffffu;   // all-ones per negative half
+                bfrag[sidx][j] = w & negmask;
+                bfrag[D / 16 + sidx][j] = w & ~negmask;
+            }
+        }
+    }
+    const uint32_t lm_off = (uint32_t)(((lane & 7) + 8 * ((lane >> 3) & 1)) * PITCH + (lane >> 4) * 16);
+    uint32_t phases = 0u;
+    const int newest = n_r - 1;                  // the page whose summary is recomputed from K
+    const int nv_newest = min(kPage, len - newest * kPage);
+
+    for (int j0 = 0; j0 < nbw; j0 += NBC) {
+        const int nc = min(NBC, nbw - j0);
+        // page-table entries of this chunk of batches: entry e = batch (e >> 4), page offset (e & 15)
+#pragma unroll
+        for (int rep = 0; rep < NBC * kPage / 32; ++rep) {
+            const int e = rep * 32 + lane;
+            const int page = b_lo + (warp + kDecWarps * (j0 + (e >> 4))) * kPage + (e & 15);
+            int pid = -1;
+            if ((e >> 4) < nc && page < b_hi) pid = __ldg(pt_row + page);
+            if (pid >= P_phys) {
+                atomicOr(status, SE_DEV_BAD_PAGE_ID);
+                pid = -1;
+            }
+            pids[e] = pid;
+        }
+        __syncwarp();
+        auto issue = [&](int j) {                // batch j of the chunk into buffer j & 1
+            const int page = b_lo + (warp + kDecWarps * (j0 + j)) * kPage + lane;
+            int pid = lane < kPage ? pids[j * kPage + lane] : -1;
+            if (page == newest) pid = -1;        // summarised from K instead of copied
+            const unsigned valid = __ballot_sync(kFull, pid >= 0);
+            const uint32_t bar = bar0 + (j & 1) * 8;
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)__popc(valid) * PHB);
+            __syncwarp();
+            if (pid >= 0)
+                bulk_g2s(buf0 + (j & 1) * BUF + lane * PITCH, fs.meta + ((size_t)pid * H_kv + hh) * PHB, PHB, bar);
+        };
+        issue(0);
+        if (nc > 1) issue(1);
+        for (int j = 0; j < nc; ++j) {
+            const int slot = j & 1;
+            const int page0 = b_lo + (warp + kDecWarps * (j0 + j)) * kPage;
+            if (!mbar_wait(bar0 + slot * 8, (phases >> slot) & 1u)) return false;
+            phases ^= 1u << slot;
+            const int my_pid = lane < kPage ? pids[j * kPage + lane] : -1;
+            if (newest >= page0 && newest < page0 + kPage) {
+                // the newest page of the request: summary from K (all kv-heads' pages are contiguous per head)
+                const int fl = newest - page0;
+                const int fpid = __shfl_sync(kFull, my_pid, fl);
+                if (fpid >= 0) {
+                    constexpr int LPR = D / 8, TPP = 32 / LPR, KROWS = kPage / TPP;
+                    const int tg = lane / LPR, lr = lane % LPR;
+                    const uint4 *kp = reinterpret_cast<const uint4 *>(fs.k_cache) + ((size_t)fpid * H_kv + hh) * (kPage * D / 8);
+                    uint4 w[KROWS];
+#pragma unroll
+                    for (int i = 0; i < KROWS; ++i) {
+                        const int t = i * TPP + tg;
+                        w[i] = __ldg(kp + (t < nv_newest ? t : 0) * LPR + lr);      // rows past the length repeat row 0
+                    }
+                    uint4 mn = w[0], mx = w[0];
+#pragma unroll
+                    for (int i = 1; i < KROWS; ++i) {
+                        mn.x = bmin2(mn.x, w[i].x); mn.y = bmin2(mn.y, w[i].y); mn.z = bmin2(mn.z, w[i].z); mn.w = bmin2(mn.w, w[i].w);
+                        mx.x = bmax2(mx.x, w[i].x); mx.y = bmax2(mx.y, w[i].y); mx.z = bmax2(mx.z, w[i].z); mx.w = bmax2(mx.w, w[i].w);
+                    }
+#pragma unroll
+                    for (int m = LPR; m < 32; m <<= 1) {
+                        mn.x = bmin2(mn.x, __shfl_xor_sync(kFull, mn.x, m)); mn.y = bmin2(mn.y, __shfl_xor_sync(kFull, mn.y, m));
+                        mn.z = bmin2(mn.z, __shfl_xor_sync(kFull, mn.z, m)); mn.w = bmin2(mn.w, __shfl_xor_sync(kFull, mn.w, m));
+                        mx.x = bmax2(mx.x, __shfl_xor_sync(kFull, mx.x, m)); mx.y = bmax2(mx.y, __shfl_xor_sync(kFull, mx.y, m));
+                        mx.z = bmax2(mx.z, __shfl_xor_sync(kFull, mx.z, m)); mx.w = bmax2(mx.w, __shfl_xor_sync(kFull, mx.w, m));
+                    }
+                    if (tg < 2) {
+                        const uint4 val = tg == 0 ? mn : mx;
+                        uint4 *gp = reinterpret_cast<uint4 *>(const_cast<uint8_t *>(fs.meta)) + ((size_t)fpid * H_kv + hh) * (2 * D / 8);
+                        gp[tg * LPR + lr] = val;
+                        sts128(buf0 + slot * BUF + fl * PITCH + (tg * LPR + lr) * 16, val);
+                    }
+                    __syncwarp();
+                }
+            }
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t a_base = buf0 + slot * BUF + lm_off;
+#pragma unroll
+            for (int sidx = 0; sidx < KSTEPS; ++sidx) {
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4(a_base + sidx * 32, a0, a1, a2, a3);
+                mma_bf16_16816(acc, a0, a1, a2, a3, bfrag[sidx][0], bfrag[sidx][1]);
+            }
+            // acc[0],acc[1]: page gid, heads 2*tid4, 2*tid4+1;  acc[2],acc[3]: page gid+8, same heads
+            const float ninf = -INFINITY;
+            float s_lo = fmaxf(2 * tid4 < G ? acc[0] : ninf, 2 * tid4 + 1 < G ? acc[1] : ninf);
+            float s_hi = fmaxf(2 * tid4 < G ? acc[2] : ninf, 2 * tid4 + 1 < G ? acc[3] : ninf);
+            s_lo = fmaxf(s_lo, __shfl_xor_sync(kFull, s_lo, 1));
+            s_hi = fmaxf(s_hi, __shfl_xor_sync(kFull, s_hi, 1));
+            s_lo = fmaxf(s_lo, __shfl_xor_sync(kFull, s_lo, 2));
+            s_hi = fmaxf(s_hi, __shfl_xor_sync(kFull, s_hi, 2));
+            const int pid_lo = __shfl_sync(kFull, my_pid, gid);
+            const int pid_hi = __shfl_sync(kFull, my_pid, gid + 8);
+            if (tid4 == 0) {
+                if (page0 + gid < b_hi) score_row[page0 + gid] = (pid_lo >= 0) ? s_lo * fs.scale : ninf;
+                if (page0 + gid + 8 < b_hi) score_row[page0 + gid + 8] = (pid_hi >= 0) ? s_hi * fs.scale : ninf;
+            }
+            __syncwarp();        // every lane is done reading the buffer before it is refilled
+            if (j + 2 < nc) {
+                fence_proxy_async();             // the newest page's summary may have been stored with ordinary stores
+                issue(j + 2);
+            }
+        }
+        __syncwarp();
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------------
 // decode_cta_kernel: one CTA per (pair, CTA-split); gridDim.x = pairs * cpp.
 //   1. selection list of the pair in shared memory: the caller's, or (kSelect) the CTA's own top-k of
 //      the score row (every CTA of a pair computes the same list; CTA-split 0 writes it out);
@@ -563,14 +725,16 @@ struct CtaCfg {
     static size_t smem_bytes(int k_max) { return kSel + (size_t)k_max * sizeof(int) + 1024; }
 };
 
-template <int D, bool kSelect>
+// kFused (implies kSelect): the CTAs of a pair form a thread-block cluster and score the pair's pages
+// first (cta_score_range), each its share; a cluster barrier later every CTA reads the whole score row.
+template <int D, bool kSelect, bool kFused>
 __global__ void __launch_bounds__(kDecWarps * 32, 1)
 decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                   const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
-                  const int32_t *__restrict__ seq_lens, const SelectArgs sa, float *__restrict__ out,
-                  float *__restrict__ lse, float *partials, float *__restrict__ zbuf, int H_kv, int G, int GP,
-                  int max_pages, int P_phys, int k_max, int cpp, int merge_here, float scale_log2, uint32_t *status,
-                  uint32_t *ticket) {
+                  const int32_t *__restrict__ seq_lens, const SelectArgs sa, const FusedScoreArgs fs,
+                  float *__restrict__ out, float *__restrict__ lse, float *partials, float *__restrict__ zbuf,
+                  int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int cpp, int merge_here,
+                  float scale_log2, uint32_t *status, uint32_t *ticket) {
     using C = DecCfg<D>;
     using L = CtaCfg<D>;
     extern __shared__ uint8_t smem_dyn[];
@@ -588,8 +752,13 @@ decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + L::kBars) + warp * C::MAXST;
     if (lane == 0) {
         for (int s = 0; s < P.nstage; ++s) mbar_init(smem_u32(&bars[s]), 2);
+        if (kFused) {                             // the scoring phase has two buffers with a barrier each
+            mbar_init(smem_u32(&bars[C::MAXST - 2]), 1);
+            mbar_init(smem_u32(&bars[C::MAXST - 1]), 1);
+        }
         mbar_fence_init();
     }
+    __syncwarp();
     P.bar0 = smem_u32(&bars[0]);
     P.ring0 = smem_u32(ring);
     P.phases = 0;
@@ -609,6 +778,24 @@ decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const int len = __ldg(seq_lens + r);
     const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
     int32_t *sel_row = sa.sel_idx + (size_t)pair * k_max;
+    if (kFused) {
+        // this CTA's share of the pair's pages, in whole batches of 16
+        const int per = ((n_r + cpp - 1) / cpp + kPage - 1) / kPage * kPage;
+        const int b_lo = min(n_r, cs * per), b_hi = min(n_r, b_lo + per);
+        const bool ok = cta_score_range<D>(ring, smem_u32(&bars[C::MAXST - 2]), P.ent_y, q, head0, G, fs,
+                                           page_table + (size_t)r * max_pages, n_r, len, b_lo, b_hi, h, H_kv, P_phys,
+                                           fs.scores + (size_t)pair * fs.pitch, status, warp, lane);
+        if (!ok && lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
+        // every CTA of the pair has written its scores before any of them reads the row
+        __threadfence();
+        if (cpp > 1) {
+            asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+            asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        } else {
+            __syncthreads();
+        }
+        fence_proxy_async();
+    }
     int cnt;
     if (kSelect) {
         TopkScratch &S = *reinterpret_cast<TopkScratch *>(smem_al);
@@ -938,13 +1125,38 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
         const float scale_log2 = effective_scale(p) * kLog2e;
         if (plan.cta_units) {
             const size_t smem = CtaCfg<D>::smem_bytes(p.k_max);
-            auto kern = select ? decode_cta_kernel<D, true> : decode_cta_kernel<D, false>;
+            const bool fused = select && from_scores->meta != nullptr;
+            auto kern = fused ? decode_cta_kernel<D, true, true>
+                              : (select ? decode_cta_kernel<D, true, false> : decode_cta_kernel<D, false, false>);
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
-                k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sa, out, lse, partials, zbuf, p.H_kv, G, GP,
-                p.max_pages, p.num_phys_pages, p.k_max, plan.max_splits, plan.merge_in_kernel ? 1 : 0, scale_log2,
-                status, reinterpret_cast<uint32_t *>(ws + L.pairctl));
+            FusedScoreArgs fs = {};
+            if (fused) {
+                fs.meta = static_cast<const uint8_t *>(from_scores->meta);
+                fs.k_cache = static_cast<const uint8_t *>(k_cache);
+                fs.scores = reinterpret_cast<float *>(ws + L.scores);
+                fs.pitch = score_pitch(p);
+                fs.scale = effective_scale(p);
+            }
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(plan.grid);
+            cfg.blockDim = dim3(kDecWarps * 32);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            if (fused && plan.max_splits > 1) {       // the CTAs of a pair form a cluster (they share a barrier)
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = plan.max_splits;
+                attr[0].val.clusterDim.y = 1;
+                attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+            }
+            e = cudaLaunchKernelEx(&cfg, kern, k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sa, fs, out, lse,
+                                   partials, zbuf, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max,
+                                   plan.max_splits, plan.merge_in_kernel ? 1 : 0, scale_log2, status,
+                                   reinterpret_cast<uint32_t *>(ws + L.pairctl));
+            if (e != cudaSuccess) return e;
         } else {
             const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
                                 (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 16 + 1024;

@@ -23,12 +23,16 @@ struct DecodePlan {
 // the selection comes from the page scores in the workspace: the attention kernel runs the top-k
 struct SelectFromScores {
     int k_pages;
+    void *meta;              // != nullptr: fused step - the attention kernel also scores the pages (CTA units whose
+                             // CTAs per pair fit a thread-block cluster), refreshing the newest page's summary
 };
 
 int  device_sm_count();
 DecodePlan make_decode_plan(const se_params &p, bool warp_units_only = false);
 // whether the attention kernel's own top-k covers the shape (otherwise the top-k kernel runs)
 bool select_in_decode_ok(const se_params &p);
+// whether the attention kernel can also score the pages (one launch for the whole step)
+bool score_in_decode_ok(const se_params &p);
 WorkspaceLayout make_layout(const se_params &p);
 float effective_scale(const se_params &p);
 // floats per (request, kv-head) row of the score scratch: rows start 16-byte aligned

@@ -475,8 +475,14 @@ def test_decode_step_equals_the_separate_calls(name):
         st.step(score_accum=u if accum else None, fused=fused)
         torch.cuda.synchronize()
         assert st.status() == 0
+        # the fp32 page scores left in the workspace (whichever kernel wrote them), up to each request's last page
+        sc = binding.page_scores_view(st.p, st.workspace).clone()
+        for r in range(w.B):
+            sc[r, :, (int(w.seq_lens[r]) + 15) // 16:] = 0
+        if w.budget // 16 >= w.max_pages:
+            sc.zero_()                        # dense-layer mode: nothing is scored
         res.append((st.meta.view(torch.int16).clone(), st.sel_idx.clone(), st.sel_cnt.clone(), st.out.clone(),
-                    st.lse.clone(), u))
+                    st.lse.clone(), u, sc.view(torch.int32)))
     for other in res[1:]:
         for x, y in zip(res[0], other):
             assert torch.equal(x, y)
