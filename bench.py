@@ -1,27 +1,36 @@
 #!/usr/bin/env python
 """Benchmark of the sparse decode-attention hot path.
 
-A *step* is one pass of the whole path over one batch of synthetic requests, per layer:
-summary of the page holding each request's newest token -> page scores + top-k
-(``se_page_select_fused`` does both; ``se_meta_update`` + ``se_page_select`` are the separate
-calls) -> ``se_sparse_decode`` (split-K attention over the selected pages, LSE merge, optional
-H2O statistic).  The default workload is the
-continuous-batching mix (config 3: 64 requests, 4096..65536 tokens, 32/8 heads, D=128,
-budget 2048, page tables permuted over one pool); ``--config`` picks another one.
+A *step* is one pass of the whole path over one batch of synthetic requests, per layer: summary of
+the page holding each request's newest token -> page scores -> top-k -> attention over the selected
+pages, LSE merge, optional H2O statistic.  One call does it all: ``se_decode_step`` (the library
+picks the launch plan from the shape).  The default workload is the continuous-batching mix
+(config 3: 64 requests, 4096..65536 tokens, 32/8 heads, D=128, budget 2048, page tables permuted over
+one pool); ``--config`` picks another one, and the default run also times the other four configs
+briefly (``other_configs`` in the JSON line).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
 
-N > 1 is launched with torch.distributed.run, one rank per GPU; every rank runs the same
-shape on its own data (the path shards by request / kv-head without any collective), so
-scaling is weak.  Rank 0 prints ONE JSON line.
+N > 1: one rank per GPU (started by the driver with torch.distributed.run, or by this script itself
+when it is called without a rank environment); every rank runs the same shape on its own data - the
+path shards by request / kv-head without any collective - so scaling is weak.  Rank 0 prints ONE JSON
+line.
+
+Timing follows the paper's protocol (Experimental Settings, "Measurement Protocol"): one discarded
+run, then three windows, each 32 untimed replays followed by K/3 timed ones, CUDA events on the
+launching stream, host synchronisation only at window boundaries.  Cold L2 either by construction
+(inputs larger than L2, or R independent instances replayed round-robin so that R steps touch at
+least four times the L2) or, for the tiny config, by a flush between steps.
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import dataclasses
 import json
 import os
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -39,26 +48,14 @@ METRIC = "sparse_decode_us_per_step"
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+WINDOW_WARMUP = 32                     # untimed replays in front of every timed window
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
-# capture summarised in profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {
-    # profiles/full_capture_config3_b24.md: 201.91 MB read for 24576 tiles, scaled to 65536 tiles,
-    # plus the 1.06 MB of out/lse a full-size launch writes (it writes no partials: one split)
-    "config3_contbatch_b64_mix": 539.5e6,
-}
-NCU_TRAFFIC_BYTES_SCORE = {
-    # same capture: 244.97 MB read + 5.07 MB written for 249.3 MB of summaries, scaled to 561.5 MB
-    "config3_contbatch_b64_mix": 563.2e6,
-}
-
-
-# dram bytes of one h2o_compact_kernel launch on the 64-request eviction workload (profiles/)
-H2O_NCU_TRAFFIC_BYTES = 2055e6        # 770.7 MB at 24 requests, scaled by the request count
-
-
-# dram bytes of one token_decode_kernel launch on the 24-request selection-reuse workload (profiles/)
-OMNIKV_NCU_TRAFFIC_BYTES = 209e6     # 69.8 MB at 8 requests, scaled by the request count
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in profiles/
+# (small-batch captures scaled by the pages processed; null where no capture of that workload exists)
+NCU_TRAFFIC_BYTES = {"config3_contbatch_b64_mix": 539.5e6}          # decode_kernel
+NCU_TRAFFIC_BYTES_SCORE = {"config3_contbatch_b64_mix": 563.2e6}    # score_kernel
+H2O_NCU_TRAFFIC_BYTES = 2055e6         # h2o_compact_kernel, 64-request eviction workload
+OMNIKV_NCU_TRAFFIC_BYTES = 209e6       # token_decode_kernel, 24-request selection-reuse workload
 
 
 def measured_peak():
@@ -170,7 +167,9 @@ def checksums(w):
             "page_table": s64(w.page_table), "seq_lens": s64(w.seq_lens)}
 
 
-def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0):
+def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0, instance: int = 0):
+    """The layers of one instance of a config.  Structure (lengths, page table) is the same for every layer
+    and instance; q/K/V values differ (seeded by layer index; other instances and ranks use other layer seeds)."""
     fn = wl.CONFIGS[config]
     if batch:
         base = fn
@@ -178,7 +177,7 @@ def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0):
     layers = []
     first = None
     for l in range(n_layers):
-        w = fn(device, layer=l + 100 * rank) if config != 5 else fn(device, layer=l)
+        w = fn(device, layer=l + 100 * rank + 1000 * instance)
         if first is None:
             first = w
         else:                                 # the block table is per request, shared by all layers
@@ -188,172 +187,472 @@ def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0):
 
 
 # ------------------------------------------------------------------ CPU oracle timing
-def oracle_time(w, target_s=(10.0, 30.0)):
-    """Times the oracle, as it stands, on a bounded sample of the workload's requests and
-    scales to the full batch by the number of (present + selected) pages."""
+def _omp_set_threads(n: int):
+    """Thread count of the oracle's OpenMP loops for the following calls (a libgomp call, not oracle code)."""
+    try:
+        ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+        return True
+    except Exception:
+        return False
+
+
+def oracle_step_time(w, meta_bits, threads=None, min_runs=3, budget_s=20.0):
+    """The oracle, as it stands, on the WHOLE batch of ``w`` (one layer): seconds per decode step, best of
+    >= min_runs.  ``meta_bits``: the page summaries (the rebuild after prefill is set-up for both sides)."""
     import oracle
-    order = list(range(0, w.B, max(1, w.B // 16)))[:16]
-    sub = wl.sub_workload(w, order, "cpu")
-    q, k, v = wl.bf16_bits(sub.q), wl.bf16_bits(sub.k_cache), wl.bf16_bits(sub.v_cache)
-    pt, sl = sub.page_table.numpy(), sub.seq_lens.numpy()
-    meta = oracle.quest_meta(k, pt, sl, first_tok=np.zeros(sub.B, np.int32))
-    u = None if sub.score_accum is None else sub.score_accum.numpy().astype(np.float64)
+    w_cpu = w.to("cpu")
+    q, k, v = wl.bf16_bits(w_cpu.q), wl.bf16_bits(w_cpu.k_cache), wl.bf16_bits(w_cpu.v_cache)
+    pt, sl = w_cpu.page_table.numpy(), w_cpu.seq_lens.numpy()
+    u = None if w_cpu.score_accum is None else w_cpu.score_accum.numpy().astype(np.float64)
+    cores = oracle.num_threads()
+    if threads is not None and _omp_set_threads(threads):
+        cores = threads
     times = []
     t_begin = time.perf_counter()
-    while len(times) < 3 or time.perf_counter() - t_begin < target_s[0]:
+    while len(times) < min_runs or (time.perf_counter() - t_begin < budget_s and len(times) < 10):
         t0 = time.perf_counter()
-        oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
+        oracle.decode_step(q, k, v, pt, sl, w_cpu.budget, meta=meta_bits, u_accum=None if u is None else u.copy())
         times.append(time.perf_counter() - t0)
-        if time.perf_counter() - t_begin > target_s[1]:
-            break
-    n_all = (w.seq_lens.cpu().numpy() + 15) // 16
-    n_sub = (sl + 15) // 16
-    scale = float(n_all.sum()) / float(n_sub.sum())
-    best = min(times)
-    return dict(value=best * scale * 1e6, unit="us", cores=oracle.num_threads(), kind="oracle",
-                sample="%d of %d requests (every %d-th), fp64 C oracle with OpenMP over (request, kv-head), "
-                       "best of %d runs (%.0f s of wall time) = %.1f ms, scaled x%.2f by page count to the full batch"
-                       % (sub.B, w.B, max(1, w.B // 16), len(times), time.perf_counter() - t_begin, best * 1e3, scale),
-                sample_seconds=best)
+    if threads is not None:
+        _omp_set_threads(oracle.num_threads())
+    return min(times), len(times), cores
 
 
-# ------------------------------------------------------------------ main
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=3, choices=sorted(wl.CONFIGS))
-    ap.add_argument("--layers", type=int, default=0, help="layers per step (default 1; 28 for config 5)")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--batch", type=int, default=0,
-                    help="override the number of requests (configs 3-5; for small profiling captures)")
-    ap.add_argument("--no-graph", action="store_true", help="launch the calls directly instead of a CUDA graph")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "h2o_evict", "omnikv_reuse"],
-                    help="decode = the sparse decode step (the headline); h2o_evict = one H2O eviction "
-                         "(retained set + in-place compaction) of 64 requests, 5120 -> 4096 tokens; "
-                         "omnikv_reuse = one observation layer (full attention + token selection) and four "
-                         "sparse layers reusing its 2048+32 tokens, 24 requests of 32768 tokens")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
+# ------------------------------------------------------------------ one config on one rank
+class Instance:
+    """One independent copy of a config's layers with its states, H2O accumulators and the graph of its step."""
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    n_layers = args.layers or (28 if args.config == 5 else 1)
+    def __init__(self, binding, config, dev, n_layers, rank, batch, index, dense_layers=0, use_graph=True):
+        self.layers = make_layers(config, dev, n_layers, rank, batch, index)
+        w0 = self.layers[0]
+        self.h2o = w0.score_accum is not None
+        self.dense_layers = dense_layers
+        self.states = []
+        shared = {}                            # layers with the same shape share one workspace, as an engine would
+        for l, w in enumerate(self.layers):
+            k_max = w0.max_pages if l < dense_layers else None
+            st = binding.DecodeState(w, k_max=k_max, workspace=shared.get(k_max))
+            shared.setdefault(k_max, st.workspace)
+            self.states.append(st)
+        self.accums = [w.score_accum.clone() if self.h2o else None for w in self.layers]
+        for st in self.states:
+            st.rebuild_meta()
+        torch.cuda.synchronize()
+        self.graph = None
+        if use_graph:
+            s = torch.cuda.Stream()
+            s.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(s):
+                self.step()
+            torch.cuda.current_stream().wait_stream(s)
+            torch.cuda.synchronize()
+            self.graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.graph):
+                self.step()
+        self.step()
+        torch.cuda.synchronize()
+        for st in self.states:
+            if st.status() != 0:
+                raise SystemExit("device status word not clean")
 
-    if args.workload in ("h2o_evict", "omnikv_reuse"):
-        if rank == 0:                        # these steps have no multi-GPU leg of their own
-            (run_h2o_evict if args.workload == "h2o_evict" else run_omnikv)(args, local_rank)
-        return
-    if args.impl == "reference":
-        if rank == 0:
-            run_reference(args, n_layers)
-        return
+    def step(self):
+        for l, (st, u) in enumerate(zip(self.states, self.accums)):
+            if l < self.dense_layers:
+                st.step(score_accum=u, budget=16 * st.w.max_pages)
+            else:
+                st.step(score_accum=u)
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    def run(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.step()
 
-    from paper_2609_39068_b200 import binding
-    binding.load()
 
-    layers = make_layers(args.config, dev, n_layers, rank, args.batch)
-    h2o = layers[0].score_accum is not None
-    states = [binding.DecodeState(w) for w in layers]
-    accums = [w.score_accum.clone() if h2o else None for w in layers]
-    for st in states:
-        st.rebuild_meta()
+class Flusher:
+    """Evicts the step's data from L2: a 252 MiB write, then a 252 MiB read of another buffer, so that the
+    lines the timed step displaces are clean (displacing the write's dirty lines would charge the step one
+    write-back per byte it reads)."""
+
+    def __init__(self, dev):
+        self.buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        self.src = torch.zeros(2 * L2_BYTES // 4, dtype=torch.int32, device=dev)
+        self.sink = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.i = 0
+
+    def __call__(self):
+        self.i += 1
+        self.buf.fill_(self.i & 0xFF)
+        self.sink.copy_(self.src.max().reshape(1))
+
+
+def chained_graph(insts):
+    """One CUDA graph that runs the steps of ``insts`` one after the other; returns its replay function."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for i in insts:
+            i.step()
+    torch.cuda.current_stream().wait_stream(s)
     torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in insts:
+            i.step()
+    return g.replay
 
-    def step():
-        for st, u in zip(states, accums):
-            st.step(score_accum=u)
 
-    step()
-    torch.cuda.synchronize()
-    for st in states:
-        if st.status() != 0:
-            raise SystemExit("device status word not clean")
+def timed_windows(run_one, K, barrier, world, dev, flusher=None):
+    """K timed steps in up to three windows (32 untimed replays in front of each); returns (ms per step,
+    per-window ms per step, wall-clock interval)."""
+    n_win = 3 if K >= 96 else 1
+    sizes = [K // n_win] * n_win
+    sizes[-1] += K - sum(sizes)
+    per_window = []
+    t_wall0 = time.perf_counter()
+    for n in sizes:
+        for _ in range(WINDOW_WARMUP):
+            run_one()
+        barrier()
+        if flusher is not None:
+            starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+            ends = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+            for i in range(n):
+                flusher()
+                starts[i].record()
+                run_one()
+                ends[i].record()
+            barrier()
+            ms = sum(a.elapsed_time(b) for a, b in zip(starts, ends))
+        else:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                run_one()
+            e1.record()
+            barrier()
+            ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            ms = float(t.item())
+        per_window.append(ms / n)
+    t_wall1 = time.perf_counter()
+    total = sum(m * n for m, n in zip(per_window, sizes))
+    return total / K, per_window, (t_wall0, t_wall1)
+
+
+class E2E:
+    """The step driven from HOST buffers the way a serving loop drives the library: per step one pinned
+    block per layer goes up (q; with layer 0 also the lengths and the page-table entries that changed -
+    one per request: the entry of its newest page), the step runs, out + lse come back into pinned
+    memory, and the host waits for them.  Uploads, steps and downloads of consecutive layers overlap
+    (three streams inside one graph)."""
+
+    def __init__(self, inst: Instance, dev, use_graph=True):
+        self.inst = inst
+        w0 = inst.layers[0]
+        B = w0.B
+        sl = w0.seq_lens.cpu()
+        pt = w0.page_table.cpu()
+        col = ((sl.to(torch.int64) - 1).clamp(min=0)) // 16
+        flat = torch.arange(B, dtype=torch.int64) * w0.max_pages + col
+        newest = pt.view(-1)[flat].clone()
+        self.up_host, self.up_dev, self.views = [], [], []
+        self.dn_host, self.dn_dev = [], []
+        self.states = []
+        import copy
+        for l, (w, st) in enumerate(zip(inst.layers, inst.states)):
+            tensors = [w.q] + ([w.seq_lens, flat.to(dev), newest.to(dev)] if l == 0 else [])
+            hb, hv = self._packed(tensors, "cpu", True)
+            db, dv = self._packed(tensors, dev, False)
+            for src, h_, d_ in zip(tensors, hv, dv):
+                h_.copy_(src)
+                d_.copy_(src)
+            ob, ov = self._packed([st.out, st.lse], dev, False)
+            hob, _ = self._packed([st.out, st.lse], "cpu", True)
+            st2 = copy.copy(st)               # same params, workspace, summaries and selection buffers
+            st2.w = dataclasses.replace(w, q=dv[0], seq_lens=(dv[1] if l == 0 else self.states[0].w.seq_lens))
+            st2.out, st2.lse = ov
+            self.states.append(st2)
+            self.up_host.append(hb); self.up_dev.append(db); self.views.append(dv)
+            self.dn_host.append(hob); self.dn_dev.append(ob)
+        self.h2d = sum(b.numel() for b in self.up_host)
+        self.d2h = sum(b.numel() for b in self.dn_host)
+        self.s_up, self.s_dn = torch.cuda.Stream(), torch.cuda.Stream()
+        self.graph = None
+        if use_graph:
+            s = torch.cuda.Stream()
+            s.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(s):
+                self.body()
+            torch.cuda.current_stream().wait_stream(s)
+            torch.cuda.synchronize()
+            self.graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.graph):
+                self.body()
+
+    @staticmethod
+    def _packed(tensors, device, pin):
+        """One byte block holding the tensors back to back (16-byte aligned); returns (block, views)."""
+        offs, total = [], 0
+        for t in tensors:
+            offs.append(total)
+            total += (t.numel() * t.element_size() + 15) // 16 * 16
+        block = torch.empty(total, dtype=torch.uint8, device=device)
+        if pin:
+            block = block.pin_memory()
+        views = [block[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for o, t in zip(offs, tensors)]
+        return block, views
+
+    def body(self):
+        main = torch.cuda.current_stream()
+        inst = self.inst
+        self.s_up.wait_stream(main)
+        ups, dones = [], []
+        with torch.cuda.stream(self.s_up):
+            for hb, db in zip(self.up_host, self.up_dev):
+                db.copy_(hb, non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record()
+                ups.append(ev)
+        for l, (st2, u) in enumerate(zip(self.states, inst.accums)):
+            main.wait_event(ups[l])
+            if l == 0:                       # the page-table entries that changed since the last step
+                pt = inst.layers[0].page_table
+                pt.view(-1).index_copy_(0, self.views[0][2], self.views[0][3])
+            if l < inst.dense_layers:
+                st2.step(score_accum=u, budget=16 * st2.w.max_pages)
+            else:
+                st2.step(score_accum=u)
+            ev = torch.cuda.Event()
+            ev.record()
+            dones.append(ev)
+        with torch.cuda.stream(self.s_dn):
+            for l, (ob, hob) in enumerate(zip(self.dn_dev, self.dn_host)):
+                self.s_dn.wait_event(dones[l])
+                hob.copy_(ob, non_blocking=True)
+        main.wait_stream(self.s_dn)
+        main.wait_stream(self.s_up)
+
+    def step(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.body()
+        torch.cuda.synchronize()              # the host needs the result before the next step
+
+
+def gather_ceilings(binding, inst: Instance, dev, iters=20):
+    """Read-only gathers with the access pattern and pipeline shape of the two streaming kernels on the
+    very pages layer 0 reads (se_probe_gather): what the memory system allows for those patterns."""
+    w, st = inst.layers[0], inst.states[0]
+    pt = w.page_table.to(torch.int64)
+    n_r = (w.seq_lens.to(torch.int64) + 15) // 16
+    cols = torch.arange(w.max_pages, device=dev)[None, :]
+    present = (cols < n_r[:, None]) & (pt >= 0)
+    heads = torch.arange(w.H_kv, device=dev, dtype=torch.int64)
+    # summaries: (request, kv-head, page) order, piece = pid*H_kv + h
+    pieces = []
+    for r in range(w.B):
+        pid = pt[r][present[r]]
+        pieces.append((pid[None, :] * w.H_kv + heads[:, None]).reshape(-1))
+    meta_idx = torch.cat(pieces).to(torch.int32).contiguous()
+    # selected pages: K page and V page of the same index next to each other
+    sel = st.sel_idx.to(torch.int64)
+    cnt = st.sel_cnt
+    ok = torch.arange(st.k_max, device=dev)[None, None, :] < cnt[:, :, None]
+    rr = torch.arange(w.B, device=dev)[:, None, None].expand_as(sel)
+    hh = heads[None, :, None].expand_as(sel)
+    pid = pt[rr[ok], sel[ok]]
+    kv_idx = (pid * w.H_kv + hh[ok]).to(torch.int32)
+    kv_idx = torch.stack([kv_idx, kv_idx], dim=1).reshape(-1).contiguous()
+    out = {}
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters * 1e3
+
+    row = 2 * w.D * 2
+    us = timed(lambda: binding.se_probe_gather(st.meta, meta_idx, row, 16, 2, 4, 3))
+    out["summaries_%dB" % row] = {"us": us, "bytes": int(meta_idx.numel()) * row, "gbs": int(meta_idx.numel()) * row / us / 1e3,
+                                  "shape": "16 pieces x 2 stages x 4 warps x 3 CTAs/SM"}
+    page = 16 * w.D * 2
+    us = timed(lambda: binding.se_probe_gather(w.k_cache, kv_idx, page, 2, 5, 4, 1, base1=w.v_cache))
+    out["pages_%dB" % page] = {"us": us, "bytes": int(kv_idx.numel()) * page, "gbs": int(kv_idx.numel()) * page / us / 1e3,
+                               "shape": "K+V page x 5 stages x 4 warps x 1 CTA/SM"}
+    return out
+
+
+def run_config(binding, config, dev, args, rank, world, barrier, full: bool, K: int):
+    """Times one config on this rank.  ``full``: also the per-call times, rooflines, the end-to-end number and
+    the gather ceilings; otherwise a short record for ``other_configs``."""
+    n_layers = args.layers if (full and args.layers) else (28 if config == 5 else 1)
+    batch = args.batch if full else 0
+    use_graph = not args.no_graph
+    dense = args.dense_layers if (full or config == 5) else 0
+    inst0 = Instance(binding, config, dev, n_layers, rank, batch, 0, dense_layers=dense, use_graph=use_graph)
+    layers, states = inst0.layers, inst0.states
+    h2o = inst0.h2o
     bytes_l = [algorithmic_bytes(st.w, st.sel_cnt, h2o) for st in states]
     total_bytes = sum(b["total"] for b in bytes_l)
-    working_set = total_bytes
-    flush = working_set < 2 * L2_BYTES
-    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
-    flush_src = torch.zeros(2 * L2_BYTES // 4, dtype=torch.int32, device=dev) if flush else None
-    flush_sink = torch.zeros(1, dtype=torch.int32, device=dev) if flush else None
+    # cold L2: by size, by rotation over R independent instances (R steps touch >= 4 x L2), or by a flush
+    mode, instances, flusher = "stream", [inst0], None
+    if total_bytes < 2 * L2_BYTES:
+        R = -(-4 * L2_BYTES // total_bytes)
+        if R <= 8:
+            mode = "rotate"
+            instances += [Instance(binding, config, dev, n_layers, rank, batch, i, dense_layers=dense, use_graph=use_graph)
+                          for i in range(1, R)]
+        else:
+            mode = "flush"
+            flusher = Flusher(dev)
+    turn = [0]
 
-    def flush_l2(i):
-        """Evicts the step's data from L2: a 252 MiB write, then a 252 MiB read of another buffer, so that
-        the lines the timed step displaces are clean (displacing the write's dirty lines would charge
-        the step one write-back per byte it reads)."""
-        flush_buf.fill_(i & 0xFF)
-        flush_sink.copy_(flush_src.max().reshape(1))
+    def run_one():
+        instances[turn[0] % len(instances)].run()
+        turn[0] += 1
 
-    graph = None
-    if not args.no_graph:
-        s = torch.cuda.Stream()
-        s.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(s):
-            step()
-        torch.cuda.current_stream().wait_stream(s)
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            step()
-    run_step = graph.replay if graph is not None else step
+    # Steps of a few tens of microseconds: a serving engine replays the layers of a model step as ONE graph,
+    # so the steps of the R instances are chained into one graph of `chain` steps (a replay per step would
+    # add the graph-launch gap, several microseconds, to every step).
+    chain, run_chain = 1, None
+    if mode == "rotate" and use_graph:
+        chain = len(instances) * max(1, 8 // len(instances))
+        if K % chain == 0:
+            run_chain = chained_graph([instances[i % len(instances)] for i in range(chain)])
+        else:
+            chain = 1
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev.index)
     sampler.start()
-
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        run_step()
+    for _ in range(max(args.warmup, 3)):       # the discarded run
+        run_one()
     barrier()
-    K = args.steps
-    t_wall0 = time.perf_counter()
-    if flush:
-        starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
-        ends = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
-        for i in range(K):
-            flush_l2(i)
-            starts[i].record()
-            run_step()
-            ends[i].record()
-        barrier()
-        total_ms = sum(a.elapsed_time(b) for a, b in zip(starts, ends))
+    if run_chain is not None:
+        ms_chain, windows, (t0, t1) = timed_windows(run_chain, K // chain, barrier, world, dev, None)
+        ms_per_step, windows = ms_chain / chain, [m / chain for m in windows]
     else:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(K):
-            run_step()
-        e1.record()
-        barrier()
-        total_ms = e0.elapsed_time(e1)
-    t_wall1 = time.perf_counter()
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / K
-    clocks = sampler.summary(t_wall0, t_wall1)
+        ms_per_step, windows, (t0, t1) = timed_windows(run_one, K, barrier, world, dev, flusher)
+    clocks = sampler.summary(t0, t1)
+    peak, peak_kind = measured_peak()
+    step_gbs = total_bytes / (ms_per_step * 1e-3) / 1e9
+    w0 = layers[0]
+    rec = {
+        "value": ms_per_step * 1e3, "unit": "us", "steps": K, "windows_us": [m * 1e3 for m in windows],
+        "config": {
+            "workload": w0.name, "config_id": config, "layers": n_layers, "B": w0.B, "H_q": w0.H_q, "H_kv": w0.H_kv,
+            "D": w0.D, "page_size": 16, "budget_tokens": w0.budget, "storage_dtype": "bf16",
+            "present_pages": bytes_l[0]["present_pages"], "selected_pages": bytes_l[0]["selected_pages"],
+            "h2o_epilogue": h2o, "cuda_graph": use_graph, "dense_layers": dense,
+            "l2": {"stream": "inputs larger than L2 (%.0f MB touched per step)" % (total_bytes / 1e6),
+                   "rotate": "%d independent instances in turn (%.0f MB per step, %.0f MB before an instance is touched "
+                             "again), %d steps chained per graph replay" % (len(instances), total_bytes / 1e6,
+                                                                             len(instances) * total_bytes / 1e6, chain),
+                   "flush": "flushed before every step: a %d MiB write, then a %d MiB read (leaves clean lines); the "
+                            "step then pays its launch latency inside the timed region" % (2 * L2_BYTES >> 20, 2 * L2_BYTES >> 20)}[mode],
+            "protocol": "1 discarded run, %d window(s) of 32 untimed + %s timed replays" % (len(windows), "/".join(str(int(round(K / len(windows)))) for _ in windows)),
+            "parallelism": "1 GPU" if world == 1 else "%d replicas, no collective" % world,
+            "global_batch": w0.B * world,
+        },
+        "algorithmic_bytes_per_step": total_bytes,
+        "achieved_gbs": step_gbs * world,
+        "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+        "frac_of_measured_copy": step_gbs / peak,
+        "launches_per_step": sum(binding.se_decode_step_launches(st.p, 16 * st.w.max_pages if l < dense else st.w.budget, h2o)
+                                 for l, st in enumerate(states)),
+        "clocks": clocks,
+    }
+    # warm L2 (same instance back to back) where the step fits in L2, and the flush-based latency of one step
+    if mode != "stream":
+        warm = chained_graph([inst0] * 8) if use_graph else inst0.run
+        per = 8 if use_graph else 1
+        for _ in range(5):
+            warm()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = max(5, min(K, 200) // per)
+        a.record()
+        for _ in range(n):
+            warm()
+        b.record()
+        torch.cuda.synchronize()
+        rec["l2_warm_us"] = a.elapsed_time(b) / (n * per) * 1e3
+        del warm
+        fl = flusher or Flusher(dev)
+        tot = 0.0
+        n = 30
+        for _ in range(n):
+            fl()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); inst0.run(); b.record()
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        rec["single_step_after_flush_us"] = tot / n * 1e3
+        del fl
 
-    # ---- per-call timing (same stream, CUDA events, each call in its own loop)
+    # ---- end to end
+    e2e = E2E(inst0, dev, use_graph)
+    for _ in range(3):
+        e2e.step()
+    e2e_iters = max(10, min(K, 200 if n_layers == 1 else 30))
+    others = [E2E(i, dev, use_graph) for i in instances[1:]] if mode == "rotate" else []
+    ring = [e2e] + others
+    barrier()
+    tot_ms = 0.0
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if flusher is None:
+        a.record()
+        for i in range(e2e_iters):
+            ring[i % len(ring)].step()
+        b.record()
+        barrier()
+        tot_ms = a.elapsed_time(b)
+    else:
+        for i in range(e2e_iters):
+            flusher()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); e2e.step(); b.record()
+            torch.cuda.synchronize()
+            tot_ms += a.elapsed_time(b)
+    e2e_ms = tot_ms / e2e_iters
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    rec["e2e"] = {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": e2e.h2d, "d2h_bytes_per_step": e2e.d2h,
+                  "what": "pinned q (+ lengths and the changed page-table entries) up, step, out + lse down into pinned "
+                          "memory, host sync; copies of consecutive layers overlap the steps"}
+    del others, ring
+    sampler.stop()
+
+    if full:
+        rec.update(per_call_and_rooflines(binding, inst0, dev, bytes_l[0], flusher if mode == "flush" else None, K, peak, peak_kind))
+        rec["config"]["checksums_layer0"] = checksums(w0)
+    rec["_inst0"] = inst0
+    return rec
+
+
+def per_call_and_rooflines(binding, inst, dev, b0, flusher, K, peak, peak_kind):
+    """Every entry point timed on its own (same stream, CUDA events, each call in its own loop) and the
+    roofline record of the two streaming kernels."""
+    st0, u0 = inst.states[0], inst.accums[0]
+    w0 = inst.layers[0]
+
     def time_call(fn, iters):
         for _ in range(3):
             fn()
-        if flush:
+        if flusher is not None:
             tot = 0.0
             for i in range(iters):
-                flush_l2(i)
+                flusher()
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(); fn(); b.record()
                 torch.cuda.synchronize()
@@ -368,158 +667,147 @@ def main():
         return a.elapsed_time(b) / iters * 1e3
 
     iters = max(10, min(K, 200))
-    st0, u0 = states[0], accums[0]
     call_us = {
         "se_meta_update": time_call(st0.update_meta, iters),
         "se_page_select": time_call(st0.select, iters),
         "se_page_select_scores": time_call(lambda: st0.select(entry="se_page_select_scores"), iters),
         "se_page_select_topk": time_call(lambda: st0.select(entry="se_page_select_topk"), iters),
         "se_page_select_fused": time_call(st0.select_fused, iters),
-        "se_decode_step": time_call(lambda: st0.step(u0), iters),
         "se_sparse_decode": time_call(lambda: st0.decode(u0), iters),
         "se_sparse_decode_splits": time_call(lambda: st0.decode(u0, entry="se_sparse_decode_splits"), iters),
         "se_combine": time_call(lambda: st0.decode(u0, entry="se_combine"), iters),
+        "se_decode_step": time_call(lambda: st0.step(u0), iters),
     }
-    b0 = bytes_l[0]
-    peak, peak_kind = measured_peak()
-    # the dominant kernel, timed on its own: decode_kernel is all that se_sparse_decode_splits launches
+    ceil = gather_ceilings(binding, inst, dev)
+    c_meta = next(v for k, v in ceil.items() if k.startswith("summaries"))
+    c_kv = next(v for k, v in ceil.items() if k.startswith("pages"))
     dec_gbs = b0["decode_kernel"] / (call_us["se_sparse_decode_splits"] * 1e-6) / 1e9
-    sel_gbs = b0["select_call"] / (call_us["se_page_select"] * 1e-6) / 1e9
     score_gbs = b0["select_call"] / (call_us["se_page_select_scores"] * 1e-6) / 1e9
-    rl_decode = {"bound": "hbm", "kernel": "decode_kernel (se_sparse_decode_splits)", "achieved": dec_gbs,
+    rl_decode = {"bound": "hbm", "kernel": "attention kernel (se_sparse_decode_splits)", "achieved": dec_gbs,
                  "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": dec_gbs / peak,
-                 "traffic": NCU_TRAFFIC_BYTES.get(layers[0].name), "algorithmic_bytes": b0["decode_kernel"],
-                 "us": call_us["se_sparse_decode_splits"]}
+                 "traffic": NCU_TRAFFIC_BYTES.get(w0.name), "algorithmic_bytes": b0["decode_kernel"],
+                 "us": call_us["se_sparse_decode_splits"], "gather_ceiling_gbs": c_kv["gbs"],
+                 "frac_of_gather_ceiling": dec_gbs / c_kv["gbs"]}
     rl_score = {"bound": "hbm", "kernel": "score_kernel (se_page_select_scores)", "achieved": score_gbs,
                 "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": score_gbs / peak,
-                "traffic": NCU_TRAFFIC_BYTES_SCORE.get(layers[0].name), "algorithmic_bytes": b0["select_call"],
-                "us": call_us["se_page_select_scores"]}
+                "traffic": NCU_TRAFFIC_BYTES_SCORE.get(w0.name), "algorithmic_bytes": b0["select_call"],
+                "us": call_us["se_page_select_scores"], "gather_ceiling_gbs": c_meta["gbs"],
+                "frac_of_gather_ceiling": score_gbs / c_meta["gbs"]}
     # the dominant kernel is whichever of the two streaming kernels takes longer on this workload
     rl_main, rl_other = (rl_score, rl_decode) if rl_score["us"] >= rl_decode["us"] else (rl_decode, rl_score)
-    step_gbs = total_bytes / (ms_per_step * 1e-3) / 1e9
+    return {"calls_us": call_us, "roofline": rl_main, "roofline_second_kernel": rl_other, "gather_ceiling": ceil}
 
-    # ---- end to end through the public API with host buffers: the step's inputs (q, lengths, page
-    # table) sit in one pinned block and go up in one copy, out + lse come back in one copy
-    import copy
 
-    def packed(tensors, device, pin):
-        """One byte block holding the tensors back to back (16-byte aligned); returns (block, views)."""
-        offs, total = [], 0
-        for t in tensors:
-            offs.append(total)
-            total += (t.numel() * t.element_size() + 15) // 16 * 16
-        block = torch.empty(total, dtype=torch.uint8, device=device)
-        if pin:
-            block = block.pin_memory()
-        views = [block[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for o, t in zip(offs, tensors)]
-        return block, views
+def spawn_ranks(args):
+    """bench.py --gpus N without a rank environment: start the N ranks ourselves, one per GPU."""
+    port = 29500 + (os.getpid() % 2000)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
 
-    e2e_states, host_in, dev_in, host_out, dev_out = [], [], [], [], []
-    for w, st in zip(layers, states):
-        ins = [w.q, w.seq_lens, w.page_table]
-        hb, hv = packed(ins, "cpu", True)
-        db, dv = packed(ins, dev, False)
-        for src, h, d in zip(ins, hv, dv):
-            h.copy_(src)
-            d.copy_(src)
-        outs = [st.out, st.lse]
-        ob, ov = packed(outs, dev, False)
-        hob, _ = packed(outs, "cpu", True)
-        st2 = copy.copy(st)                       # same params, workspace, summaries and selection buffers
-        st2.w = dataclasses.replace(w, q=dv[0], seq_lens=dv[1], page_table=dv[2])
-        st2.out, st2.lse = ov
-        e2e_states.append(st2)
-        host_in.append(hb); dev_in.append(db); host_out.append(hob); dev_out.append(ob)
-    h2d = sum(b.numel() for b in host_in)
-    d2h = sum(b.numel() for b in host_out)
 
-    def e2e_body():
-        for st2, u, hb, db, ob, hob in zip(e2e_states, accums, host_in, dev_in, dev_out, host_out):
-            db.copy_(hb, non_blocking=True)
-            st2.step(score_accum=u)
-            hob.copy_(ob, non_blocking=True)
+# ------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=768, help="timed steps (default 768 = 3 windows of 256)")
+    ap.add_argument("--warmup", type=int, default=32)
+    ap.add_argument("--config", type=int, default=3, choices=sorted(wl.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="layers per step (default 1; 28 for config 5)")
+    ap.add_argument("--dense-layers", type=int, default=0,
+                    help="the first this many layers attend every page (budget >= context), the others select under "
+                         "the budget (the paper's per-layer policy); all in the same graph")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the number of requests (configs 3-5; for small profiling captures)")
+    ap.add_argument("--no-graph", action="store_true", help="launch the calls directly instead of a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the short runs of the other configs")
+    ap.add_argument("--workload", default="decode", choices=["decode", "h2o_evict", "omnikv_reuse"],
+                    help="decode = the sparse decode step (the headline); h2o_evict = one H2O eviction "
+                         "(retained set + in-place compaction) of 64 requests, 5120 -> 4096 tokens; "
+                         "omnikv_reuse = one observation layer (full attention + token selection) and four "
+                         "sparse layers reusing its 2048+32 tokens, 24 requests of 32768 tokens")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
 
-    # the way a serving loop drives the library: the host fills fixed pinned buffers, one graph launch
-    # does upload + step + download, and the host waits for the result before the next step
-    e2e_graph = None
-    if not args.no_graph:
-        s2 = torch.cuda.Stream()
-        s2.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(s2):
-            e2e_body()
-        torch.cuda.current_stream().wait_stream(s2)
-        torch.cuda.synchronize()
-        e2e_graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(e2e_graph):
-            e2e_body()
+    if args.gpus > 1 and "RANK" not in os.environ and args.impl == "ours" and args.workload == "decode":
+        spawn_ranks(args)
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
 
-    def e2e_step():
-        if e2e_graph is not None:
-            e2e_graph.replay()
-        else:
-            e2e_body()
-        torch.cuda.synchronize()
+    if args.workload in ("h2o_evict", "omnikv_reuse"):
+        if rank == 0:                        # these steps have no multi-GPU leg of their own
+            (run_h2o_evict if args.workload == "h2o_evict" else run_omnikv)(args, local_rank)
+        return
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return
 
-    for _ in range(3):
-        e2e_step()
-    e2e_iters = max(10, min(K, 200))
-    barrier()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for i in range(e2e_iters):
-        if flush:
-            flush_l2(i)
-        e2e_step()
-    b.record()
-    barrier()
-    e2e_ms = a.elapsed_time(b) / e2e_iters
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
     if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    sampler.stop()
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2609_39068_b200 import binding
+    binding.load()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    K = args.steps
+    rec = run_config(binding, args.config, dev, args, rank, world, barrier, True, K)
+    inst0 = rec.pop("_inst0")
+    n_layers = rec["config"]["layers"]
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = oracle_time(layers[0])
-        if n_layers > 1:
-            cpu_baseline["value"] *= n_layers
-            cpu_baseline["sample"] += "; one layer timed, x%d layers" % n_layers
+        sec, runs, cores = oracle_step_time(inst0.layers[0], wl.bf16_bits(inst0.states[0].meta))
+        cpu_baseline = dict(value=sec * n_layers * 1e6, unit="us", cores=cores, kind="oracle",
+                            sample="the whole batch (%d requests) of layer 0, fp64 C oracle with OpenMP over (request, "
+                                   "kv-head), best of %d runs = %.1f ms%s" % (inst0.layers[0].B, runs, sec * 1e3,
+                                   "; x%d layers" % n_layers if n_layers > 1 else ""),
+                            sample_seconds=sec)
+    del inst0
+    torch.cuda.empty_cache()
+
+    other = None
+    if rank == 0 and world == 1 and not args.no_other_configs and not args.batch:
+        other = {}
+        for c in sorted(wl.CONFIGS):
+            if c == args.config:
+                continue
+            r = run_config(binding, c, dev, args, rank, world, barrier, False, 96 if c != 5 else 12)
+            i0 = r.pop("_inst0")
+            if c in (1, 2) and not args.no_cpu_baseline:
+                meta_bits = wl.bf16_bits(i0.states[0].meta)
+                sec, runs, cores = oracle_step_time(i0.layers[0], meta_bits, budget_s=3.0)
+                sec1, runs1, _ = oracle_step_time(i0.layers[0], meta_bits, threads=1, budget_s=3.0)
+                r["cpu_baseline"] = {"value": sec * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+                                     "one_thread_us": sec1 * 1e6, "sample": "whole batch, best of %d / %d runs" % (runs, runs1)}
+            other["config%d" % c] = r
+            del i0
+            torch.cuda.empty_cache()
 
     if rank == 0:
-        # score, top-k, decode (summary update fused into score); the merge kernel runs only when
-        # the pairs are split or the H2O epilogue is on
-        launches_per_step = n_layers * binding.se_decode_step_launches(states[0].p, layers[0].budget, h2o)
         line = {
-            "metric": METRIC, "value": ms_per_step * 1e3, "unit": "us", "n_gpus": world,
-            "steps": K, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "metric": METRIC, "value": rec["value"], "unit": "us", "n_gpus": world,
+            "steps": K, "warmup": args.warmup, "ms_per_step": rec["value"] / 1e3,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {
-                "workload": layers[0].name, "config_id": args.config, "layers": n_layers,
-                "B": layers[0].B, "H_q": layers[0].H_q, "H_kv": layers[0].H_kv, "D": layers[0].D,
-                "page_size": 16, "budget_tokens": layers[0].budget, "storage_dtype": "bf16",
-                "present_pages": b0["present_pages"], "selected_pages": b0["selected_pages"],
-                "h2o_epilogue": h2o, "cuda_graph": graph is not None,
-                "l2": ("flushed before every step: a %d MiB write, then a %d MiB read (leaves clean lines)" % (2 * L2_BYTES >> 20, 2 * L2_BYTES >> 20)) if flush
-                      else "inputs larger than L2 (%.0f MB touched per step)" % (working_set / 1e6),
-                "parallelism": "1 GPU" if world == 1 else "%d replicas, no collective" % world,
-                "global_batch": layers[0].B * world,
-                "checksums_layer0": checksums(layers[0]),
-            },
-            "algorithmic_bytes_per_step": total_bytes,
-            "achieved_gbs": step_gbs * world,
-            "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
-            "frac_of_measured_copy": step_gbs / peak,
-            "calls_us": call_us,
-            "calls_gbs": {"se_page_select": sel_gbs, "se_sparse_decode": dec_gbs},
-            "roofline": rl_main,
-            "roofline_second_kernel": rl_other,
-            "clocks": clocks,
-            "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": launches_per_step * K,
-            "cpu_baseline": cpu_baseline,
         }
+        line.update({k: v for k, v in rec.items() if k not in ("value", "unit", "steps")})
+        line["gpu_launches"] = rec["launches_per_step"] * K
+        line["cpu_baseline"] = cpu_baseline
+        if other is not None:
+            line["other_configs"] = other
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
@@ -797,44 +1085,47 @@ def run_omnikv(args, local_rank):
         "cpu_baseline": cb}))
 
 
-def run_reference(args, n_layers):
-    """Reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload."""
+def run_reference(args):
+    """Reference arm: the CPU oracle, as it stands, on the host cores, on the whole batch of the config
+    (one layer; a multi-layer config is that time x layers).  Without a GPU to generate the pool on, a
+    reduced batch is generated on the CPU and scaled by the page count (said in the sample string)."""
     import oracle
-    dev = "cuda" if torch.cuda.is_available() else "cpu"
-    if dev == "cpu" and args.config in (3, 4, 5):
+    n_layers = args.layers or (28 if args.config == 5 else 1)
+    scale, note = 1.0, "whole batch, generated on the GPU and copied to the host"
+    if torch.cuda.is_available():
+        w = wl.CONFIGS[args.config]("cuda")
+        w_cpu = w.to("cpu")
+        del w
+        torch.cuda.empty_cache()
+    elif args.config in (3, 4, 5):
         kw = {3: dict(B=4), 4: dict(B=1, length=32768), 5: dict(B=8)}[args.config]
-        w = wl.CONFIGS[args.config](dev, **kw)
-        # no GPU to generate the full pool on: a sixteenth of the workload, scaled back up
-        reduced = 16.0
-        note = "generated on the CPU at reduced size (%s), then x%.0f to the full workload" % (kw, reduced)
+        w_cpu = wl.CONFIGS[args.config]("cpu", **kw)
+        scale, note = 16.0, "no GPU: reduced batch generated on the CPU (%s), x16 to the full workload" % (kw,)
     else:
-        w = wl.CONFIGS[args.config](dev)
-        reduced = 1.0
-        note = "full workload generated on the GPU, sample copied to the host"
-    order = list(range(0, w.B, max(1, w.B // 16)))[:16]
-    sub = wl.sub_workload(w, order, "cpu")
-    q, k, v = wl.bf16_bits(sub.q), wl.bf16_bits(sub.k_cache), wl.bf16_bits(sub.v_cache)
-    pt, sl = sub.page_table.numpy(), sub.seq_lens.numpy()
-    meta = oracle.quest_meta(k, pt, sl, first_tok=np.zeros(sub.B, np.int32))
-    u = None if sub.score_accum is None else sub.score_accum.numpy().astype(np.float64)
-    n_all = (w.seq_lens.cpu().numpy() + 15) // 16
-    scale = float(n_all.sum()) / float(((sl + 15) // 16).sum()) * n_layers * reduced
+        w_cpu = wl.CONFIGS[args.config]("cpu")
+        note = "whole batch, generated on the CPU"
+    q, k, v = wl.bf16_bits(w_cpu.q), wl.bf16_bits(w_cpu.k_cache), wl.bf16_bits(w_cpu.v_cache)
+    pt, sl = w_cpu.page_table.numpy(), w_cpu.seq_lens.numpy()
+    meta = oracle.quest_meta(k, pt, sl, first_tok=np.zeros(w_cpu.B, np.int32))     # set-up: summaries after prefill
+    u = None if w_cpu.score_accum is None else w_cpu.score_accum.numpy().astype(np.float64)
     steps = max(1, min(args.steps, 20))
     warm = max(1, min(args.warmup, 3))
     for _ in range(warm):
-        oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
+        oracle.decode_step(q, k, v, pt, sl, w_cpu.budget, meta=meta, u_accum=None if u is None else u.copy())
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle.decode_step(q, k, v, pt, sl, sub.budget, meta=meta, u_accum=u)
+        oracle.decode_step(q, k, v, pt, sl, w_cpu.budget, meta=meta, u_accum=None if u is None else u.copy())
     per = (time.perf_counter() - t0) / steps
-    val = per * scale * 1e6
-    sample = ("%d of %d requests per step (%s), %.1f ms per sample step, scaled x%.2f by page count%s"
-              % (sub.B, w.B, note, per * 1e3, scale, " and layers" if n_layers > 1 else ""))
+    val = per * scale * n_layers * 1e6
+    sample = "%d requests per step (%s), %.1f ms per oracle step%s" % (
+        w_cpu.B, note, per * 1e3, "; one layer timed, x%d layers" % n_layers if n_layers > 1 else "")
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": "us", "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": val / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "config_id": args.config, "layers": n_layers},
+        "config": {"workload": w_cpu.name, "config_id": args.config, "layers": n_layers, "B": w_cpu.B,
+                   "H_q": w_cpu.H_q, "H_kv": w_cpu.H_kv, "D": w_cpu.D, "page_size": 16,
+                   "budget_tokens": w_cpu.budget, "storage_dtype": "bf16"},
         "cpu_baseline": {"value": val, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

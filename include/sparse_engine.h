@@ -207,20 +207,23 @@ int se_sparse_decode(const se_params *p, const void *q, const void *k_cache,
 /*
  * One decode step of a layer in one call: se_meta_update(first_tok = NULL), se_page_select and
  * se_sparse_decode, with the same results (meta, sel_idx, sel_cnt, out, lse, score_accum; Appendix A,
- * Quest summary and score equations, TopK, selected-attention and H2O equations).  The call picks
- * the launch plan from the shape alone:
- *   - budget_tokens/16 < max_pages (a sparse layer): the scoring kernel (which also refreshes the
- *     summary of each request's newest page) leaves the fp32 page scores in the workspace, and the
- *     attention kernel selects each pair's pages from them in its prologue - no top-k kernel, no
- *     round trip of the selection through memory before the first page is fetched.  With at most one
- *     (request, kv-head) pair per SM the attention kernel also merges its split partials itself, so
- *     the step is two launches (three with score_accum, whose epilogue needs the final lse).
- *     Shapes the in-kernel top-k does not cover (more than 4096 pages per request together with
- *     more than one pair per SM) run the top-k kernel in between.
- *   - budget_tokens/16 >= max_pages and k_max >= max_pages (a dense layer, e.g. the first layers of
+ * Quest summary and score equations, TopK, selected-attention and H2O equations; the fused per-pair
+ * form follows Appendix B's requirement that a step replays as a fixed sequence of launches over
+ * stable buffers).  The call picks the launch plan from the shape alone:
+ *   - a sparse layer (budget_tokens/16 < max_pages) with at most one (request, kv-head) pair per SM
+ *     and at most 8 CTAs per pair: ONE kernel.  The CTAs of a pair form a thread-block cluster; each
+ *     scores its share of the pair's pages (refreshing the summary of the request's newest page),
+ *     after a cluster barrier every CTA selects the pair's pages from the score row (top-k in shared
+ *     memory), attends its share of them with eight warps, merges the warps' partials through shared
+ *     memory, and the CTA that arrives last merges the CTAs' partials and applies the H2O update.
+ *   - a sparse layer with more pairs: the scoring kernel, the top-k kernel, the attention kernel
+ *     (one warp per pair or per split of a pair), and the merge kernel where pairs are split or
+ *     score_accum is given.
+ *   - a dense layer (budget_tokens/16 >= max_pages and k_max >= max_pages, e.g. the first layers of
  *     a model whose remaining layers are sparse): summary update, list of all present pages,
  *     attention.
- * sel_idx / sel_cnt are outputs here.  se_decode_step_launches tells how many kernels a step
+ * sel_idx / sel_cnt are outputs here; the fp32 page scores are left in the workspace as
+ * se_page_select_scores leaves them.  se_decode_step_launches tells how many kernels a step
  * launches for `p` (host, pure; 0 if the arguments are invalid).
  */
 int se_decode_step(const se_params *p, const void *q, const void *k_cache, const void *v_cache, void *meta,
@@ -369,6 +372,22 @@ int se_h2o_retain(const se_params *p, const float *score_accum, const int32_t *p
 int se_h2o_compact(const se_params *p, void *k_cache, void *v_cache, float *score_accum,
                    const int32_t *page_table, const int32_t *keep_idx, const int32_t *keep_cnt,
                    int32_t budget_tokens, int32_t *new_seq_lens, void *workspace, void *stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): a read-only gather with the access pattern and
+ * pipeline shape of the library's kernels and no arithmetic, to find what the memory system of a
+ * given GPU allows for that pattern.  Piece i of the list lives at base + piece_idx[i]*piece_bytes
+ * (with base1 != NULL the odd lanes of a batch read from base1 instead: K and V pages of the same
+ * list).  Every warp of a persistent grid (148 * ctas_per_sm CTAs of warps_per_cta warps) keeps
+ * stages_per_warp batches of pieces_per_stage (<= 32) pieces in flight in shared memory, fetched by
+ * bulk asynchronous copies.  piece_bytes is a multiple of 16; the shared memory needed
+ * (warps * stages * pieces * piece_bytes) must fit 227 KB.  All pointers are DEVICE pointers, 16-byte
+ * aligned; the call is asynchronous on `stream`.  Shapes used by the benchmark: summaries 512 B x 16 x 2
+ * stages x 4 warps x 3 CTAs/SM; pages 4096 B x 2 x 5 x 4 x 1; token rows 256 B x 32 x 5 x 4 x 1.
+ */
+int se_probe_gather(const void *base0, const void *base1, const int32_t *piece_idx, int64_t n_pieces,
+                    int32_t piece_bytes, int32_t pieces_per_stage, int32_t stages_per_warp,
+                    int32_t warps_per_cta, int32_t ctas_per_sm, void *stream);
 
 /*
  * Copies the device status word (an OR of SE_DEV_* bits, 0 = clean) to *host_out and

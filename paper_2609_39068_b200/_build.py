@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libsparse_engine.so")
-SOURCES = ["se_api.cu", "se_meta.cu", "se_select.cu", "se_decode.cu", "se_h2o.cu"]
+SOURCES = ["se_api.cu", "se_meta.cu", "se_select.cu", "se_decode.cu", "se_h2o.cu", "se_probe.cu"]
 HEADERS = ["se_device.cuh", "se_internal.h", "se_topk.cuh", os.path.join("..", "..", "include", "sparse_engine.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]

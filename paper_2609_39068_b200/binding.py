@@ -25,7 +25,7 @@ EXPORTS = ("se_version", "se_strerror", "se_workspace_bytes", "se_decode_num_spl
            "se_page_select", "se_page_select_scores", "se_page_select_topk", "se_page_select_fused", "se_sparse_decode", "se_sparse_decode_splits", "se_combine",
            "se_last_device_status", "se_h2o_retain", "se_h2o_compact", "se_observe_decode", "se_token_select",
            "se_token_decode",
-           "se_page_select_static", "se_decode_step", "se_decode_step_launches")
+           "se_page_select_static", "se_decode_step", "se_decode_step_launches", "se_probe_gather")
 SE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -84,6 +84,9 @@ def load(build_if_missing: bool = True):
     lib.se_page_select_static.argtypes = [pp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, i32p, vp]
     lib.se_decode_step.argtypes = [pp, vp, vp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, i32p, fp, fp, fp, vp, vp]
     lib.se_decode_step_launches.argtypes = [pp, ctypes.c_int32, ctypes.c_int]
+    lib.se_probe_gather.argtypes = [vp, vp, i32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                    ctypes.c_int32, ctypes.c_int32, vp]
+    lib.se_probe_gather.restype = ctypes.c_int
     for name in ("se_workspace_init", "se_meta_update", "se_page_select", "se_page_select_fused",
                  "se_sparse_decode", "se_sparse_decode_splits", "se_combine", "se_last_device_status",
                  "se_h2o_retain", "se_h2o_compact", "se_decode_num_splits", "se_page_select_static",
@@ -233,6 +236,22 @@ def se_decode_step(p, q, k_cache, v_cache, meta, page_table, seq_lens, budget_to
 
 def se_decode_step_launches(p: SeParams, budget_tokens: int, with_score_accum: bool) -> int:
     return int(load().se_decode_step_launches(ctypes.byref(p), int(budget_tokens), int(bool(with_score_accum))))
+
+
+def se_probe_gather(base0, piece_idx, piece_bytes, pieces_per_stage, stages_per_warp, warps_per_cta, ctas_per_sm,
+                    base1=None) -> None:
+    """Read-only gather of the pieces ``piece_idx`` (int32 CUDA tensor) of ``base0`` (any CUDA tensor; odd
+    lanes read ``base1`` when given) with the given pipeline shape; see the header."""
+    for t in (base0, base1, piece_idx):
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise SparseEngineError("se_probe_gather needs contiguous CUDA tensors")
+    if piece_idx.dtype != torch.int32:
+        raise SparseEngineError("piece_idx must be int32")
+    _check(load().se_probe_gather(ctypes.c_void_p(base0.data_ptr()),
+                                  None if base1 is None else ctypes.c_void_p(base1.data_ptr()),
+                                  ctypes.c_void_p(piece_idx.data_ptr()), int(piece_idx.numel()), int(piece_bytes),
+                                  int(pieces_per_stage), int(stages_per_warp), int(warps_per_cta), int(ctas_per_sm),
+                                  _stream()), "se_probe_gather")
 
 
 def se_page_select_static(p, q, meta, page_table, seq_lens, budget_tokens, sel_idx, sel_cnt,

@@ -49,8 +49,8 @@ int decode_warps_per_cta();
 
 // Launch geometry of the attention step, from the shape alone.
 //  - at most one pair per SM: CTA units.  A pair gets cpp = min(SMs / pairs, ceil(k_max / 8)) CTAs (a
-//    warp should hold at least one page); up to kMergeInKernelMax of them are merged by the
-//    last-arriving CTA, more by the merge kernel.
+//    warp should hold at least one page); up to 8 of them form a thread-block cluster and merge
+//    their partials themselves, more are merged by the merge kernel.
 //  - fewer than two pairs per SM: warp units, every pair cut into as many splits as the persistent
 //    warps of the grid can take in one round; the merge kernel combines them.
 //  - two or more pairs per SM: warp units, one per pair (a few warps per SM, each with a deep copy
@@ -301,7 +301,9 @@ int se_decode_step_launches(const se_params *p, int32_t budget_tokens, int with_
     const int plan = step_plan(*p, budget_tokens / kPage);
     const DecodePlan dp = make_decode_plan(*p);
     const bool merged = dp.max_splits == 1 || (dp.cta_units && dp.merge_in_kernel);
-    const int attention = 1 + ((!merged || with_score_accum) ? 1 : 0);
+    // CTA units with the in-kernel merge also run the H2O epilogue in the kernel
+    const bool second = (dp.cta_units && dp.merge_in_kernel) ? false : (!merged || with_score_accum);
+    const int attention = 1 + (second ? 1 : 0);
     return (plan == 3 ? 0 : plan == 1 ? 1 : 2) + attention;
 }
 

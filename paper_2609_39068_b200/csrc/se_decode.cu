@@ -9,9 +9,10 @@
 //                    a pair is one unit and its warp writes out/lse itself, otherwise the pair is cut
 //                    into splits whose partials (acc, m, l) combine_kernel merges.
 // decode_cta_kernel  at most one pair per SM.  A CTA is one (pair, CTA-split); its eight warps share
-//                    the CTA's pages, their partials are merged through shared memory, and when a
-//                    pair has several CTAs the last one to arrive (an atomic ticket: nobody waits)
-//                    merges the CTAs' partials - no merge kernel, no partials of single warps.
+//                    the CTA's pages and their partials are merged through shared memory.  The CTAs
+//                    of a pair (up to 8) form a thread-block cluster: after a cluster barrier each
+//                    of them merges a share of the CTAs' partials and applies the H2O update to the
+//                    tokens it attended - no merge kernel, no partials of single warps.
 //
 // decode_cta_kernel can take the selection from the page scores themselves (kSelect): the CTA runs
 // the top-k in its prologue (se_topk.cuh: cta_topk), while the shared-memory ring is still empty and
@@ -45,7 +46,6 @@ constexpr int kChunk = 128;              // selected pages looked up at once
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileBytes = kPage * 128;  // one TMA box: 16 rows x 64 bf16
-constexpr int kMergeInKernelMax = 8;     // CTA-splits per pair the last-arriving CTA merges itself
 
 template <int D>
 struct DecCfg {
@@ -704,9 +704,10 @@ __device__ __forceinline__ bool cta_score_range(uint8_t *wbuf, uint32_t bar0, in
 //   2. the cnt selected pages are cut into n_active = ceil(cnt / ceil(cnt / cpp)) equal CTA slices, a
 //      slice into eight warp ranges; each warp attends its range (attend_range);
 //   3. the warps' partials are merged through shared memory (weights 2^(m_w - m*));
-//   4. one active CTA: out / lse are final.  Several: the CTA stores its partial and takes a ticket
-//      (atomic counter per pair, zero between launches); with merge_here the CTA holding the last
-//      ticket merges all of them, otherwise combine_kernel does.
+//   4. one active CTA: out / lse are final.  Several: every CTA stores its partial; with merge_here (the
+//      CTAs are a cluster) they meet at a cluster barrier, after which each computes the pair's final
+//      log-sum-exp, its share of the final output and the H2O update of its own tokens; without it
+//      combine_kernel merges the partials.
 // ---------------------------------------------------------------------------------
 template <int D>
 struct CtaCfg {
@@ -717,8 +718,8 @@ struct CtaCfg {
     static constexpr size_t kBars = kStages;
     static constexpr size_t kLists = kBars + (size_t)kDecWarps * C::MAXST * 8;
     static constexpr size_t kZero = kLists + (size_t)kDecWarps * 3 * kChunk * sizeof(int);
-    static constexpr size_t kSmall = kZero + 16;               // merge statistics: 4 * 64 floats + flags
-    static constexpr size_t kSel = kSmall + 4 * 64 * sizeof(float) + 64;
+    static constexpr size_t kSmall = kZero + 16;               // merge statistics: 4 * 64 floats
+    static constexpr size_t kSel = kSmall + 4 * 64 * sizeof(float);
     static_assert(sizeof(TopkScratch) + cta_topk_key_words(8192, kDecWarps * 32) * 4 <= kStages,
                   "the top-k keys and scratch live in the empty ring");
     static_assert((size_t)kDecWarps * 8 * RED_PITCH * sizeof(float) <= kStages, "merge buffer lives in the drained ring");
@@ -732,9 +733,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
 decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                   const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
                   const int32_t *__restrict__ seq_lens, const SelectArgs sa, const FusedScoreArgs fs,
-                  float *__restrict__ out, float *__restrict__ lse, float *partials, float *__restrict__ zbuf,
-                  int H_kv, int G, int GP, int max_pages, int P_phys, int k_max, int cpp, int merge_here,
-                  float scale_log2, uint32_t *status, uint32_t *ticket) {
+                  float *__restrict__ out, float *__restrict__ lse, float *partials, float *zbuf,
+                  float *__restrict__ score_accum, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max,
+                  int cpp, int merge_here, float scale_log2, uint32_t *status) {
     using C = DecCfg<D>;
     using L = CtaCfg<D>;
     extern __shared__ uint8_t smem_dyn[];
@@ -772,7 +773,6 @@ decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     float *s_l = s_m + 64;                                            // [warp][head]
     float *s_M = s_l + 64;                                            // [head] merged maximum
     float *s_L = s_M + 64;                                            // [head] merged sum
-    int *s_flag = reinterpret_cast<int *>(s_L + 64);
     int *list = reinterpret_cast<int *>(smem_al + L::kSel);
 
     const int len = __ldg(seq_lens + r);
@@ -822,134 +822,160 @@ decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     }
     const int per_cta = (cnt + cpp - 1) / cpp;
     const int n_active = (cnt + per_cta - 1) / per_cta;
-    if (cs >= n_active) return;
-    const int c_lo = cs * per_cta, c_hi = min(cnt, c_lo + per_cta);
-    const int per_warp = (c_hi - c_lo + kDecWarps - 1) / kDecWarps;
-    const int i_lo = min(c_hi, c_lo + warp * per_warp), i_hi = min(c_hi, i_lo + per_warp);
-
-    AttendArgs a;
-    a.k_map = &k_map;
-    a.v_map = &v_map;
-    a.page_table = page_table;
-    a.max_pages = max_pages;
-    a.H_kv = H_kv;
-    a.P_phys = P_phys;
-    a.G = G;
-    a.GP = GP;
-    a.scale_log2 = scale_log2;
-    a.zero_chunk = smem_u32(smem_al + L::kZero);
-    a.status = status;
-    a.zrow = zbuf != nullptr ? zbuf + (size_t)pair * k_max * kPage * GP : nullptr;
-    a.keys_row = nullptr;
-
-    WarpAttn<D> A;
-    A.init_lane(lane);
-    A.reset();
-    bool ok = true;
-    if (i_lo < i_hi) {
-        A.load_q(q, head0, lane, G);
-        const int none[kChunk / 32] = {};
-        ok = attend_range<D, false, false>(P, A, a, [&](int i) { return list[i]; }, none, i_lo, i_hi, r, h, len, n_r,
-                                           lane);
-    }
-    if (!ok) {
-        if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
-        for (int s = 0; s < P.nstage; ++s) mbar_wait(P.bar0 + s * 8, (P.phases >> s) & 1u);
-    }
-    A.finish();
-
-    // ---- merge of the eight warps through shared memory.  Rows past the group hold zero queries:
-    // finite values that nobody reads.
-    if (tid4 == 0) {
-        s_m[warp * 8 + gid] = A.m_run;
-        s_l[warp * 8 + gid] = A.l_run;
-    }
-    __syncthreads();                  // every warp has drained its ring: it becomes the merge buffer
-    float mstar = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kDecWarps; ++w) mstar = fmaxf(mstar, s_m[w * 8 + gid]);
-    float lsum = 0.f;
-#pragma unroll
-    for (int w = 0; w < kDecWarps; ++w) {
-        const float mw = s_m[w * 8 + gid];
-        lsum += (mw == -INFINITY) ? 0.f : exp2f(mw - mstar) * s_l[w * 8 + gid];
-    }
-    const float wgt = (A.m_run == -INFINITY) ? 0.f : exp2f(A.m_run - mstar);
-    float *red = reinterpret_cast<float *>(smem_al);
-    {
-        float *dst = red + (size_t)(warp * 8 + gid) * L::RED_PITCH + 2 * tid4;
-#pragma unroll
-        for (int nt = 0; nt < C::NTILES; ++nt)
-            *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(A.o_acc[nt][0] * wgt, A.o_acc[nt][1] * wgt);
-    }
-    if (warp == 0 && tid4 == 0) {
-        s_M[gid] = mstar;
-        s_L[gid] = lsum;
-    }
-    __syncthreads();
     const bool single = n_active == 1;
-    for (int e = tid; e < G * D; e += kDecWarps * 32) {
-        const int g = e / D, c = e - g * D;
-        float acc = 0.f;
-#pragma unroll
-        for (int w = 0; w < kDecWarps; ++w) acc += red[(size_t)(w * 8 + g) * L::RED_PITCH + c];
-        if (single) {
-            const float lg = s_L[g];
-            out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
-        } else {
-            partials[((head0 + g) * cpp + cs) * C::PSTRIDE + c] = acc;
-        }
-    }
-    if (tid < G) {
-        const float lg = s_L[tid], mg = s_M[tid];
-        if (single) {
-            lse[head0 + tid] = lg > 0.f ? (mg + log2f(lg)) * kLn2 : -INFINITY;
-        } else {
-            float *pr = partials + ((head0 + tid) * cpp + cs) * C::PSTRIDE;
-            pr[D] = mg;
-            pr[D + 1] = lg;
-        }
-    }
-    if (single || !merge_here) return;
+    // merge_here: the CTAs of the pair are a cluster and meet at a cluster barrier below, so a CTA without
+    // pages (cs >= n_active) stays until then; otherwise (partials merged by combine_kernel) it is done.
+    const bool active = cs < n_active;
+    if (!active && (single || !merge_here)) return;
+    const int c_lo = min(cnt, cs * per_cta), c_hi = min(cnt, c_lo + per_cta);
+    float *s_lse2 = s_l;                  // final log2-sum-exp per head (the per-warp sums are dead by then)
 
-    // ---- several CTAs share the pair: the one holding the last ticket merges their partials
-    __threadfence();                  // this CTA's partial, before its ticket
-    __syncthreads();
-    if (tid == 0) {
-        const uint32_t t = atomicAdd(ticket + pair, 1u);
-        const int last = t == (uint32_t)n_active - 1u;
-        if (last) ticket[pair] = 0u;  // every other CTA has drawn already: left at zero for the next launch
-        *s_flag = last;
+    if (active) {
+        const int per_warp = (c_hi - c_lo + kDecWarps - 1) / kDecWarps;
+        const int i_lo = min(c_hi, c_lo + warp * per_warp), i_hi = min(c_hi, i_lo + per_warp);
+
+        AttendArgs a;
+        a.k_map = &k_map;
+        a.v_map = &v_map;
+        a.page_table = page_table;
+        a.max_pages = max_pages;
+        a.H_kv = H_kv;
+        a.P_phys = P_phys;
+        a.G = G;
+        a.GP = GP;
+        a.scale_log2 = scale_log2;
+        a.zero_chunk = smem_u32(smem_al + L::kZero);
+        a.status = status;
+        a.zrow = zbuf != nullptr ? zbuf + (size_t)pair * k_max * kPage * GP : nullptr;
+        a.keys_row = nullptr;
+
+        WarpAttn<D> A;
+        A.init_lane(lane);
+        A.reset();
+        bool ok = true;
+        if (i_lo < i_hi) {
+            A.load_q(q, head0, lane, G);
+            const int none[kChunk / 32] = {};
+            ok = attend_range<D, false, false>(P, A, a, [&](int i) { return list[i]; }, none, i_lo, i_hi, r, h, len,
+                                               n_r, lane);
+        }
+        if (!ok) {
+            if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
+            for (int s = 0; s < P.nstage; ++s) mbar_wait(P.bar0 + s * 8, (P.phases >> s) & 1u);
+        }
+        A.finish();
+
+        // ---- merge of the eight warps through shared memory.  Rows past the group hold zero queries:
+        // finite values that nobody reads.
+        if (tid4 == 0) {
+            s_m[warp * 8 + gid] = A.m_run;
+            s_l[warp * 8 + gid] = A.l_run;
+        }
+        __syncthreads();                  // every warp has drained its ring: it becomes the merge buffer
+        float mstar = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kDecWarps; ++w) mstar = fmaxf(mstar, s_m[w * 8 + gid]);
+        float lsum = 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecWarps; ++w) {
+            const float mw = s_m[w * 8 + gid];
+            lsum += (mw == -INFINITY) ? 0.f : exp2f(mw - mstar) * s_l[w * 8 + gid];
+        }
+        const float wgt = (A.m_run == -INFINITY) ? 0.f : exp2f(A.m_run - mstar);
+        float *red = reinterpret_cast<float *>(smem_al);
+        {
+            float *dst = red + (size_t)(warp * 8 + gid) * L::RED_PITCH + 2 * tid4;
+#pragma unroll
+            for (int nt = 0; nt < C::NTILES; ++nt)
+                *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(A.o_acc[nt][0] * wgt, A.o_acc[nt][1] * wgt);
+        }
+        if (warp == 0 && tid4 == 0) {
+            s_M[gid] = mstar;
+            s_L[gid] = lsum;
+        }
+        __syncthreads();
+        for (int e = tid; e < G * D; e += kDecWarps * 32) {
+            const int g = e / D, c = e - g * D;
+            float acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) acc += red[(size_t)(w * 8 + g) * L::RED_PITCH + c];
+            if (single) {
+                const float lg = s_L[g];
+                out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
+            } else {
+                partials[((head0 + g) * cpp + cs) * C::PSTRIDE + c] = acc;
+            }
+        }
+        if (tid < G) {
+            const float lg = s_L[tid], mg = s_M[tid];
+            if (single) {
+                const float l2 = lg > 0.f ? mg + log2f(lg) : -INFINITY;
+                lse[head0 + tid] = l2 * kLn2;
+                s_lse2[tid] = l2;
+            } else {
+                float *pr = partials + ((head0 + tid) * cpp + cs) * C::PSTRIDE;
+                pr[D] = mg;
+                pr[D + 1] = lg;
+            }
+        }
     }
-    __syncthreads();
-    if (!*s_flag) return;
-    __threadfence();                  // the other CTAs' partials are visible from here on
-    for (int e = tid; e < G * D; e += kDecWarps * 32) {
-        const int g = e / D, c = e - g * D;
-        const float *pr = partials + ((head0 + g) * cpp) * C::PSTRIDE;
-        float ms[kMergeInKernelMax], accs[kMergeInKernelMax];
-        float mg = -INFINITY;
-#pragma unroll
-        for (int s = 0; s < kMergeInKernelMax; ++s) {
-            ms[s] = -INFINITY;
-            accs[s] = 0.f;
-            if (s < n_active) {
-                ms[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
-                accs[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + c);
+    if (!single) {
+        if (!merge_here) return;          // combine_kernel merges the partials (and applies the H2O update)
+        // ---- several CTAs share the pair: after a cluster barrier every one of them knows all partials.
+        // Each computes the pair's final statistics (cheap), a share of the final output, and - below -
+        // the H2O update of the tokens it attended itself.
+        __threadfence();
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (!active) return;
+        if (tid < G) {
+            const float *pr = partials + ((head0 + tid) * cpp) * C::PSTRIDE;
+            float mg = -INFINITY, lg = 0.f;
+            for (int s = 0; s < n_active; ++s) mg = fmaxf(mg, __ldcg(pr + (size_t)s * C::PSTRIDE + D));
+            for (int s = 0; s < n_active; ++s) {
+                const float ms = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
+                if (ms != -INFINITY) lg += exp2f(ms - mg) * __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
             }
-            mg = fmaxf(mg, ms[s]);
+            s_M[tid] = mg;
+            s_L[tid] = lg;
+            const float l2 = lg > 0.f ? mg + log2f(lg) : -INFINITY;
+            s_lse2[tid] = l2;
+            if (cs == 0) lse[head0 + tid] = l2 * kLn2;
         }
-        float acc = 0.f, lg = 0.f;
-#pragma unroll
-        for (int s = 0; s < kMergeInKernelMax; ++s) {
-            if (s < n_active && ms[s] != -INFINITY) {
-                const float ws = exp2f(ms[s] - mg);
-                acc += ws * accs[s];
-                lg += ws * __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
+        __syncthreads();
+        for (int e = cs * (kDecWarps * 32) + tid; e < G * D; e += n_active * kDecWarps * 32) {
+            const int g = e / D, c = e - g * D;
+            const float *pr = partials + ((head0 + g) * cpp) * C::PSTRIDE;
+            const float mg = s_M[g], lg = s_L[g];
+            float acc = 0.f;
+            for (int s = 0; s < n_active; ++s) {
+                const float ms = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
+                if (ms != -INFINITY) acc += exp2f(ms - mg) * __ldcg(pr + (size_t)s * C::PSTRIDE + c);
             }
+            out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
         }
-        out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
-        if (c == 0) lse[head0 + g] = lg > 0.f ? (mg + log2f(lg)) * kLn2 : -INFINITY;
+    } else {
+        __syncthreads();                  // s_lse2
+    }
+    if (score_accum == nullptr || !merge_here) return;
+
+    // ---- H2O epilogue (Appendix A, H2O accumulated-score equation) for the tokens this CTA attended:
+    // score_accum[slot] += sum over the group's heads of 2^(z - lse2); their logits were written by this
+    // CTA's own warps.
+    for (int e = tid; e < (c_hi - c_lo) * kPage; e += kDecWarps * 32) {
+        const int i = c_lo + e / kPage, t = e % kPage;
+        const int b = list[i];
+        if (b < 0 || b >= n_r) continue;
+        const int pid = __ldg(page_table + (size_t)r * max_pages + b);
+        if (pid < 0 || pid >= P_phys) continue;
+        if (t >= min(kPage, len - b * kPage)) continue;
+        const float *z = zbuf + (((size_t)pair * k_max + i) * kPage + t) * GP;
+        float add = 0.f;
+        for (int gg = 0; gg < G; ++gg) {
+            const float zz = __ldcg(z + gg);
+            if (zz != -INFINITY) add += exp2f(zz - s_lse2[gg]);
+        }
+        score_accum[((size_t)pid * H_kv + h) * kPage + t] += add;
     }
 }
 
@@ -1144,7 +1170,7 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
             cfg.dynamicSmemBytes = smem;
             cfg.stream = stream;
             cudaLaunchAttribute attr[1];
-            if (fused && plan.max_splits > 1) {       // the CTAs of a pair form a cluster (they share a barrier)
+            if (plan.merge_in_kernel && plan.max_splits > 1) {   // the CTAs of a pair form a cluster (they share barriers)
                 attr[0].id = cudaLaunchAttributeClusterDimension;
                 attr[0].val.clusterDim.x = plan.max_splits;
                 attr[0].val.clusterDim.y = 1;
@@ -1153,9 +1179,9 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
                 cfg.numAttrs = 1;
             }
             e = cudaLaunchKernelEx(&cfg, kern, k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sa, fs, out, lse,
-                                   partials, zbuf, p.H_kv, G, GP, p.max_pages, p.num_phys_pages, p.k_max,
-                                   plan.max_splits, plan.merge_in_kernel ? 1 : 0, scale_log2, status,
-                                   reinterpret_cast<uint32_t *>(ws + L.pairctl));
+                                   partials, zbuf, plan.merge_in_kernel ? score_accum : (float *)nullptr, p.H_kv, G, GP,
+                                   p.max_pages, p.num_phys_pages, p.k_max, plan.max_splits,
+                                   plan.merge_in_kernel ? 1 : 0, scale_log2, status);
             if (e != cudaSuccess) return e;
         } else {
             const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
@@ -1174,6 +1200,7 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
     }
     if (!(stages & 2)) return e;
     const bool merged = plan.max_splits == 1 || (plan.cta_units && plan.merge_in_kernel);
+    if (plan.cta_units && plan.merge_in_kernel) return e;     // out/lse are final, the H2O epilogue ran in the kernel
     if (merged && !score_accum) return e;                     // out/lse are final and there is no epilogue
     // with the H2O epilogue the token slots of a pair (16 per selected page) are spread over
     // several CTAs, two slots per thread
