@@ -53,14 +53,15 @@ int decode_warps_per_cta();
 //    their partials themselves, more are merged by the merge kernel.
 //  - fewer than two pairs per SM: warp units, every pair cut into as many splits as the persistent
 //    warps of the grid can take in one round; the merge kernel combines them.
-//  - two or more pairs per SM: warp units, one per pair (a few warps per SM, each with a deep copy
-//    pipeline, already saturate HBM; splitting would only add the merge).
+//  - two to four pairs per SM: two adjacent warps per pair, merged through shared memory (decode_duo_kernel).
+//  - more: warp units, one warp per pair (splitting would only add the merge).
 DecodePlan make_decode_plan(const se_params &p, bool warp_units_only) {
     DecodePlan plan;
     const int warps_per_cta = decode_warps_per_cta();
     const long long pairs = (long long)p.B * p.H_kv;
     plan.cta_units = !warp_units_only && pairs <= kAssumedSMs;
     plan.merge_in_kernel = false;
+    plan.duo = false;
     if (plan.cta_units) {
         long long cpp = kAssumedSMs / pairs;
         const long long useful = (p.k_max + warps_per_cta - 1) / warps_per_cta;
@@ -82,6 +83,8 @@ DecodePlan make_decode_plan(const se_params &p, bool warp_units_only) {
     const long long units = pairs * plan.max_splits;
     long long grid = units < kAssumedSMs ? units : kAssumedSMs;
     plan.grid = (int)grid;
+    // two to four unsplit pairs per SM: two warps per pair (more busy warps per SM, even load)
+    plan.duo = !warp_units_only && plan.max_splits == 1 && pairs <= 4LL * kAssumedSMs;
     return plan;
 }
 

@@ -243,7 +243,7 @@ struct AttendArgs {
 template <int D, bool kObserve, bool kFirst, typename SelAt>
 __device__ __forceinline__ bool attend_range(WarpPipe &P, WarpAttn<D> &A, const AttendArgs &a, SelAt sel_at,
                                              const int (&first)[kChunk / 32], int i_lo, int i_hi, int r, int hh, int len,
-                                             int n_r, int lane) {
+                                             int n_r, int lane, bool use_first = true) {
     using C = DecCfg<D>;
     const int gid = lane >> 2, tid4 = lane & 3;
     const float scale_log2 = a.scale_log2;
@@ -262,7 +262,7 @@ __device__ __forceinline__ bool attend_range(WarpPipe &P, WarpAttn<D> &A, const 
             const int i = base + rep * 32 + lane;
             int pid = -1, meta = 0, lb = 0;
             if (i < end) {
-                const int b = (kFirst && base == i_lo) ? first[rep] : sel_at(i);
+                const int b = (kFirst && use_first && base == i_lo) ? first[rep] : sel_at(i);
                 if (b < 0 || b >= n_r) {
                     atomicOr(a.status, SE_DEV_BAD_SELECTION);
                 } else {
@@ -531,6 +531,180 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
     if (failed) {
         if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         // bounded wait for whatever this warp still has in flight before the CTA can retire
+        for (int s = 0; s < P.nstage; ++s) mbar_wait(P.bar0 + s * 8, (P.phases >> s) & 1u);
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// decode_duo_kernel: two to four pairs per SM.  Two adjacent warps share a pair: each attends half of
+// its selected pages, then the two exchange their statistics and half of their accumulators through
+// shared memory (named barriers of 64 threads) and each writes half of the output channels.  Six to
+// eight busy warps per SM with three stages each draw more bandwidth than three or four warps with
+// five or six stages (measured with the gather probe on the same page lists: 81.9 us against 87.5 us
+// for the 537 MB of config 3), and the halves even out the 4-against-3 pairs imbalance between CTAs.
+// Slot s = warp / 2 of CTA b holds the pairs b + s*gridDim.x (+ 4*gridDim.x ...).
+// ---------------------------------------------------------------------------------
+constexpr int kDuoStages = 16;           // stages per CTA (D = 128): two per warp; three per warp were 5 % slower
+
+__device__ __forceinline__ void duo_bar(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
+
+template <int D>
+__global__ void __launch_bounds__(kDecWarps * 32, 1)
+decode_duo_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+                  const uint16_t *__restrict__ q, const int32_t *__restrict__ page_table,
+                  const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ sel_idx,
+                  const int32_t *__restrict__ sel_cnt, float *__restrict__ out, float *__restrict__ lse,
+                  float *__restrict__ zbuf, int B, int H_kv, int G, int GP, int max_pages, int P_phys, int k_max,
+                  float scale_log2, uint32_t *status) {
+    using C = DecCfg<D>;
+    constexpr int STAGES = kDuoStages * (128 / D);
+    constexpr int XPITCH = D / 2 + 8;            // floats per head row of the exchange area
+    extern __shared__ uint8_t smem_dyn[];
+    uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int slot = warp >> 1, half = warp & 1;
+    const int pairs = B * H_kv;
+    // every busy warp of the grid gets the same number of stages (that of the fullest CTAs)
+    const int slots_max = min(kDecWarps / 2, (pairs + (int)gridDim.x - 1) / (int)gridDim.x);
+    const bool busy = slot * (int)gridDim.x + (int)blockIdx.x < pairs;
+    WarpPipe P;
+    P.nstage = busy ? min(C::MAXST, STAGES / (2 * slots_max)) : 0;
+    const int nst = min(C::MAXST, STAGES / (2 * slots_max));
+    uint8_t *ring = smem_al + (size_t)(warp * nst) * C::STAGEB;
+    uint8_t *ring_partner = smem_al + (size_t)((warp ^ 1) * nst) * C::STAGEB;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + (size_t)STAGES * C::STAGEB) + warp * C::MAXST;
+    if (lane == 0) {
+        for (int s = 0; s < P.nstage; ++s) mbar_init(smem_u32(&bars[s]), 2);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    P.bar0 = smem_u32(&bars[0]);
+    P.ring0 = smem_u32(ring);
+    P.phases = 0;
+    P.stage_c = 0;
+    P.stage_i = 0;
+    uint8_t *lists = smem_al + (size_t)STAGES * C::STAGEB + kDecWarps * C::MAXST * 8;
+    P.ent_y = reinterpret_cast<int *>(lists) + warp * 3 * kChunk;
+    P.ent_info = P.ent_y + kChunk;
+    P.ent_b = P.ent_info + kChunk;
+    uint8_t *zero_bytes = lists + (size_t)kDecWarps * 3 * kChunk * sizeof(int);
+    if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(zero_bytes)[threadIdx.x] = 0u;
+    __syncthreads();
+
+    AttendArgs a;
+    a.k_map = &k_map;
+    a.v_map = &v_map;
+    a.page_table = page_table;
+    a.max_pages = max_pages;
+    a.H_kv = H_kv;
+    a.P_phys = P_phys;
+    a.G = G;
+    a.GP = GP;
+    a.scale_log2 = scale_log2;
+    a.zero_chunk = smem_u32(zero_bytes);
+    a.status = status;
+    a.keys_row = nullptr;
+
+    const int H_q = H_kv * G;
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const bool head_ok = gid < G;
+    const int hs = (k_max + 1) / 2;              // where the second half starts when the whole row is selected
+    bool failed = false;
+    WarpAttn<D> A;
+    A.init_lane(lane);
+    float *xme = reinterpret_cast<float *>(ring), *xpa = reinterpret_cast<float *>(ring_partner);
+
+    for (int pair = slot * gridDim.x + blockIdx.x; pair < pairs && !failed; pair += (kDecWarps / 2) * gridDim.x) {
+        const int r = pair / H_kv, h = pair % H_kv;
+        const size_t head0 = (size_t)r * H_q + h * G;
+        const int32_t *sel_row = sel_idx + (size_t)pair * k_max;
+        // loads that depend on nothing travel together: Q, the lengths, the count and the first chunk of this
+        // half's entries - where the half starts if the whole row is selected (the usual case)
+        const int i_sp = half * hs;
+        int first[kChunk / 32];
+        A.load_q(q, head0, lane, G);
+#pragma unroll
+        for (int rep = 0; rep < kChunk / 32; ++rep) {
+            const int i = i_sp + rep * 32 + lane;
+            first[rep] = i < min(i_sp + hs, k_max) ? __ldg(sel_row + i) : -1;
+        }
+        const int len = __ldg(seq_lens + r);
+        const int n_r = len > 0 ? min(max_pages, (len + kPage - 1) / kPage) : 0;
+        int cnt = __ldg(sel_cnt + pair);
+        if (cnt > k_max) {
+            if (lane == 0) atomicOr(status, SE_DEV_BAD_SELECTION);
+            cnt = k_max;
+        }
+        if (cnt <= 0 || n_r == 0) {               // both warps of the pair take this branch
+            if (half == 0) {
+                for (int g = 0; g < G; ++g) {
+                    float *o = out + (head0 + g) * D;
+                    for (int c = lane; c < D; c += 32) o[c] = 0.f;
+                    if (lane == 0) lse[head0 + g] = -INFINITY;
+                }
+            }
+            continue;
+        }
+        const int hc = (cnt + 1) / 2;
+        const int i_lo = half ? hc : 0, i_hi = half ? cnt : hc;
+        A.reset();
+        a.zrow = zbuf != nullptr ? zbuf + (size_t)pair * k_max * kPage * GP : nullptr;
+        if (i_lo < i_hi) {
+            auto sel_at = [&](int i) { return __ldg(sel_row + i); };
+            if (!attend_range<D, false, true>(P, A, a, sel_at, first, i_lo, i_hi, r, h, len, n_r, lane, i_lo == i_sp))
+                failed = true;                    // still goes through the pair's barriers below
+        }
+        A.finish();
+
+        // ---- the two halves meet: statistics, then the accumulators of the channels the partner finishes
+        const int bar_id = 1 + slot;
+        if (tid4 == 0) {
+            xme[gid] = A.m_run;
+            xme[8 + gid] = A.l_run;
+        }
+        duo_bar(bar_id);
+        const float mo = xpa[gid], lo = xpa[8 + gid];
+        const float mstar = fmaxf(A.m_run, mo);
+        const float ws = (A.m_run == -INFINITY) ? 0.f : exp2f(A.m_run - mstar);
+        const float wo = (mo == -INFINITY) ? 0.f : exp2f(mo - mstar);
+        const float lsum = ws * A.l_run + wo * lo;
+        constexpr int HT = C::NTILES / 2;        // half 0 finishes the n-tiles [0, HT), half 1 the others
+        float *dst = xme + 16 + gid * XPITCH + 2 * tid4;
+        if (half == 0) {
+#pragma unroll
+            for (int t = 0; t < HT; ++t)
+                *reinterpret_cast<float2 *>(dst + t * 8) = make_float2(A.o_acc[HT + t][0] * ws, A.o_acc[HT + t][1] * ws);
+        } else {
+#pragma unroll
+            for (int t = 0; t < HT; ++t)
+                *reinterpret_cast<float2 *>(dst + t * 8) = make_float2(A.o_acc[t][0] * ws, A.o_acc[t][1] * ws);
+        }
+        duo_bar(bar_id);
+        if (head_ok) {
+            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+            const float *src = xpa + 16 + gid * XPITCH + 2 * tid4;
+            float *o = out + (head0 + gid) * D + 2 * tid4;
+            if (half == 0) {
+#pragma unroll
+                for (int t = 0; t < HT; ++t) {
+                    const float2 v = *reinterpret_cast<const float2 *>(src + t * 8);
+                    *reinterpret_cast<float2 *>(o + t * 8) = make_float2((A.o_acc[t][0] * ws + v.x) * inv, (A.o_acc[t][1] * ws + v.y) * inv);
+                }
+                if (tid4 == 0) lse[head0 + gid] = lsum > 0.f ? (mstar + log2f(lsum)) * kLn2 : -INFINITY;
+            } else {
+#pragma unroll
+                for (int t = 0; t < HT; ++t) {
+                    const float2 v = *reinterpret_cast<const float2 *>(src + t * 8);
+                    *reinterpret_cast<float2 *>(o + (HT + t) * 8) =
+                        make_float2((A.o_acc[HT + t][0] * ws + v.x) * inv, (A.o_acc[HT + t][1] * ws + v.y) * inv);
+                }
+            }
+        }
+        duo_bar(bar_id);          // the partner has read this warp's area: the ring may be refilled
+        fence_proxy_async();      // ... by tensor copies, after these ordinary stores
+    }
+    if (failed) {
+        if (lane == 0) atomicOr(status, SE_DEV_WAIT_TIMEOUT);
         for (int s = 0; s < P.nstage; ++s) mbar_wait(P.bar0 + s * 8, (P.phases >> s) & 1u);
     }
 }
@@ -1183,6 +1357,16 @@ cudaError_t launch_decode(const se_params &p, const void *q, const void *k_cache
                                    p.max_pages, p.num_phys_pages, p.k_max, plan.max_splits,
                                    plan.merge_in_kernel ? 1 : 0, scale_log2, status);
             if (e != cudaSuccess) return e;
+        } else if (plan.duo) {
+            if (select) return cudaErrorInvalidValue;         // only CTA units select in the kernel
+            const size_t smem = (size_t)kDuoStages * (128 / D) * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
+                                (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 16 + 1024;
+            auto kern = decode_duo_kernel<D>;
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            kern<<<plan.grid, kDecWarps * 32, smem, stream>>>(
+                k_map, v_map, (const uint16_t *)q, page_table, seq_lens, sel_idx, sel_cnt, out, lse, zbuf, p.B, p.H_kv,
+                G, GP, p.max_pages, p.num_phys_pages, p.k_max, scale_log2, status);
         } else {
             const size_t smem = (size_t)C::CTA_STAGES * C::STAGEB + (size_t)kDecWarps * C::MAXST * 8 +
                                 (size_t)kDecWarps * 3 * kChunk * sizeof(int) + 16 + 1024;

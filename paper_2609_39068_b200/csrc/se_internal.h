@@ -17,7 +17,8 @@ struct DecodePlan {
                             // one warp per (pair, split)
     int pages_per_split;    // warp units: selected pages of one split
     int max_splits;         // splits per pair (warp units: ceil(k_max / pages_per_split); CTA units: CTAs per pair)
-    bool merge_in_kernel;   // CTA units: the last-arriving CTA of a pair merges the pair's partials itself
+    bool merge_in_kernel;   // CTA units: the CTAs of a pair are a cluster and merge their partials themselves
+    bool duo;               // warp units, unsplit pairs: decode_duo_kernel - two adjacent warps share a pair
 };
 
 // the selection comes from the page scores in the workspace: the attention kernel runs the top-k

@@ -500,11 +500,12 @@ def test_ties_with_selection_inside_the_attention_kernel():
     compare(w_cpu, st)
 
 
-@pytest.mark.parametrize("pairs", [2, 40, 148, 200, 400])
+@pytest.mark.parametrize("pairs", [2, 40, 148, 200, 400, 592, 700])
 def test_every_launch_plan_against_the_oracle(pairs):
-    """The attention step has three geometries, picked from the number of (request, kv-head) pairs: CTA
-    units with an in-kernel merge (<= 148 pairs), warp units with splits and the merge kernel (< 296),
-    one warp per pair (>= 296).  Each one against the oracle, with and without the H2O epilogue."""
+    """The attention step has four geometries, picked from the number of (request, kv-head) pairs: CTA
+    units in a cluster (<= 148 pairs), warp units with splits and the merge kernel (< 296), two warps per
+    pair (<= 592), one warp per pair (more).  Each one against the oracle, with and without the H2O
+    epilogue."""
     H_kv = 2 if pairs % 2 == 0 else 1
     B = pairs // H_kv
     rng = np.random.default_rng(pairs)
@@ -545,7 +546,7 @@ def test_kv_head_shards_reproduce_the_unsharded_step(many_pairs):
     a pair (many_pairs) every output is bit-identical; with few pairs the split-K geometry differs
     between the shapes, so out/lse/score_accum agree to fp32 rounding and the rest bit for bit."""
     if many_pairs:
-        seq = [300 + 37 * i for i in range(100)]            # 100 requests x 8 kv-heads: 400 pairs per shard
+        seq = [300 + 23 * i for i in range(160)]            # 160 requests x 8 kv-heads: 640 pairs per shard (one warp per pair in both runs)
     else:
         seq = [5000, 3000, 9000, 17]
     w = wl.build("tp", 895, 0, seq, 16, 8, 128, 256, "cpu", permute_pool=True, prune_fraction=0.1,
