@@ -167,13 +167,16 @@ def checksums(w):
             "page_table": s64(w.page_table), "seq_lens": s64(w.seq_lens)}
 
 
-def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0, instance: int = 0):
+def make_layers(config: int, device, n_layers: int, rank: int, batch: int = 0, instance: int = 0, hi: int = 0):
     """The layers of one instance of a config.  Structure (lengths, page table) is the same for every layer
     and instance; q/K/V values differ (seeded by layer index; other instances and ranks use other layer seeds)."""
     fn = wl.CONFIGS[config]
-    if batch:
+    if batch or hi:
         base = fn
-        fn = lambda device, layer=0: base(device, layer=layer, B=batch)
+        kw = dict(B=batch) if batch else {}
+        if hi:
+            kw["hi"] = hi
+        fn = lambda device, layer=0: base(device, layer=layer, **kw)
     layers = []
     first = None
     for l in range(n_layers):
@@ -222,8 +225,8 @@ def oracle_step_time(w, meta_bits, threads=None, min_runs=3, budget_s=20.0):
 class Instance:
     """One independent copy of a config's layers with its states, H2O accumulators and the graph of its step."""
 
-    def __init__(self, binding, config, dev, n_layers, rank, batch, index, dense_layers=0, use_graph=True):
-        self.layers = make_layers(config, dev, n_layers, rank, batch, index)
+    def __init__(self, binding, config, dev, n_layers, rank, batch, index, dense_layers=0, use_graph=True, hi=0):
+        self.layers = make_layers(config, dev, n_layers, rank, batch, index, hi)
         w0 = self.layers[0]
         self.h2o = w0.score_accum is not None
         self.dense_layers = dense_layers
@@ -499,7 +502,8 @@ def run_config(binding, config, dev, args, rank, world, barrier, full: bool, K: 
     batch = args.batch if full else 0
     use_graph = not args.no_graph
     dense = args.dense_layers if (full or config == 5) else 0
-    inst0 = Instance(binding, config, dev, n_layers, rank, batch, 0, dense_layers=dense, use_graph=use_graph)
+    hi = args.hi if full else 0
+    inst0 = Instance(binding, config, dev, n_layers, rank, batch, 0, dense_layers=dense, use_graph=use_graph, hi=hi)
     layers, states = inst0.layers, inst0.states
     h2o = inst0.h2o
     bytes_l = [algorithmic_bytes(st.w, st.sel_cnt, h2o) for st in states]
@@ -510,7 +514,7 @@ def run_config(binding, config, dev, args, rank, world, barrier, full: bool, K: 
         R = -(-4 * L2_BYTES // total_bytes)
         if R <= 8:
             mode = "rotate"
-            instances += [Instance(binding, config, dev, n_layers, rank, batch, i, dense_layers=dense, use_graph=use_graph)
+            instances += [Instance(binding, config, dev, n_layers, rank, batch, i, dense_layers=dense, use_graph=use_graph, hi=hi)
                           for i in range(1, R)]
         else:
             mode = "flush"
@@ -720,6 +724,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=0,
                     help="override the number of requests (configs 3-5; for small profiling captures)")
+    ap.add_argument("--hi", type=int, default=0,
+                    help="override the longest context of configs 3 and 5 (for small profiling captures)")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls directly instead of a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the short runs of the other configs")
@@ -779,7 +785,7 @@ def main():
     torch.cuda.empty_cache()
 
     other = None
-    if rank == 0 and world == 1 and not args.no_other_configs and not args.batch:
+    if rank == 0 and world == 1 and not args.no_other_configs and not args.batch and not args.hi:
         other = {}
         for c in sorted(wl.CONFIGS):
             if c == args.config:

@@ -17,7 +17,9 @@
  *  - `stream` is a `cudaStream_t` passed as `void*` (NULL = the default stream).  Calls
  *    enqueue work on it and return; only `se_last_device_status` synchronises.
  *  - Return value: SE_OK (0) or a negative SE_ERR_* code.  Arguments are validated on
- *    the host before anything is launched; on error nothing has been enqueued.
+ *    the host before anything is launched: a call that fails validation enqueues nothing.
+ *    SE_ERR_CUDA (a launch or a runtime call failed after validation) may leave part of
+ *    the call's work - a memset, an earlier kernel of a multi-kernel call - enqueued.
  *  - Shapes: B requests, H_q query heads, H_kv kv-heads, G = H_q / H_kv in 1..8,
  *    D in {64, 128}, page size 16 tokens.  Query head a reads kv-head a / G
  *    (Appendix A, "MHA, MQA, and GQA").
@@ -68,7 +70,7 @@ extern "C" {
 /* bits of the device status word */
 #define SE_DEV_BAD_PAGE_ID          1u  /* page_table entry >= num_phys_pages              */
 #define SE_DEV_BAD_SELECTION        2u  /* sel_idx entry outside the request / sel_cnt > k_max */
-#define SE_DEV_WAIT_TIMEOUT         4u  /* a bounded wait on an asynchronous copy gave up   */
+#define SE_DEV_WAIT_TIMEOUT         4u  /* a bounded wait (200 ms) on an asynchronous copy gave up */
 
 typedef struct se_params {
     int32_t B;               /* requests in the batch (>= 1)                                */

@@ -41,6 +41,8 @@ bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u
 
 int device_sm_count() { return kAssumedSMs; }
 
+int validate_params(const se_params *p) { return validate(p); }
+
 float effective_scale(const se_params &p) {
     return p.sm_scale > 0.f ? p.sm_scale : 1.0f / sqrtf((float)p.D);
 }

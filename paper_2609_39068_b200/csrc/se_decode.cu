@@ -1619,6 +1619,8 @@ token_decode_kernel(const uint16_t *__restrict__ q, const uint8_t *__restrict__ 
                     mma_bf16_16816(o_acc[2 * c2 + 1], ph0, pl0, ph1, pl1, v10, v11);
                 }
                 __syncwarp();
+                // rows cleared with ordinary stores come before the bulk copies that refill the stage
+                if (vmask != 0xffffu) fence_proxy_async();
                 ++ce;
                 top_up();
             }

@@ -61,14 +61,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after kWaitLimit polls (each poll may itself block for a
-// hardware-defined short time) and reports failure instead of spinning forever.
-constexpr int kWaitLimit = 1 << 20;
+// Bounded wait: gives up after kWaitLimitNs of wall-clock time (%globaltimer; far beyond any copy's
+// latency) and reports failure instead of spinning forever.
+constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int it = 0; it < kWaitLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 256; ++it)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+    }
 }
 
 // One-dimensional bulk asynchronous copy global -> shared (no tensor map, no multicast).

@@ -29,6 +29,7 @@ struct SelectFromScores {
 };
 
 int  device_sm_count();
+int  validate_params(const se_params *p);        // SE_OK or the SE_ERR_* code every entry point returns for a bad `p`
 DecodePlan make_decode_plan(const se_params &p, bool warp_units_only = false);
 // whether the attention kernel's own top-k covers the shape (otherwise the top-k kernel runs)
 bool select_in_decode_ok(const se_params &p);

@@ -19,6 +19,8 @@
 //                threshold by a histogram over the keys' span plus a brute-force ranking of the
 //                crossing bin, then a page-ordered compaction, so equal scores go to the lower
 //                page and the list is ascending.
+#include <atomic>
+
 #include "se_internal.h"
 #include "se_topk.cuh"
 
@@ -496,21 +498,22 @@ static __device__ __align__(256) unsigned char g_select_scratch[SE_STATIC_SCRATC
 namespace {
 
 constexpr int kMaxDevices = 64;
-void *g_scratch_ptr[kMaxDevices];          // device address of g_select_scratch, per device ordinal
-bool g_scratch_ready[kMaxDevices];
+// device address of g_select_scratch, per device ordinal (nullptr = not looked up yet).  Host threads may
+// race on the first call of a device: the look-up is idempotent, the slot is written atomically.
+std::atomic<void *> g_scratch_ptr[kMaxDevices];
 
 // The array's name is only a host-side handle: the address kernels can use has to be asked for,
-// once per device, with that device current.
+// once per device, with that device current (the caller's buffers and stream belong to the current
+// device, as with every other entry point).
 int static_scratch(void **out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SE_ERR_CUDA;
-    if (!g_scratch_ready[dev]) {
-        void *ptr = nullptr;
+    void *ptr = g_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (ptr == nullptr) {
         if (cudaGetSymbolAddress(&ptr, g_select_scratch) != cudaSuccess || ptr == nullptr) return SE_ERR_CUDA;
-        g_scratch_ptr[dev] = ptr;
-        g_scratch_ready[dev] = true;
+        g_scratch_ptr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_ptr[dev];
+    *out = ptr;
     return SE_OK;
 }
 
@@ -520,8 +523,8 @@ extern "C" int se_page_select_static(const se_params *p, const void *q, const vo
                                      const int32_t *page_table, const int32_t *seq_lens,
                                      int32_t budget_tokens, int32_t *sel_idx, int32_t *sel_cnt,
                                      int32_t *dev_status, void *stream) {
-    if (!p) return SE_ERR_NULL_POINTER;
-    if (se_workspace_bytes(p) == 0) return SE_ERR_INVALID_ARG;          // same shape rules as every call
+    const int vrc = se::validate_params(p);                             // same shape rules and codes as every call
+    if (vrc != SE_OK) return vrc;
     if (!q || !meta || !page_table || !seq_lens || !sel_idx || !sel_cnt) return SE_ERR_NULL_POINTER;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(meta) |
                            reinterpret_cast<uintptr_t>(page_table) | reinterpret_cast<uintptr_t>(seq_lens) |
