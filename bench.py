@@ -51,9 +51,10 @@ FALLBACK_HBM_GBS = 6650.0
 WINDOW_WARMUP = 32                     # untimed replays in front of every timed window
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in profiles/
-# (small-batch captures scaled by the pages processed; null where no capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"config3_contbatch_b64_mix": 539.5e6}          # decode_kernel
-NCU_TRAFFIC_BYTES_SCORE = {"config3_contbatch_b64_mix": 563.2e6}    # score_kernel
+# (profiles/full_capture_config3_b40.md: a 40-request capture scaled to the full launch by the pages processed;
+# null where no capture of that workload exists)
+NCU_TRAFFIC_BYTES = {"config3_contbatch_b64_mix": 543.8e6}          # decode_duo_kernel: 339.89 MB x 65536 / 40960
+NCU_TRAFFIC_BYTES_SCORE = {"config3_contbatch_b64_mix": 577.6e6}    # score_kernel: 200.28 MB x 137094 / 47538
 H2O_NCU_TRAFFIC_BYTES = 2055e6         # h2o_compact_kernel, 64-request eviction workload
 OMNIKV_NCU_TRAFFIC_BYTES = 209e6       # token_decode_kernel, 24-request selection-reuse workload
 
