@@ -48,12 +48,51 @@ def test_workspace_bytes_is_pure_and_monotone():
 
 
 def test_decode_split_plan():
-    # few pairs: split so that every persistent warp has a unit; two or more pairs per SM: no split
+    # few pairs: split (CTAs per pair, or warps per pair); two or more pairs per SM: no split
     few = binding.make_params(8, 32, 8, 128, 2048, 16384, 128)
     many = binding.make_params(64, 32, 8, 128, 4096, 140000, 128)
-    assert binding.se_decode_num_splits(few) > 1
+    assert binding.se_decode_num_splits(few) == 2                 # 64 pairs: two CTAs per pair
+    assert binding.se_decode_num_splits(binding.make_params(24, 32, 8, 128, 2048, 16384, 128)) == 6   # 192 pairs: warps
     assert binding.se_decode_num_splits(many) == 1
     assert binding.se_decode_num_splits(binding.make_params(8, 32, 8, 96, 2048, 16384, 128)) == 0
+
+
+@pytest.mark.parametrize("B,H_kv,k_max,budget,h2o,launches", [
+    (1, 2, 16, 256, False, 1),        # config 1: one fused kernel per step
+    (8, 8, 128, 2048, False, 1),      # config 2
+    (4, 8, 256, 4096, True, 1),       # config 4: the H2O update runs in the same kernel
+    (1, 1, 4096, 65536, False, 3),    # one pair, 148 CTAs: scoring, attention (top-k in its prologue), merge kernel
+    (24, 8, 128, 2048, False, 4),     # 192 pairs: scoring, top-k, warp-split attention, merge
+    (64, 8, 128, 2048, False, 3),     # config 3: scoring, top-k, two warps per pair
+    (64, 8, 128, 2048, True, 4),      # ... + the H2O epilogue kernel
+    (128, 8, 64, 1024, False, 3),     # 1024 pairs: one warp per pair
+    (8, 8, 2048, 16 * 2048, False, 3),  # dense layer: summary update, list of all pages, attention
+])
+def test_step_launch_plan_follows_from_the_shape(B, H_kv, k_max, budget, h2o, launches):
+    p = binding.make_params(B, 4 * H_kv, H_kv, 128, 8192 if k_max > 2048 else 2048, 1 << 16, k_max)
+    assert binding.se_decode_step_launches(p, budget, h2o) == launches
+    assert binding.se_decode_step_launches(p, 8, h2o) == 0                   # budget below one page
+    assert binding.se_decode_step_launches(binding.make_params(B, 4 * H_kv, H_kv, 96, 2048, 1 << 16, k_max), budget, h2o) == 0
+
+
+def test_decode_step_and_probe_reject_bad_arguments_before_launch():
+    lib = binding.load()
+    p = binding.make_params(2, 32, 8, 128, 64, 128, 16)
+    pp = ctypes.byref(p)
+    ok, odd = ctypes.c_void_p(4096), ctypes.c_void_p(4100)
+    args = [pp, ok, ok, ok, ok, ok, ok, 256, ok, ok, ok, ok, None, ok, None]
+    bad = list(args); bad[4] = None
+    assert lib.se_decode_step(*bad) == -3                                     # meta missing
+    bad = list(args); bad[10] = odd
+    assert lib.se_decode_step(*bad) == -4
+    bad = list(args); bad[7] = 8
+    assert lib.se_decode_step(*bad) == -1                                     # budget below one page
+    bad = list(args); bad[7] = 16 * 17
+    assert lib.se_decode_step(*bad) == -1                                     # more pages than k_max
+    assert lib.se_probe_gather(None, None, ok, 16, 512, 16, 2, 4, 3, None) == -3
+    assert lib.se_probe_gather(ok, None, ok, 16, 500, 16, 2, 4, 3, None) == -1   # piece size not a multiple of 16
+    assert lib.se_probe_gather(ok, None, ok, 16, 4096, 32, 8, 8, 1, None) == -1  # does not fit shared memory
+    assert lib.se_probe_gather(ok, None, odd, 16, 512, 16, 2, 4, 3, None) == -4
 
 
 @pytest.mark.parametrize("kw", [
