@@ -32,9 +32,9 @@ def needs_build() -> bool:
     return os.path.getmtime(LIB) < _newest(deps)
 
 
-def _compile(src: str, verbose: bool) -> str:
-    obj = os.path.join(OBJ, src.replace(".cu", ".o"))
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
+def _compile(src: str, verbose: bool, extra=(), suffix: str = "") -> str:
+    obj = os.path.join(OBJ, src.replace(".cu", suffix + ".o"))
+    cmd = [_nvcc()] + NVCC_FLAGS + list(extra) + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed for %s:\n%s\n%s" % (src, res.stdout, res.stderr))
@@ -54,6 +54,25 @@ def build(force: bool = False, verbose: bool = False) -> str:
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
     os.replace(tmp, LIB)
     return LIB
+
+
+# A second build of the same sources with -DSE_TEST_SHORT_TX: the scoring kernel's waits run out (see
+# se_select.cu).  Only tests/test_gpu_timeout.py loads it.
+LIB_SHORT_TX = os.path.join(HERE, "libsparse_engine_shorttx.so")
+
+
+def build_short_tx(force: bool = False) -> str:
+    deps = [os.path.join(CSRC, s) for s in SOURCES] + [os.path.join(CSRC, h) for h in HEADERS]
+    if not force and os.path.exists(LIB_SHORT_TX) and os.path.getmtime(LIB_SHORT_TX) >= _newest(deps):
+        return LIB_SHORT_TX
+    os.makedirs(OBJ, exist_ok=True)
+    with concurrent.futures.ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
+        list(ex.map(lambda s: _compile(s, False, ["-DSE_TEST_SHORT_TX"], "_shorttx"), SOURCES))
+    objs = [os.path.join(OBJ, s.replace(".cu", "_shorttx.o")) for s in SOURCES]
+    tmp = LIB_SHORT_TX + ".tmp%d" % os.getpid()
+    subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+    os.replace(tmp, LIB_SHORT_TX)
+    return LIB_SHORT_TX
 
 
 if __name__ == "__main__":

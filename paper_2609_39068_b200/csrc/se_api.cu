@@ -41,6 +41,12 @@ bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u
 
 int device_sm_count() { return kAssumedSMs; }
 
+// cudaOccupancyMaxActiveClusters on a B200 for a 256-thread CTA with 217 KB of shared memory (one CTA per SM)
+int max_resident_clusters(int size) {
+    static const int kTable[9] = {0, 148, 74, 45, 33, 26, 22, 15, 15};
+    return (size >= 1 && size <= 8) ? kTable[size] : 0;
+}
+
 int validate_params(const se_params *p) { return validate(p); }
 
 float effective_scale(const se_params &p) {
@@ -69,6 +75,9 @@ DecodePlan make_decode_plan(const se_params &p, bool warp_units_only) {
         const long long useful = (p.k_max + warps_per_cta - 1) / warps_per_cta;
         if (cpp > useful) cpp = useful;
         if (cpp < 1) cpp = 1;
+        // as a cluster (up to 8 CTAs) all pairs' clusters must be resident at once: a second wave doubles the time
+        if (cpp <= 8)
+            while (cpp > 1 && max_resident_clusters((int)cpp) < pairs) --cpp;
         plan.max_splits = (int)cpp;
         plan.pages_per_split = (int)((p.k_max + cpp - 1) / cpp);
         plan.merge_in_kernel = cpp <= 8;

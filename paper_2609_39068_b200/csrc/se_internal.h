@@ -29,6 +29,9 @@ struct SelectFromScores {
 };
 
 int  device_sm_count();
+// Thread-block clusters of `size` CTAs that can be resident at once when a CTA fills an SM (B200: the CTAs
+// of a cluster sit in one GPC, so not every size packs all 148 SMs).
+int  max_resident_clusters(int size);
 int  validate_params(const se_params *p);        // SE_OK or the SE_ERR_* code every entry point returns for a bad `p`
 DecodePlan make_decode_plan(const se_params &p, bool warp_units_only = false);
 // whether the attention kernel's own top-k covers the shape (otherwise the top-k kernel runs)

@@ -28,6 +28,15 @@ namespace se {
 
 namespace {
 
+// Fault injection for the test of the bounded waits (a second build of the library, -DSE_TEST_SHORT_TX,
+// never the product): every batch announces 16 bytes more than its copies deliver, so the wait for it
+// runs out, the kernel reports SE_DEV_WAIT_TIMEOUT and returns.
+#ifdef SE_TEST_SHORT_TX
+constexpr uint32_t kTestExtraTx = 16;
+#else
+constexpr uint32_t kTestExtraTx = 0;
+#endif
+
 constexpr int kScoreWarps = 4;     // warps per CTA of the score kernel
 constexpr int kPB = 16;            // pages per warp batch (one m16 tile)
 constexpr int kNBU = 4;            // batches per work unit  -> 64 pages per (pair, unit)
@@ -264,7 +273,7 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
         }
         const unsigned valid = __ballot_sync(kFull, pid >= 0 && lane != fresh);
         const uint32_t bar = bar0 + slot * 8;
-        if (lane == 0) mbar_expect_tx(bar, (uint32_t)__popc(valid) * C::PHB);
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)__popc(valid) * C::PHB + kTestExtraTx);
         __syncwarp();
         if (pid >= 0 && lane != fresh) {
             const uint8_t *src = meta + ((size_t)pid * H_kv + d.h) * C::PHB;

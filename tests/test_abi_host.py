@@ -52,6 +52,8 @@ def test_decode_split_plan():
     few = binding.make_params(8, 32, 8, 128, 2048, 16384, 128)
     many = binding.make_params(64, 32, 8, 128, 4096, 140000, 128)
     assert binding.se_decode_num_splits(few) == 2                 # 64 pairs: two CTAs per pair
+    # 24 pairs: 148 / 24 = 6 CTAs per pair would need 24 clusters of 6 resident at once; only 22 are, so 5
+    assert binding.se_decode_num_splits(binding.make_params(3, 32, 8, 128, 2048, 16384, 128)) == 5
     assert binding.se_decode_num_splits(binding.make_params(24, 32, 8, 128, 2048, 16384, 128)) == 6   # 192 pairs: warps
     assert binding.se_decode_num_splits(many) == 1
     assert binding.se_decode_num_splits(binding.make_params(8, 32, 8, 96, 2048, 16384, 128)) == 0

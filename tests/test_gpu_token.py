@@ -90,7 +90,8 @@ def check_attend(w_cpu, tok_idx, tok_cnt, out, lse, rows=None):
     assert np.abs(l[fin] - l_ref[fin]).max(initial=0.0) <= LSE_ABS
 
 
-@pytest.mark.parametrize("D,H_q,H_kv", [(128, 8, 2), (64, 4, 4), (128, 7, 1)])
+# (one to sixteen kv-heads and both head sizes: the kernel's work units are (request, kv-head, token chunk))
+@pytest.mark.parametrize("D,H_q,H_kv", [(128, 8, 2), (64, 4, 4), (128, 7, 1), (128, 16, 16), (64, 8, 8)])
 @pytest.mark.parametrize("prune", [0.0, 0.3])
 def test_observe_select_reuse_small(D, H_q, H_kv, prune):
     w_cpu = wl.build("tok", 980, 0, [700, 300, 17, 1, 1200], H_q, H_kv, D, 64, "cpu", permute_pool=True,
