@@ -1,13 +1,16 @@
 // Paged attention over the selected pages, log-sum-exp merge and the H2O epilogue
 // (Appendix A, selected-attention equation and H2O accumulated-score equation).
 //
-// Two attention kernels share the per-page arithmetic (WarpAttn) and the per-warp copy pipeline
+// Three attention kernels share the per-page arithmetic (WarpAttn) and the per-warp copy pipeline
 // (attend_range); which one runs follows from the shape alone (make_decode_plan):
 //
 // decode_kernel      many (request, kv-head) pairs.  Persistent grid, every warp an autonomous
-//                    pipeline working through (pair, split) units; with two or more pairs per SM
-//                    a pair is one unit and its warp writes out/lse itself, otherwise the pair is cut
-//                    into splits whose partials (acc, m, l) combine_kernel merges.
+//                    pipeline working through (pair, split) units; with more than four pairs per SM
+//                    a pair is one unit and its warp writes out/lse itself, with fewer than two the
+//                    pair is cut into splits whose partials (acc, m, l) combine_kernel merges.
+// decode_duo_kernel  two to four pairs per SM.  Two adjacent warps share a pair (the two halves of
+//                    its list) and merge through the shared memory of their drained rings: twice
+//                    the busy warps per SM of the one-warp form, no partials in global memory.
 // decode_cta_kernel  at most one pair per SM.  A CTA is one (pair, CTA-split); its eight warps share
 //                    the CTA's pages and their partials are merged through shared memory.  The CTAs
 //                    of a pair (up to 8) form a thread-block cluster: after a cluster barrier each
@@ -18,7 +21,10 @@
 // the top-k in its prologue (se_topk.cuh: cta_topk), while the shared-memory ring is still empty and
 // serves as its scratch; the list is also written to sel_idx / sel_cnt.  That removes the top-k
 // kernel and the selection's round trip from the step.  (With warp units a warp would have to run the
-// top-k alone, which is slower than the top-k kernel: those shapes keep it.)
+// top-k alone, which is slower than the top-k kernel: those shapes keep it.)  With kFused the CTAs of the
+// pair's cluster first score the pair's pages themselves (cta_score_range: the page summaries stream
+// through the same ring, the scores go to the workspace, a cluster barrier ends the phase), so the
+// whole step - summary of the newest page, scores, top-k, attention, merge, H2O update - is one launch.
 //
 // Per page, for the G query heads of the kv-head at once:
 //     S^T[head, token] = Q[head, :] . K[token, :]^T      (m16n8k16, fp32 accumulate)
@@ -539,7 +545,7 @@ decode_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__
 // decode_duo_kernel: two to four pairs per SM.  Two adjacent warps share a pair: each attends half of
 // its selected pages, then the two exchange their statistics and half of their accumulators through
 // shared memory (named barriers of 64 threads) and each writes half of the output channels.  Six to
-// eight busy warps per SM with three stages each draw more bandwidth than three or four warps with
+// eight busy warps per SM with two stages each draw more bandwidth than three or four warps with
 // five or six stages (measured with the gather probe on the same page lists: 81.9 us against 87.5 us
 // for the 537 MB of config 3), and the halves even out the 4-against-3 pairs imbalance between CTAs.
 // Slot s = warp / 2 of CTA b holds the pairs b + s*gridDim.x (+ 4*gridDim.x ...).

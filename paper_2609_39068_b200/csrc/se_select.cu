@@ -15,10 +15,11 @@
 //                and accumulate in fp32.  An earlier plain-FMA version of this kernel was
 //                issue-bound at 64 % of the copy bandwidth (57 warp instructions per page
 //                summary); this one needs 3.
-// topk_kernel    one CTA per (request, kv-head): order-preserving integer keys held in registers,
-//                threshold by a histogram over the keys' span plus a brute-force ranking of the
-//                crossing bin, then a page-ordered compaction, so equal scores go to the lower
-//                page and the list is ascending.
+// topk_kernel    one CTA per (request, kv-head) runs cta_topk (se_topk.cuh): order-preserving integer
+//                keys in thread-private 16-byte groups of shared memory, threshold by a histogram
+//                over the keys' span plus a brute-force ranking of the crossing bin, then a
+//                page-ordered compaction, so equal scores go to the lower page and the list is
+//                ascending.  The attention kernel of small shapes calls the same function itself.
 #include <atomic>
 
 #include "se_internal.h"
