@@ -61,7 +61,7 @@ extern "C" {
 
 #define SE_OK                       0
 #define SE_ERR_INVALID_ARG         -1   /* a size or value is out of range                 */
-#define SE_ERR_UNSUPPORTED_SHAPE   -2   /* D, G or page_size not supported                 */
+#define SE_ERR_UNSUPPORTED_SHAPE   -2   /* D, G, page_size or B not supported              */
 #define SE_ERR_NULL_POINTER        -3   /* a required pointer is NULL                      */
 #define SE_ERR_MISALIGNED          -4   /* a pointer is not 16-byte aligned                */
 #define SE_ERR_CUDA                -5   /* a CUDA runtime call failed (launch, attribute)  */
@@ -73,7 +73,7 @@ extern "C" {
 #define SE_DEV_WAIT_TIMEOUT         4u  /* a bounded wait (200 ms) on an asynchronous copy gave up */
 
 typedef struct se_params {
-    int32_t B;               /* requests in the batch (>= 1)                                */
+    int32_t B;               /* requests in the batch, 1..8192                              */
     int32_t H_q;             /* query heads                                                 */
     int32_t H_kv;            /* kv heads; H_q % H_kv == 0, H_q / H_kv in 1..8               */
     int32_t D;               /* head dimension, 64 or 128                                   */

@@ -17,6 +17,7 @@ int validate(const se_params *p) {
     if (p->page_size != kPage) return SE_ERR_UNSUPPORTED_SHAPE;
     if (p->D != 64 && p->D != 128) return SE_ERR_UNSUPPORTED_SHAPE;
     if (p->B < 1 || p->H_q < 1 || p->H_kv < 1) return SE_ERR_INVALID_ARG;
+    if (p->B > 8192) return SE_ERR_UNSUPPORTED_SHAPE;      // the scoring kernel keeps three ints per request in shared memory
     if (p->H_q % p->H_kv != 0) return SE_ERR_INVALID_ARG;
     const int G = p->H_q / p->H_kv;
     if (G < 1 || G > 8) return SE_ERR_UNSUPPORTED_SHAPE;
@@ -143,7 +144,7 @@ const char *se_strerror(int code) {
     switch (code) {
         case SE_OK: return "ok";
         case SE_ERR_INVALID_ARG: return "invalid argument";
-        case SE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need page_size 16, D in {64,128}, 1 <= H_q/H_kv <= 8)";
+        case SE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need page_size 16, D in {64,128}, 1 <= H_q/H_kv <= 8, B <= 8192)";
         case SE_ERR_NULL_POINTER: return "required pointer is NULL";
         case SE_ERR_MISALIGNED: return "pointer is not 16-byte aligned";
         case SE_ERR_CUDA: return "CUDA runtime error";

@@ -54,6 +54,9 @@ def test_decode_split_plan():
     assert binding.se_decode_num_splits(few) == 2                 # 64 pairs: two CTAs per pair
     # 24 pairs: 148 / 24 = 6 CTAs per pair would need 24 clusters of 6 resident at once; only 22 are, so 5
     assert binding.se_decode_num_splits(binding.make_params(3, 32, 8, 128, 2048, 16384, 128)) == 5
+    # more requests than the scoring kernel's per-request tables hold: refused as a shape, not at launch
+    assert binding.se_workspace_bytes(binding.make_params(8192, 8, 8, 128, 64, 1 << 20, 16)) > 0
+    assert binding.se_workspace_bytes(binding.make_params(8193, 8, 8, 128, 64, 1 << 20, 16)) == 0
     assert binding.se_decode_num_splits(binding.make_params(24, 32, 8, 128, 2048, 16384, 128)) == 6   # 192 pairs: warps
     assert binding.se_decode_num_splits(many) == 1
     assert binding.se_decode_num_splits(binding.make_params(8, 32, 8, 96, 2048, 16384, 128)) == 0
