@@ -527,6 +527,22 @@ def test_every_launch_plan_against_the_oracle(pairs):
             compare(w_cpu, st)
 
 
+def test_maximum_batch_of_short_requests():
+    """The largest batch the library takes (8192 requests: the scoring kernel's per-request tables fill
+    a third of its shared memory, so it runs with one CTA per SM), one to five pages each."""
+    rng = np.random.default_rng(8192)
+    seq = [int(x) for x in rng.integers(1, 80, size=8192)]
+    seq[17] = 0
+    w_cpu = wl.build("maxbatch", 899, 0, seq, 2, 1, 64, 32, "cpu", permute_pool=True)
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w)
+    st.rebuild_meta()
+    st.step()
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    compare(w_cpu, st)
+
+
 def _run_shard(w, accum):
     st = binding.DecodeState(w)
     short = (w.seq_lens - 1).clamp(min=0).contiguous()
