@@ -106,19 +106,21 @@ score_kernel(const uint16_t *__restrict__ q, const uint8_t *meta, const uint8_t 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int H_q = H_kv * G;
 
-    // ---- per-CTA: units before each request (exclusive prefix over ceil(n_r/64)*H_kv)
+    // ---- per-CTA: units before each request (exclusive prefix over ceil(n_r/64)*H_kv).  All threads
+    // fetch the lengths (one round trip for up to 128 requests), one warp scans them.
+    for (int r = threadIdx.x; r < B; r += kScoreWarps * 32) {
+        const int len = __ldg(seq_lens + r);
+        int n = len > 0 ? (len + kPage - 1) / kPage : 0;
+        if (n > max_pages) n = max_pages;
+        npages[r] = n;
+        lens[r] = len;
+    }
+    __syncthreads();
     if (warp == 0) {
         int run = 0;
         for (int base = 0; base < B; base += 32) {
             const int r = base + lane;
-            int n = 0;
-            if (r < B) {
-                const int len = seq_lens[r];
-                n = len > 0 ? (len + kPage - 1) / kPage : 0;
-                if (n > max_pages) n = max_pages;
-                npages[r] = n;
-                lens[r] = len;
-            }
+            const int n = r < B ? npages[r] : 0;
             int u = ((n + kUnitPages - 1) / kUnitPages) * H_kv;
             int inc = u;
 #pragma unroll
