@@ -16,9 +16,9 @@
 // All NT threads of a CTA take part; thread t owns a run of consecutive pages (16-byte groups in slots
 // of its own), so thread order is page order and one prefix sum places the taken pages.  Keys and
 // histogram are accessed with explicit shared-space instructions.  Measured on a B200, 256 threads:
-// 4.2 K cycles for 128 pages, 6.4 K for 2048, 10 K for 4060, 15.6 K for 8192.  (A one-warp form of the
-// same algorithm took 7 K cycles for 264 pages and 46 K for 4060: too slow for the prologue of a
-// warp-per-pair attention kernel, which therefore keeps the top-k kernel.)
+// 4.8 K cycles for 128 pages, 6.3 K for 2048, 8.8 K for 4060, 12.1 K for 8192 with the CTA alone on its
+// SM.  (A one-warp form of the same algorithm took 7 K cycles for 264 pages and 46 K for 4060: too slow
+// for the prologue of a warp-per-pair attention kernel, which therefore keeps the top-k kernel.)
 #pragma once
 
 #include "se_device.cuh"
@@ -33,7 +33,7 @@ constexpr int kTopkList = 32;        // bins with up to this many keys are ranke
 struct TopkScratch {
     int hist[kTopkBins];             // indexed by 2047 - digit: prefix = keys above
     int tot[4][32];
-    int red[4][32];
+    int red[6][32];
     int res[8];
     uint32_t lkey[kTopkList];
     int lpage[kTopkList];
@@ -94,22 +94,28 @@ __device__ __forceinline__ int cta_topk(const float *row, int n, int k_pages, in
     const uint32_t kbase = smem_u32(keys) + (uint32_t)tid * (r4 | 1) * 16;
     const uint32_t hbase = smem_u32(S.hist);
 
-    // ---- load (all of the thread's groups in flight at once), scores -> keys, candidates, span
+    // ---- load, scores -> keys, candidates, span.  The loads are coalesced (group g = j*NT + tid, all of
+    // a thread's loads in flight at once); each group is then stored into the slots of its owner.
+    // Besides the span the threads reduce a lower bound of the threshold: `holders` threads loaded at
+    // least one candidate, so at least `holders` keys are >= tau = the smallest of those threads'
+    // maxima, and with k_eff <= holders the k_eff-th best key cannot lie below tau.
     uint32_t kmin = 0xffffffffu, kmax = 0u;
     int present = 0, forced = 0;
     {
-        const float4 *row4 = reinterpret_cast<const float4 *>(row) + tid * r4;
+        const float4 *row4 = reinterpret_cast<const float4 *>(row);
+        const uint32_t kb0 = smem_u32(keys);
         float4 v[kCtaTopkMaxGroups];
 #pragma unroll
         for (int j = 0; j < kCtaTopkMaxGroups; ++j)
-            if (j < my4) v[j] = __ldcg(row4 + j);
+            if (j < r4 && j * NT + tid < n4) v[j] = __ldcg(row4 + j * NT + tid);
 #pragma unroll
         for (int j = 0; j < kCtaTopkMaxGroups; ++j) {
-            if (j < my4) {
+            const int g = j * NT + tid;
+            if (j < r4 && g < n4) {
                 uint32_t k[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const int page = base + 4 * j + c;
+                    const int page = 4 * g + c;
                     const float ev = c == 0 ? v[j].x : c == 1 ? v[j].y : c == 2 ? v[j].z : v[j].w;
                     uint32_t key = page < n ? f32_key(ev) : kKeyAbsent;      // absent pages score -inf = kKeyAbsent
                     if (key != kKeyAbsent) {
@@ -124,35 +130,45 @@ __device__ __forceinline__ int cta_topk(const float *row, int n, int k_pages, in
                     }
                     k[c] = key;
                 }
-                sts128(kbase + j * 16, make_uint4(k[0], k[1], k[2], k[3]));
+                const int owner = g / r4;
+                sts128(kb0 + (uint32_t)(owner * (r4 | 1) + (g - owner * r4)) * 16, make_uint4(k[0], k[1], k[2], k[3]));
             }
         }
     }
 #pragma unroll
     for (int e = 0; e < BPT; ++e) S.hist[tid * BPT + e] = 0;
     if (tid == 0) S.ln = 0;
+    uint32_t tau = present > 0 ? kmax : 0xffffffffu;           // this thread's best candidate
+    int holders = present > 0 ? 1 : 0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         present += __shfl_xor_sync(kFull, present, o);
         forced += __shfl_xor_sync(kFull, forced, o);
+        holders += __shfl_xor_sync(kFull, holders, o);
         kmin = min(kmin, __shfl_xor_sync(kFull, kmin, o));
         kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
+        tau = min(tau, __shfl_xor_sync(kFull, tau, o));
     }
     if (lane == 0) {
         S.red[0][warp] = present;
         S.red[1][warp] = (int)kmin;
         S.red[2][warp] = (int)kmax;
         S.red[3][warp] = forced;
+        S.red[4][warp] = holders;
+        S.red[5][warp] = (int)tau;
     }
     __syncthreads();
     present = 0;
     forced = 0;
+    holders = 0;
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
         present += S.red[0][w];
         forced += S.red[3][w];
+        holders += S.red[4][w];
         kmin = min(kmin, (uint32_t)S.red[1][w]);
         kmax = max(kmax, (uint32_t)S.red[2][w]);
+        tau = min(tau, (uint32_t)S.red[5][w]);
     }
     forced = min(forced, k_max);
     const int k_eff = min(min(k_pages, k_max - forced), present);      // candidates to take
@@ -176,9 +192,10 @@ __device__ __forceinline__ int cta_topk(const float *row, int n, int k_pages, in
         T_key = kmin;
         ties = true;
     } else if (k_eff > 0) {
-        uint32_t lo = kmin;                              // the current span is [lo, lo + span)
-        uint32_t span = kmax - kmin + 1u;
-        int width = 32 - __clz(kmax - kmin);             // span <= 2^width
+        // keys below tau cannot be taken (see above): they stay out of the histogram, and the bins get finer
+        uint32_t lo = k_eff <= holders ? tau : kmin;     // the current span is [lo, lo + span)
+        uint32_t span = kmax - lo + 1u;
+        int width = 32 - __clz(kmax - lo);               // span <= 2^width
         for (int level = 0;; ++level) {
             const int sh = width > kTopkBinBits ? width - kTopkBinBits : 0;
             if (level > 0) {
@@ -290,33 +307,28 @@ __device__ __forceinline__ int cta_topk(const float *row, int n, int k_pages, in
         T_page = S.res[5];
     }
 
-    // ---- ordered compaction: count, prefix, write
-    int cnt = 0;
+    // ---- ordered compaction: mark (bit 4j + c of `taken` = page base + 4j + c), prefix, write
+    uint32_t taken = 0u;
     for (int j = 0; j < my4; ++j) {
         const uint4 v = lds128(kbase + j * 16);
         const uint32_t k[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            cnt += k[c] == kKeyForced || k[c] > T_key || (k[c] == T_key && base + 4 * j + c <= T_page);
+            if (k[c] == kKeyForced || k[c] > T_key || (k[c] == T_key && base + 4 * j + c <= T_page))
+                taken |= 1u << (4 * j + c);
     }
-    int pos = cta_excl_scan<NW>(cnt, S.tot[3], lane, warp);
+    int pos = cta_excl_scan<NW>(__popc(taken), S.tot[3], lane, warp);
     // the list is put together in shared memory (the caller's list, or the histogram, which is no longer
     // needed, when it is large enough) and written out with coalesced stores, padding included
     int *stage = list != nullptr ? list : (k_max <= kTopkBins ? S.hist : nullptr);
-    for (int j = 0; j < my4; ++j) {
-        const uint4 v = lds128(kbase + j * 16);
-        const uint32_t k[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const int page = base + 4 * j + c;
-            if (k[c] == kKeyForced || k[c] > T_key || (k[c] == T_key && page <= T_page)) {
-                if (pos < k_max) {
-                    if (stage != nullptr) stage[pos] = page;
-                    else out[pos] = page;
-                }
-                ++pos;
-            }
+    while (taken != 0u) {
+        const int page = base + __ffs(taken) - 1;
+        taken &= taken - 1u;
+        if (pos < k_max) {
+            if (stage != nullptr) stage[pos] = page;
+            else out[pos] = page;
         }
+        ++pos;
     }
     __syncthreads();
     if (out != nullptr) {
