@@ -1108,32 +1108,60 @@ decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         if (!active) return;
+        // (the partials are in L2; every thread issues all the loads it needs before it uses one, so the
+        // merge costs one round trip and not one per CTA of the pair)
+        constexpr int MAXC = 8;                  // a cluster has at most 8 CTAs
         if (tid < G) {
             const float *pr = partials + ((head0 + tid) * cpp) * C::PSTRIDE;
-            float mg = -INFINITY, lg = 0.f;
-            for (int s = 0; s < n_active; ++s) mg = fmaxf(mg, __ldcg(pr + (size_t)s * C::PSTRIDE + D));
-            for (int s = 0; s < n_active; ++s) {
-                const float ms = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
-                if (ms != -INFINITY) lg += exp2f(ms - mg) * __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
+            float ms[MAXC], ls[MAXC];
+#pragma unroll
+            for (int s = 0; s < MAXC; ++s) {
+                ms[s] = -INFINITY;
+                ls[s] = 0.f;
+                if (s < n_active) {
+                    ms[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
+                    ls[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
+                }
             }
-            s_M[tid] = mg;
-            s_L[tid] = lg;
+            float mg = -INFINITY, lg = 0.f;
+#pragma unroll
+            for (int s = 0; s < MAXC; ++s) mg = fmaxf(mg, ms[s]);
+#pragma unroll
+            for (int s = 0; s < MAXC; ++s)
+                if (ms[s] != -INFINITY) lg += exp2f(ms[s] - mg) * ls[s];
             const float l2 = lg > 0.f ? mg + log2f(lg) : -INFINITY;
             s_lse2[tid] = l2;
             if (cs == 0) lse[head0 + tid] = l2 * kLn2;
         }
-        __syncthreads();
         for (int e = cs * (kDecWarps * 32) + tid; e < G * D; e += n_active * kDecWarps * 32) {
             const int g = e / D, c = e - g * D;
             const float *pr = partials + ((head0 + g) * cpp) * C::PSTRIDE;
-            const float mg = s_M[g], lg = s_L[g];
-            float acc = 0.f;
-            for (int s = 0; s < n_active; ++s) {
-                const float ms = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
-                if (ms != -INFINITY) acc += exp2f(ms - mg) * __ldcg(pr + (size_t)s * C::PSTRIDE + c);
+            float ms[MAXC], ls[MAXC], vs[MAXC];
+#pragma unroll
+            for (int s = 0; s < MAXC; ++s) {
+                ms[s] = -INFINITY;
+                ls[s] = 0.f;
+                vs[s] = 0.f;
+                if (s < n_active) {
+                    ms[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + D);
+                    ls[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + D + 1);
+                    vs[s] = __ldcg(pr + (size_t)s * C::PSTRIDE + c);
+                }
+            }
+            float mg = -INFINITY, lg = 0.f, acc = 0.f;
+#pragma unroll
+            for (int s = 0; s < MAXC; ++s) mg = fmaxf(mg, ms[s]);
+#pragma unroll
+            for (int s = 0; s < MAXC; ++s) {
+                if (ms[s] != -INFINITY) {
+                    const float wgt = exp2f(ms[s] - mg);
+                    lg += wgt * ls[s];
+                    acc += wgt * vs[s];
+                }
             }
             out[(head0 + g) * D + c] = lg > 0.f ? acc / lg : 0.f;
         }
+        __syncthreads();                  // s_lse2
     } else {
         __syncthreads();                  // s_lse2
     }
@@ -1142,20 +1170,41 @@ decode_cta_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     // ---- H2O epilogue (Appendix A, H2O accumulated-score equation) for the tokens this CTA attended:
     // score_accum[slot] += sum over the group's heads of 2^(z - lse2); their logits were written by this
     // CTA's own warps.
-    for (int e = tid; e < (c_hi - c_lo) * kPage; e += kDecWarps * 32) {
-        const int i = c_lo + e / kPage, t = e % kPage;
-        const int b = list[i];
-        if (b < 0 || b >= n_r) continue;
-        const int pid = __ldg(page_table + (size_t)r * max_pages + b);
-        if (pid < 0 || pid >= P_phys) continue;
-        if (t >= min(kPage, len - b * kPage)) continue;
-        const float *z = zbuf + (((size_t)pair * k_max + i) * kPage + t) * GP;
-        float add = 0.f;
-        for (int gg = 0; gg < G; ++gg) {
-            const float zz = __ldcg(z + gg);
-            if (zz != -INFINITY) add += exp2f(zz - s_lse2[gg]);
+    // Four tokens per thread and round: their page-table entries and logits are fetched together, and
+    // the sum goes out as a reduction (nothing waits for the old value).
+    constexpr int EU = 4;
+    for (int e0 = tid; e0 < (c_hi - c_lo) * kPage; e0 += EU * kDecWarps * 32) {
+        int pid[EU], tt[EU];
+        float zz[EU][8];
+#pragma unroll
+        for (int u = 0; u < EU; ++u) {
+            const int e = e0 + u * kDecWarps * 32;
+            pid[u] = -1;
+            tt[u] = 0;
+#pragma unroll
+            for (int gg = 0; gg < 8; ++gg) zz[u][gg] = -INFINITY;
+            if (e < (c_hi - c_lo) * kPage) {
+                const int i = c_lo + e / kPage, t = e % kPage;
+                const int b = list[i];
+                if (b >= 0 && b < n_r && t < min(kPage, len - b * kPage)) {
+                    pid[u] = __ldg(page_table + (size_t)r * max_pages + b);
+                    tt[u] = t;
+                    const float *z = zbuf + (((size_t)pair * k_max + i) * kPage + t) * GP;
+#pragma unroll
+                    for (int gg = 0; gg < 8; ++gg)
+                        if (gg < G) zz[u][gg] = __ldcg(z + gg);
+                }
+            }
         }
-        score_accum[((size_t)pid * H_kv + h) * kPage + t] += add;
+#pragma unroll
+        for (int u = 0; u < EU; ++u) {
+            if (pid[u] < 0 || pid[u] >= P_phys) continue;
+            float add = 0.f;
+#pragma unroll
+            for (int gg = 0; gg < 8; ++gg)
+                if (zz[u][gg] != -INFINITY) add += exp2f(zz[u][gg] - s_lse2[gg]);
+            atomicAdd(score_accum + ((size_t)pid[u] * H_kv + h) * kPage + tt[u], add);
+        }
     }
 }
 
