@@ -53,6 +53,40 @@ def test_random_shapes(seed):
         compare(w_cpu, st, sink_pages=c["sink"], recent_pages=c["recent"])
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_many_requests(seed):
+    """The same sweep with up to 200 requests, so that every launch plan (cluster per pair, warp splits and
+    the merge kernel, two warps per pair, one warp per pair) meets random shapes, not only the listed ones."""
+    rng = np.random.default_rng(50000 + seed)
+    D = int(rng.choice([64, 128]))
+    H_kv = int(rng.choice([1, 2, 3, 4, 8]))
+    G = int(rng.integers(1, 9))
+    B = min(int(rng.choice([9, 20, 37, 50, 74, 75, 99, 120, 150, 200])), 1300 // H_kv)
+    hi = {"short": 80, "mixed": 900, "long": 3000}[str(rng.choice(["short", "mixed", "long"]))]
+    seq = [int(x) for x in rng.integers(1, hi + 1, size=B)]
+    if rng.random() < 0.3:
+        seq[int(rng.integers(0, B))] = 0
+    budget = 16 * int(rng.integers(1, 1 + max(1, min(120, max(seq) // 16 + 3))))
+    kw = dict(permute_pool=bool(rng.random() < 0.7), poison_tail=True,
+              prune_fraction=float(rng.choice([0.0, 0.0, 0.15, 0.5])),
+              outliers=bool(rng.random() < 0.3), with_score_accum=bool(rng.random() < 0.4),
+              spare_pages=int(rng.integers(0, 4)))
+    sink, recent = (int(rng.integers(0, 3)), int(rng.integers(0, 4))) if rng.random() < 0.3 else (0, 0)
+    w_cpu = wl.build("fuzzmany%d" % seed, 600 + seed, 0, seq, H_kv * G, H_kv, D, budget, "cpu", **kw)
+    w = w_cpu.to("cuda")
+    st = binding.DecodeState(w, sink_pages=sink, recent_pages=recent)
+    st.rebuild_meta()
+    u = w.score_accum.clone() if w.score_accum is not None else None
+    st.step(score_accum=u, fused=bool(seed % 2))
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    if u is not None:
+        compare(w_cpu, st, u_before=w_cpu.score_accum.numpy(), u_after=u.cpu().numpy(), sink_pages=sink,
+                recent_pages=recent)
+    else:
+        compare(w_cpu, st, sink_pages=sink, recent_pages=recent)
+
+
 @pytest.mark.parametrize("seed", range(20))
 def test_random_h2o_evictions(seed):
     from test_gpu_h2o import check_retain
