@@ -82,7 +82,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
 }
 
-// One-dimensional bulk asynchronous copy global -> shared (no tensor map, no multicast).
+// One-dimensional bulk asynchronous copy global -> shared of this CTA (no tensor map).
 // src, dst 16-byte aligned, bytes a multiple of 16; completion is signalled on `bar`.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile(
