@@ -351,7 +351,13 @@ __device__ __forceinline__ bool attend_range(WarpPipe &P, WarpAttn<D> &A, const 
             zp[(t0 + 8) * GP] = z[2];
             zp[(t0 + 9) * GP] = z[3];
         }
+        A.accumulate(Vs, nv_j, z, zero_chunk);
+        const int page_b = kObserve ? P.ent_b[ce] : 0;
+        __syncwarp();     // all lanes are done with this stage before it is refilled
+        ++ce;
+        top_up();
         if (kObserve) {
+            // (after the stage has been handed back for refilling: the scores only need z)
             // observation layer: s(j) = max over every query head of the logit (Appendix A, OmniKV
             // selection equation).  Here: max over the group's heads (rows gid; rows past the group
             // hold zero queries and are left out), then an atomic max over the kv-heads on the
@@ -365,18 +371,14 @@ __device__ __forceinline__ bool attend_range(WarpPipe &P, WarpAttn<D> &A, const 
                 v = fmaxf(v, __shfl_xor_sync(kFull, v, 16));
                 m4[e] = v;
             }
-            if (gid == 0) {
-                uint32_t *kp = a.keys_row + P.ent_b[ce] * kPage;
-                if (m4[0] > -INFINITY) atomicMax(kp + t0, f32_key(m4[0] * kLn2));
-                if (m4[1] > -INFINITY) atomicMax(kp + t0 + 1, f32_key(m4[1] * kLn2));
-                if (m4[2] > -INFINITY) atomicMax(kp + t0 + 8, f32_key(m4[2] * kLn2));
-                if (m4[3] > -INFINITY) atomicMax(kp + t0 + 9, f32_key(m4[3] * kLn2));
+            // after the butterfly every row holds the maxima; rows 0-3 send one token each, so the 16 tokens
+            // of the page leave as ONE atomic instruction over 64 contiguous bytes
+            if (gid < 4) {
+                const float mv = gid == 0 ? m4[0] : gid == 1 ? m4[1] : gid == 2 ? m4[2] : m4[3];
+                const int tok = t0 + (gid & 1) + 8 * (gid >> 1);
+                if (mv > -INFINITY) atomicMax(a.keys_row + page_b * kPage + tok, f32_key(mv * kLn2));
             }
         }
-        A.accumulate(Vs, nv_j, z, zero_chunk);
-        __syncwarp();     // all lanes are done with this stage before it is refilled
-        ++ce;
-        top_up();
     }
     return true;
 }
